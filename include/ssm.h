@@ -1,0 +1,138 @@
+/*
+ * ssm.h - C ABI of the B200 (sm_100a) S5 state-space layer library.
+ *
+ * The library evaluates, forward and backward, the diagonal complex linear
+ * state-space layer that the paper's world model uses as its sequence model
+ * (Sec. III-B "State-Space Models", Sec. IV-A "State-Space World Model"):
+ *
+ *     Abar = exp(Lambda Delta),  Bbar = Lambda^-1 (Abar - 1) B      (zero-order hold)
+ *     x_t  = (done_t ? 0 : Abar * x_{t-1}) + Bbar u_t ,   x_0 given or 0
+ *     y_t  = Re(C x_t) + D * u_t
+ *
+ * evaluated in parallel over the sequence with the associative scan of Sec. III-B
+ * (Eq. "scan".."full_scan") and its reset-aware form of Sec. IV-A
+ * (Eq. "sequence_scan_reset", "associative_reset").
+ *
+ * Conventions shared by every entry point
+ *  - All data pointers are DEVICE pointers owned by the caller; `shape` is a HOST
+ *    pointer.  The library allocates no memory, keeps no global state and never
+ *    synchronises the host (except ssm_check).  Work is enqueued on `stream`
+ *    (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *  - Tensors are dense, row-major, last index fastest.  Complex numbers are
+ *    interleaved (re, im) float pairs, bit-compatible with float2 / complex64.
+ *  - Parameters, states and their gradients are always fp32.  Only u, y, gy, du follow
+ *    shape->io_dtype (SSM_F32 or SSM_BF16).
+ *  - done[B,T] is uint8; nonzero at (b,t) means the episode ended before step t:
+ *    x_{t-1} is dropped (also x0 when t is the first step) and u_t still enters.
+ *  - Requirements: B,T >= 1; H and P positive multiples of 8; every pointer 16-byte
+ *    aligned.  Violations are detected on the host before any launch.
+ *  - Gradient convention for complex values under a real loss L:
+ *    g_z = dL/dRe(z) + i dL/dIm(z).  Gradient outputs are overwritten, not accumulated.
+ *  - Return value: SSM_OK (0) or a negative SSM_ERR_* code.  Nothing throws, aborts or
+ *    traps.  Device-side waits (the scan's inter-chunk carry) are bounded; if one gives
+ *    up it records SSM_ERR_TIMEOUT in the workspace header, which ssm_check reads back.
+ *  - Workspaces: the *_workspace_bytes functions give the size for a shape; the caller
+ *    passes a 256-byte aligned device buffer of at least that size.  A layer workspace
+ *    written by ssm_layer_fwd holds the residuals that ssm_layer_bwd reads, so it must
+ *    stay untouched between the two calls.  Calls sharing a workspace must not overlap.
+ */
+#ifndef SSM_B200_H
+#define SSM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct { float re, im; } ssm_c64;
+
+enum { SSM_F32 = 0, SSM_BF16 = 1 };
+
+enum {
+    SSM_OK = 0,
+    SSM_ERR_NULL = -1,       /* a required pointer is NULL                        */
+    SSM_ERR_SHAPE = -2,      /* B,T < 1, or H,P not positive multiples of 8        */
+    SSM_ERR_ALIGN = -3,      /* a pointer is not aligned as required               */
+    SSM_ERR_DTYPE = -4,      /* io_dtype is neither SSM_F32 nor SSM_BF16           */
+    SSM_ERR_WORKSPACE = -5,  /* workspace missing or too small                     */
+    SSM_ERR_CUDA = -6,       /* a CUDA runtime call or launch reported an error    */
+    SSM_ERR_TIMEOUT = -7     /* a bounded device-side wait gave up                 */
+};
+
+typedef struct {
+    int32_t B;         /* sequences in the batch                                   */
+    int32_t T;         /* steps per sequence (the paper's L)                       */
+    int32_t H;         /* width of u and y                                         */
+    int32_t P;         /* number of complex diagonal states                        */
+    int32_t io_dtype;  /* SSM_F32 or SSM_BF16: storage type of u, y, gy, du        */
+    int32_t reserved;  /* must be 0                                                */
+} ssm_shape;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* ssm_status_string(int status);
+
+/* Reads the workspace header back to the host (synchronises `stream`) and returns
+ * SSM_OK, or SSM_ERR_TIMEOUT if a kernel that used this workspace gave up a wait. */
+int ssm_check(const void* ws, void* stream);
+
+/* ---- discretisation: Sec. III-B, Eq. 3 (rule: zero-order hold) --------------------
+ * Abar[P] = exp(Lambda Delta);  Bbar[P,H] = ((Abar - 1)/Lambda) * B.  Lambda must be
+ * nonzero.  The P-sized part is evaluated in double precision and rounded once.
+ * Uses shape->H, shape->P. */
+int ssm_discretize(const ssm_shape* shape, const ssm_c64* Lambda /*[P]*/,
+                   const float* Delta /*[P]*/, const ssm_c64* Bc /*[P,H]*/,
+                   ssm_c64* Abar /*[P] out*/, ssm_c64* Bbar /*[P,H] out*/, void* stream);
+
+/* Adjoint of ssm_discretize: from gAbar[P], gBbar[P,H] to dLambda[P], dDelta[P], dB[P,H]. */
+int ssm_discretize_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta,
+                       const ssm_c64* Bc, const ssm_c64* gAbar, const ssm_c64* gBbar,
+                       ssm_c64* dLambda, float* dDelta, ssm_c64* dB, void* stream);
+
+/* ---- the scan: Sec. III-B Eq. "scan".."full_scan"; resets Sec. IV-A ---------------
+ * x[b,t,p] = (done[b,t] ? 0 : Abar[p] x[b,t-1,p]) + Bu[b,t,p],  x[b,-1,:] = x0[b,:] or 0.
+ * Long sequences are cut into chunks scanned concurrently; the carry between chunks
+ * uses the operator's associativity (decoupled look-back).  done, x0, xT may be NULL.
+ * x may alias Bu (in-place).  Uses shape->B, T, P. */
+size_t ssm_scan_workspace_bytes(const ssm_shape* shape);
+int ssm_scan_fwd(const ssm_shape* shape, const ssm_c64* Abar /*[P]*/,
+                 const ssm_c64* Bu /*[B,T,P]*/, const uint8_t* done /*[B,T] or NULL*/,
+                 const ssm_c64* x0 /*[B,P] or NULL*/, ssm_c64* x /*[B,T,P] out*/,
+                 ssm_c64* xT /*[B,P] out or NULL*/, void* ws, size_t ws_bytes, void* stream);
+
+/* Adjoint of ssm_scan_fwd (the same scan run backwards in time):
+ *   s_t = gx_t + (done_{t+1} ? 0 : conj(Abar) s_{t+1}),   s_{T+1} = gxT or 0
+ *   gBu = s;  gAbar[p] = sum_{b,t} (done_t ? 0 : s_t conj(x_{t-1}));
+ *   gx0 = done_1 ? 0 : conj(Abar) s_1.
+ * gxT, x0, done, gx0 may be NULL.  gBu may alias gx. */
+int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* done,
+                 const ssm_c64* x0, const ssm_c64* x /*[B,T,P] from the forward*/,
+                 const ssm_c64* gx /*[B,T,P]*/, const ssm_c64* gxT /*[B,P] or NULL*/,
+                 ssm_c64* gBu /*[B,T,P] out*/, ssm_c64* gAbar /*[P] out*/,
+                 ssm_c64* gx0 /*[B,P] out or NULL*/, void* ws, size_t ws_bytes, void* stream);
+
+/* ---- the whole layer: Sec. III-B Eq. 3 with the resets of Sec. IV-A ----------------
+ * Forward: discretise, Bu = Bbar u, scan, y = Re(C x) + D u.  u, y are [B,T,H] in
+ * io_dtype.  ws keeps the residuals (discretised parameters, states) for the backward. */
+size_t ssm_layer_workspace_bytes(const ssm_shape* shape);
+int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda /*[P]*/, const float* Delta /*[P]*/,
+                  const ssm_c64* Bc /*[P,H]*/, const ssm_c64* Cc /*[H,P]*/, const float* D /*[H]*/,
+                  const void* u /*[B,T,H] io*/, const uint8_t* done /*[B,T] or NULL*/,
+                  const ssm_c64* x0 /*[B,P] or NULL*/, void* y /*[B,T,H] io, out*/,
+                  ssm_c64* xT /*[B,P] out or NULL*/, void* ws, size_t ws_bytes, void* stream);
+
+/* Backward of L = sum(gy*y) + Re sum(conj(gxT) xT): needs the workspace ssm_layer_fwd
+ * filled for the same arguments.  Outputs: du[B,T,H] (io_dtype), dLambda[P], dDelta[P],
+ * dB[P,H], dC[H,P], dD[H], dx0[B,P] (or NULL).  gxT may be NULL. */
+int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta,
+                  const ssm_c64* Bc, const ssm_c64* Cc, const float* D, const void* u,
+                  const uint8_t* done, const ssm_c64* x0, const void* gy /*[B,T,H] io*/,
+                  const ssm_c64* gxT, void* ws, size_t ws_bytes, void* du,
+                  ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
+                  ssm_c64* dx0, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSM_B200_H */

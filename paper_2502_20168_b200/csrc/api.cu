@@ -1,0 +1,232 @@
+// C-ABI entry points (see include/ssm.h): argument checks, workspace layout, launch order.
+#include "kernels.h"
+
+using namespace ssm;
+
+#define SSM_API extern "C" __attribute__((visibility("default")))
+
+namespace {
+
+struct LayerPlan {
+    size_t hdr, Abar, Bbar, Bp, Bq, Cp, Cq, xs, gs, gAbar, gBbar, scan, part, dot, total;
+};
+
+size_t take(size_t& off, size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes, 256);
+    return at;
+}
+
+LayerPlan plan_layer(const ssm_shape& s) {
+    LayerPlan p{};
+    size_t off = 0;
+    const size_t BT = (size_t)s.B * s.T, PH = (size_t)s.P * s.H;
+    p.hdr = take(off, sizeof(WsHeader));
+    p.Abar = take(off, (size_t)s.P * 8);
+    p.Bbar = take(off, PH * 8);
+    p.Bp = take(off, 2 * PH * 4);
+    p.Bq = take(off, 2 * PH * 4);
+    p.Cp = take(off, 2 * PH * 4);
+    p.Cq = take(off, 2 * PH * 4);
+    p.xs = take(off, BT * s.P * 8);
+    p.gs = take(off, BT * s.P * 8);
+    p.gAbar = take(off, (size_t)s.P * 8);
+    p.gBbar = take(off, PH * 8);
+    p.scan = take(off, scan_scratch_bytes(s.B, s.T, s.P));
+    p.part = take(off, (size_t)gemm_nt_splits((int)BT) * 2 * PH * 4);
+    p.dot = take(off, dot_columns_tmp_floats((int)BT, s.H) * 4);
+    p.total = off;
+    return p;
+}
+
+template <typename T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(reinterpret_cast<char*>(ws) + off); }
+
+int check_ws(const void* ws, size_t have, size_t need) {
+    if (!ws) return SSM_ERR_WORKSPACE;
+    if (misaligned(ws, 256)) return SSM_ERR_ALIGN;
+    if (have < need) return SSM_ERR_WORKSPACE;
+    return SSM_OK;
+}
+
+}  // namespace
+
+SSM_API const char* ssm_status_string(int status) {
+    switch (status) {
+        case SSM_OK: return "ok";
+        case SSM_ERR_NULL: return "a required pointer is NULL";
+        case SSM_ERR_SHAPE: return "bad shape (B,T >= 1; H,P positive multiples of 8; reserved == 0)";
+        case SSM_ERR_ALIGN: return "a pointer is not aligned as required";
+        case SSM_ERR_DTYPE: return "io_dtype must be SSM_F32 or SSM_BF16";
+        case SSM_ERR_WORKSPACE: return "workspace missing or too small";
+        case SSM_ERR_CUDA: return "a CUDA call or kernel launch failed";
+        case SSM_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+SSM_API int ssm_check(const void* ws, void* stream) {
+    if (!ws) return SSM_ERR_NULL;
+    int status = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&status, ws, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SSM_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SSM_ERR_CUDA;
+    return status == 0 ? SSM_OK : SSM_ERR_TIMEOUT;
+}
+
+SSM_API int ssm_discretize(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
+                           ssm_c64* Abar, ssm_c64* Bbar, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Lambda || !Delta || !Bc || !Abar || !Bbar) return SSM_ERR_NULL;
+    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Abar) || misaligned(Bbar))
+        return SSM_ERR_ALIGN;
+    launch_discretize(shape->H, shape->P, (const float2*)Lambda, Delta, (const float2*)Bc, (float2*)Abar,
+                      (float2*)Bbar, (cudaStream_t)stream);
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_discretize_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta,
+                               const ssm_c64* Bc, const ssm_c64* gAbar, const ssm_c64* gBbar, ssm_c64* dLambda,
+                               float* dDelta, ssm_c64* dB, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Lambda || !Delta || !Bc || !gAbar || !gBbar || !dLambda || !dDelta || !dB) return SSM_ERR_NULL;
+    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(gAbar) || misaligned(gBbar) ||
+        misaligned(dLambda) || misaligned(dDelta) || misaligned(dB))
+        return SSM_ERR_ALIGN;
+    launch_discretize_bwd(shape->H, shape->P, (const float2*)Lambda, Delta, (const float2*)Bc,
+                          (const float2*)gAbar, (const float2*)gBbar, (float2*)dLambda, dDelta, (float2*)dB,
+                          (cudaStream_t)stream);
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API size_t ssm_scan_workspace_bytes(const ssm_shape* shape) {
+    if (check_shape(shape) != SSM_OK) return 0;
+    return sizeof(WsHeader) + scan_scratch_bytes(shape->B, shape->T, shape->P);
+}
+
+SSM_API int ssm_scan_fwd(const ssm_shape* shape, const ssm_c64* Abar, const ssm_c64* Bu, const uint8_t* done,
+                         const ssm_c64* x0, ssm_c64* x, ssm_c64* xT, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Abar || !Bu || !x) return SSM_ERR_NULL;
+    if (misaligned(Abar) || misaligned(Bu) || misaligned(x) || misaligned(x0) || misaligned(xT)) return SSM_ERR_ALIGN;
+    if (int rc = check_ws(ws, ws_bytes, ssm_scan_workspace_bytes(shape))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    int rc = launch_scan_fwd(shape->B, shape->T, shape->P, (const float2*)Abar, (const float2*)Bu, done,
+                             (const float2*)x0, (float2*)x, (float2*)xT, at<WsHeader>(ws, 0),
+                             at<char>(ws, sizeof(WsHeader)), st);
+    if (rc) return rc;
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* done, const ssm_c64* x0,
+                         const ssm_c64* x, const ssm_c64* gx, const ssm_c64* gxT, ssm_c64* gBu, ssm_c64* gAbar,
+                         ssm_c64* gx0, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Abar || !x || !gx || !gBu || !gAbar) return SSM_ERR_NULL;
+    if (misaligned(Abar) || misaligned(x) || misaligned(gx) || misaligned(gBu) || misaligned(gAbar) ||
+        misaligned(x0) || misaligned(gxT) || misaligned(gx0))
+        return SSM_ERR_ALIGN;
+    if (int rc = check_ws(ws, ws_bytes, ssm_scan_workspace_bytes(shape))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, done, (const float2*)x0,
+                             (const float2*)x, (const float2*)gx, (const float2*)gxT, (float2*)gBu,
+                             (float2*)gAbar, (float2*)gx0, at<WsHeader>(ws, 0), at<char>(ws, sizeof(WsHeader)), st);
+    if (rc) return rc;
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API size_t ssm_layer_workspace_bytes(const ssm_shape* shape) {
+    if (check_shape(shape) != SSM_OK) return 0;
+    return plan_layer(*shape).total;
+}
+
+SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
+                          const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
+                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Lambda || !Delta || !Bc || !Cc || !D || !u || !y) return SSM_ERR_NULL;
+    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Cc) || misaligned(D) ||
+        misaligned(u) || misaligned(y) || misaligned(x0) || misaligned(xT))
+        return SSM_ERR_ALIGN;
+    const ssm_shape& s = *shape;
+    const LayerPlan p = plan_layer(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf16 = s.io_dtype == SSM_BF16;
+    const int BT = s.B * s.T, P2 = 2 * s.P;
+
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
+                      at<float2>(ws, p.Bbar), st);
+    launch_pack_operands(s.H, s.P, bf16, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.Bp),
+                         at<void>(ws, p.Bq), at<void>(ws, p.Cp), at<void>(ws, p.Cq), st);
+    // Bu[m, 2p+c] = sum_h u[m,h] Bp[2p+c, h]
+    GemmTN g1{u, bf16, s.H, at<void>(ws, p.Bp), bf16, s.H, BT, P2, s.H, Epi::StoreF32,
+              at<void>(ws, p.xs), false, nullptr, nullptr, nullptr};
+    launch_gemm_tn(g1, st);
+    int rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.xs), done,
+                             (const float2*)x0, at<float2>(ws, p.xs), (float2*)xT, at<WsHeader>(ws, p.hdr),
+                             at<char>(ws, p.scan), st);
+    if (rc) return rc;
+    // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
+    GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.Cp), bf16, P2, BT, s.H, P2, Epi::AddDiagIo,
+              y, bf16, D, u, nullptr};
+    launch_gemm_tn(g2, st);
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
+                          const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
+                          const ssm_c64* x0, const void* gy, const ssm_c64* gxT, void* ws, size_t ws_bytes,
+                          void* du, ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
+                          ssm_c64* dx0, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Lambda || !Delta || !Bc || !Cc || !D || !u || !gy || !du || !dLambda || !dDelta || !dB || !dC || !dD)
+        return SSM_ERR_NULL;
+    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Cc) || misaligned(D) ||
+        misaligned(u) || misaligned(gy) || misaligned(du) || misaligned(dLambda) || misaligned(dDelta) ||
+        misaligned(dB) || misaligned(dC) || misaligned(dD) || misaligned(x0) || misaligned(gxT) || misaligned(dx0))
+        return SSM_ERR_ALIGN;
+    const ssm_shape& s = *shape;
+    const LayerPlan p = plan_layer(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf16 = s.io_dtype == SSM_BF16;
+    const int BT = s.B * s.T, P2 = 2 * s.P;
+
+    // gx[m, 2p+c] = sum_h gy[m,h] Cq[2p+c, h]          (= gy conj(C))
+    GemmTN g3{gy, bf16, s.H, at<void>(ws, p.Cq), bf16, s.H, BT, P2, s.H, Epi::StoreF32,
+              at<void>(ws, p.gs), false, nullptr, nullptr, nullptr};
+    launch_gemm_tn(g3, st);
+    int rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+                             at<float2>(ws, p.xs), at<float2>(ws, p.gs), (const float2*)gxT,
+                             at<float2>(ws, p.gs), at<float2>(ws, p.gAbar), (float2*)dx0,
+                             at<WsHeader>(ws, p.hdr), at<char>(ws, p.scan), st);
+    if (rc) return rc;
+    // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]      (= Re(Bbar^H s) + D gy)
+    GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.Bq), bf16, P2, BT, s.H, P2, Epi::AddDiagIo,
+              du, bf16, D, gy, nullptr};
+    launch_gemm_tn(g4, st);
+    // gBbar[p,h] = sum_m s[m,p] u[m,h]
+    const int splits = gemm_nt_splits(BT);
+    GemmNT g5{u, bf16, s.H, at<void>(ws, p.gs), false, P2, BT, splits, at<float>(ws, p.part)};
+    launch_gemm_nt(g5, st);
+    launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
+    // dC[h,p] = sum_m gy[m,h] conj(x[m,p])
+    GemmNT g6{gy, bf16, s.H, at<void>(ws, p.xs), false, P2, BT, splits, at<float>(ws, p.part)};
+    launch_gemm_nt(g6, st);
+    launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 1, (float2*)dC, st);
+    // dD[h] = sum_m gy[m,h] u[m,h]
+    launch_dot_columns(bf16, gy, u, BT, s.H, dD, at<float>(ws, p.dot), st);
+    launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
+                          at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}

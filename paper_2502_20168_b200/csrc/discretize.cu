@@ -1,0 +1,158 @@
+// Zero-order-hold discretisation of the diagonal SSM (Sec. III-B, Eq. 3) and its adjoint,
+// plus the packing of the discretised parameters into real GEMM operands.
+#include "kernels.h"
+
+namespace ssm {
+
+// exp(z) - 1 for z = a + ib without cancellation near z = 0.
+__device__ __forceinline__ void expm1_complex(double a, double b, double& re, double& im) {
+    double sb, cb;
+    sincos(b, &sb, &cb);
+    double sh = sin(0.5 * b);
+    re = expm1(a) * cb - 2.0 * sh * sh;
+    im = exp(a) * sb;
+}
+
+struct ZohTerms {
+    double ar, ai;  // Abar = exp(Lambda Delta)
+    double gr, gi;  // gamma = (Abar - 1) / Lambda
+};
+
+__device__ __forceinline__ ZohTerms zoh_terms(float2 lam, float dt) {
+    double lr = lam.x, li = lam.y, d = dt;
+    double er, ei;
+    expm1_complex(lr * d, li * d, er, ei);
+    double n = lr * lr + li * li;
+    ZohTerms z;
+    z.ar = er + 1.0;
+    z.ai = ei;
+    z.gr = (er * lr + ei * li) / n;
+    z.gi = (ei * lr - er * li) / n;
+    return z;
+}
+
+// One block per state p: Abar[p], Bbar[p, :] = gamma_p * B[p, :].
+__global__ void discretize_kernel(int H, const float2* __restrict__ Lambda, const float* __restrict__ Delta,
+                                  const float2* __restrict__ Bc, float2* __restrict__ Abar,
+                                  float2* __restrict__ Bbar) {
+    __shared__ float2 gamma_s;
+    const int p = blockIdx.x;
+    if (threadIdx.x == 0) {
+        ZohTerms z = zoh_terms(Lambda[p], Delta[p]);
+        Abar[p] = make_float2((float)z.ar, (float)z.ai);
+        gamma_s = make_float2((float)z.gr, (float)z.gi);
+    }
+    __syncthreads();
+    const float2 g = gamma_s;
+    for (int h = threadIdx.x; h < H; h += blockDim.x) Bbar[(size_t)p * H + h] = cmul(g, Bc[(size_t)p * H + h]);
+}
+
+// Adjoint.  One block per state p.
+__global__ void discretize_bwd_kernel(int H, const float2* __restrict__ Lambda, const float* __restrict__ Delta,
+                                      const float2* __restrict__ Bc, const float2* __restrict__ gAbar,
+                                      const float2* __restrict__ gBbar, float2* __restrict__ dLambda,
+                                      float* __restrict__ dDelta, float2* __restrict__ dB) {
+    __shared__ float2 gamma_s;
+    __shared__ float red[2][32];
+    const int p = blockIdx.x;
+    const float2 lam = Lambda[p];
+    const float dt = Delta[p];
+    ZohTerms z = {};
+    if (threadIdx.x == 0) {
+        z = zoh_terms(lam, dt);
+        gamma_s = make_float2((float)z.gr, (float)z.gi);
+    }
+    __syncthreads();
+    const float2 gc = cconj(gamma_s);
+    float sr = 0.f, si = 0.f;  // g_gamma = sum_h conj(B) gBbar
+    for (int h = threadIdx.x; h < H; h += blockDim.x) {
+        float2 gb = gBbar[(size_t)p * H + h];
+        float2 b = Bc[(size_t)p * H + h];
+        dB[(size_t)p * H + h] = cmul(gc, gb);
+        float2 t = cmul(cconj(b), gb);
+        sr += t.x;
+        si += t.y;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        sr += __shfl_xor_sync(0xffffffffu, sr, o);
+        si += __shfl_xor_sync(0xffffffffu, si, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        red[0][threadIdx.x >> 5] = sr;
+        red[1][threadIdx.x >> 5] = si;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double ggr = 0.0, ggi = 0.0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+            ggr += red[0][w];
+            ggi += red[1][w];
+        }
+        const double lr = lam.x, li = lam.y, d = dt;
+        const double gar = gAbar[p].x, gai = gAbar[p].y;
+        // dgamma/dLambda = (Delta Abar - gamma) / Lambda     (= (Delta Abar Lambda - (Abar-1)) / Lambda^2)
+        const double nr = d * z.ar - z.gr, ni = d * z.ai - z.gi;
+        const double n = lr * lr + li * li;
+        const double qr = (nr * lr + ni * li) / n, qi = (ni * lr - nr * li) / n;
+        // dLambda = conj(Delta Abar) gAbar + conj(dgamma/dLambda) g_gamma
+        double outr = d * (z.ar * gar + z.ai * gai) + (qr * ggr + qi * ggi);
+        double outi = d * (z.ar * gai - z.ai * gar) + (qr * ggi - qi * ggr);
+        dLambda[p] = make_float2((float)outr, (float)outi);
+        // dDelta = Re(conj(Lambda Abar) gAbar) + Re(conj(Abar) g_gamma)
+        const double lar = lr * z.ar - li * z.ai, lai = lr * z.ai + li * z.ar;
+        dDelta[p] = (float)((lar * gar + lai * gai) + (z.ar * ggr + z.ai * ggi));
+    }
+}
+
+// Real GEMM operands from the complex parameters (W = float or bf16):
+//   Bp[2p+c, h] = Bq[h, 2p+c] = c ? Im Bbar[p,h] : Re Bbar[p,h]
+//   Cp[h, 2p+c] = Cq[2p+c, h] = c ? -Im C[h,p]   : Re C[h,p]
+template <typename W>
+__global__ void pack_operands_kernel(int H, int P, const float2* __restrict__ Bbar, const float2* __restrict__ Cc,
+                                     W* __restrict__ Bp, W* __restrict__ Bq, W* __restrict__ Cp,
+                                     W* __restrict__ Cq) {
+    const size_t n = (size_t)P * H;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        {   // i indexes Bbar[p, h]
+            const int p = (int)(i / H), h = (int)(i % H);
+            const float2 v = Bbar[i];
+            Bp[(size_t)(2 * p) * H + h] = from_f32<W>(v.x);
+            Bp[(size_t)(2 * p + 1) * H + h] = from_f32<W>(v.y);
+            Bq[(size_t)h * 2 * P + 2 * p] = from_f32<W>(v.x);
+            Bq[(size_t)h * 2 * P + 2 * p + 1] = from_f32<W>(v.y);
+        }
+        {   // i indexes C[h, p]
+            const int h = (int)(i / P), p = (int)(i % P);
+            const float2 v = Cc[i];
+            Cp[(size_t)h * 2 * P + 2 * p] = from_f32<W>(v.x);
+            Cp[(size_t)h * 2 * P + 2 * p + 1] = from_f32<W>(-v.y);
+            Cq[(size_t)(2 * p) * H + h] = from_f32<W>(v.x);
+            Cq[(size_t)(2 * p + 1) * H + h] = from_f32<W>(-v.y);
+        }
+    }
+}
+
+void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc, float2* Abar,
+                       float2* Bbar, cudaStream_t st) {
+    discretize_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, Abar, Bbar);
+}
+
+void launch_discretize_bwd(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
+                           const float2* gAbar, const float2* gBbar, float2* dLambda, float* dDelta, float2* dB,
+                           cudaStream_t st) {
+    discretize_bwd_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, gAbar, gBbar, dLambda, dDelta, dB);
+}
+
+void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const float2* Cc, void* Bp, void* Bq,
+                          void* Cp, void* Cq, cudaStream_t st) {
+    const int threads = 256;
+    const int blocks = (int)(((size_t)P * H + threads - 1) / threads);
+    if (bf16)
+        pack_operands_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>(
+            H, P, Bbar, Cc, (__nv_bfloat16*)Bp, (__nv_bfloat16*)Bq, (__nv_bfloat16*)Cp, (__nv_bfloat16*)Cq);
+    else
+        pack_operands_kernel<float><<<blocks, threads, 0, st>>>(H, P, Bbar, Cc, (float*)Bp, (float*)Bq,
+                                                                 (float*)Cp, (float*)Cq);
+}
+
+}  // namespace ssm

@@ -1,0 +1,84 @@
+// Deterministic column reductions (parameter-gradient sums over all B*T rows).
+#include "kernels.h"
+
+namespace ssm {
+
+constexpr int kRowsPerBlock = 64;
+
+// block = 32 columns x 8 row lanes; grid.x = ceil(C/32), grid.y = row groups.
+// out[g, c] = sum of in[r, c] for r in group g.
+__global__ void colsum_kernel(const float* __restrict__ in, int R, int C, int rows_per_group,
+                              float* __restrict__ out) {
+    __shared__ float sm[8][33];
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    const int r0 = blockIdx.y * rows_per_group;
+    const int r1 = min(R, r0 + rows_per_group);
+    float acc = 0.f;
+    if (c < C)
+        for (int r = r0 + threadIdx.y; r < r1; r += 8) acc += in[(size_t)r * C + c];
+    sm[threadIdx.y][threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x];
+        out[(size_t)blockIdx.y * C + c] = t;
+    }
+}
+
+size_t colsum_tmp_floats(int R, int C) { return (size_t)((R + kRowsPerBlock - 1) / kRowsPerBlock) * C; }
+
+void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaStream_t st) {
+    dim3 blk(32, 8);
+    const int gx = (C + 31) / 32;
+    if (R <= kRowsPerBlock * 2) {
+        colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(in, R, C, R, out);
+        return;
+    }
+    const int groups = (R + kRowsPerBlock - 1) / kRowsPerBlock;
+    colsum_kernel<<<dim3(gx, groups), blk, 0, st>>>(in, R, C, kRowsPerBlock, tmp);
+    colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(tmp, groups, C, groups, out);
+}
+
+// part[g, c] = sum_{m in group g} a[m, c] * b[m, c]
+constexpr int kDotRows = 256;
+template <typename T>
+__global__ void dot_columns_kernel(const T* __restrict__ a, const T* __restrict__ b, int M, int C,
+                                   float* __restrict__ part) {
+    __shared__ float sm[8][33];
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    const int r0 = blockIdx.y * kDotRows;
+    const int r1 = min(M, r0 + kDotRows);
+    float acc = 0.f;
+    if (c < C)
+        for (int r = r0 + threadIdx.y; r < r1; r += 8)
+            acc = fmaf(to_f32<T>(a[(size_t)r * C + c]), to_f32<T>(b[(size_t)r * C + c]), acc);
+    sm[threadIdx.y][threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x];
+        part[(size_t)blockIdx.y * C + c] = t;
+    }
+}
+
+static inline int dot_groups(int M) { return (M + kDotRows - 1) / kDotRows; }
+
+size_t dot_columns_tmp_floats(int M, int C) {
+    const int g = dot_groups(M);
+    return (size_t)g * C + colsum_tmp_floats(g, C);
+}
+
+void launch_dot_columns(bool bf16, const void* a, const void* b, int M, int C, float* out, float* tmp,
+                        cudaStream_t st) {
+    const int g = dot_groups(M);
+    dim3 blk(32, 8), grid((C + 31) / 32, g);
+    if (bf16)
+        dot_columns_kernel<__nv_bfloat16><<<grid, blk, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, M, C, tmp);
+    else
+        dot_columns_kernel<float><<<grid, blk, 0, st>>>((const float*)a, (const float*)b, M, C, tmp);
+    launch_colsum(tmp, g, C, out, tmp + (size_t)g * C, st);
+}
+
+}  // namespace ssm

@@ -1,0 +1,87 @@
+"""Host-side plumbing around the binding: numpy <-> device buffers, output allocation.
+
+No arithmetic of the method happens here; every step of the layer runs in the
+CUDA library.  PyTorch is used only for device memory and streams.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as sb
+
+_IO = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+def to_dev(a, dtype=None, device="cuda"):
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.to(device).contiguous()
+
+
+def to_np(t):
+    if t is None:
+        return None
+    t = t.detach()
+    if t.dtype == torch.bfloat16:
+        t = t.float()
+    return t.cpu().numpy()
+
+
+class LayerBuffers:
+    """Device copies of one layer's inputs plus preallocated outputs and workspace."""
+
+    def __init__(self, d: dict, io_dtype: str, device="cuda", with_x0=False, with_gxT=False):
+        io = _IO[io_dtype]
+        B, T, H = d["u"].shape
+        P = d["Lambda"].shape[0]
+        self.shape = sb.make_shape(B, T, H, P, io_dtype)
+        self.io = io
+        self.Lambda = to_dev(d["Lambda"].astype(np.complex64), device=device)
+        self.Delta = to_dev(d["Delta"].astype(np.float32), device=device)
+        self.Bc = to_dev(d["Bc"].astype(np.complex64), device=device)
+        self.Cc = to_dev(d["Cc"].astype(np.complex64), device=device)
+        self.D = to_dev(d["D"].astype(np.float32), device=device)
+        self.u = to_dev(d["u"], io, device)
+        self.gy = to_dev(d["gy"], io, device) if d.get("gy") is not None else None
+        self.done = to_dev(d.get("done"), torch.uint8, device)
+        self.x0 = to_dev(d["x0"].astype(np.complex64), device=device) if with_x0 else None
+        self.gxT = to_dev(d["gxT"].astype(np.complex64), device=device) if with_gxT else None
+        c64 = dict(dtype=torch.complex64, device=device)
+        f32 = dict(dtype=torch.float32, device=device)
+        self.y = torch.empty((B, T, H), dtype=io, device=device)
+        self.xT = torch.empty((B, P), **c64)
+        self.du = torch.empty((B, T, H), dtype=io, device=device)
+        self.dLambda = torch.empty(P, **c64)
+        self.dDelta = torch.empty(P, **f32)
+        self.dB = torch.empty((P, H), **c64)
+        self.dC = torch.empty((H, P), **c64)
+        self.dD = torch.empty(H, **f32)
+        self.dx0 = torch.empty((B, P), **c64)
+        self.ws = sb.alloc_workspace(sb.ssm_layer_workspace_bytes(self.shape), device)
+
+    def forward(self, stream=None):
+        sb.ssm_layer_fwd(self.shape, self.Lambda, self.Delta, self.Bc, self.Cc, self.D, self.u, self.done,
+                         self.x0, self.y, self.xT, self.ws, stream)
+
+    def backward(self, stream=None):
+        sb.ssm_layer_bwd(self.shape, self.Lambda, self.Delta, self.Bc, self.Cc, self.D, self.u, self.done,
+                         self.x0, self.gy, self.gxT, self.ws, self.du, self.dLambda, self.dDelta, self.dB,
+                         self.dC, self.dD, self.dx0, stream)
+
+    def results(self) -> dict:
+        return {k: to_np(getattr(self, k)) for k in
+                ("y", "xT", "du", "dLambda", "dDelta", "dB", "dC", "dD", "dx0")}
+
+
+def run_layer(d: dict, io_dtype: str, with_x0=False, with_gxT=False) -> dict:
+    """Forward + backward of one layer on the current CUDA device; returns numpy results."""
+    buf = LayerBuffers(d, io_dtype, with_x0=with_x0, with_gxT=with_gxT)
+    buf.forward()
+    buf.backward()
+    sb.ssm_check(buf.ws)
+    torch.cuda.synchronize()
+    return buf.results()

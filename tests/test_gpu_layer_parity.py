@@ -1,0 +1,73 @@
+"""CUDA path vs the float64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2502_20168_b200 import inputs as I
+from tests.util import TOL, assert_close, compare_layer, oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+
+def run(w, with_x0=False, with_gxT=False, mutate=None):
+    from paper_2502_20168_b200 import harness
+    d = I.draw_layer(w, with_x0=with_x0, with_gxT=with_gxT)
+    if mutate:
+        mutate(d)
+    res = harness.run_layer(d, w.io_dtype, with_x0=with_x0, with_gxT=with_gxT)
+    ref = oracle_layer(d, with_x0, with_gxT)
+    keys = ["y", "xT", "du", "dLambda", "dDelta", "dB", "dC", "dD"] + (["dx0"] if with_x0 else [])
+    errs = compare_layer(res, ref, w.io_dtype, keys)
+    print(w.name, {k: f"{v:.1e}" for k, v in errs.items()})
+    return errs
+
+
+def test_c0_tiny_fp32():
+    run(I.C0)
+
+
+def test_c1_world_model_batch_fp32_with_resets():
+    run(I.C1)
+
+
+def test_c3_long_horizon_bf16():
+    run(I.C3)
+
+
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,H,P", [(3, 1, 8, 8), (2, 7, 24, 8), (5, 33, 40, 24), (2, 130, 72, 56),
+                                     (1, 300, 64, 128), (9, 64, 128, 64)])
+def test_ragged_shapes_with_resets_x0_and_gxT(io, B, T, H, P):
+    w = I.Workload("edge", B=B, T=T, H=H, P=P, io_dtype=io, p_done=0.15, seed=B * 1000 + T)
+
+    def flags(d):
+        d["done"][0, 0] = 1          # flag on the first step beats x0
+        d["done"][-1, -1] = 1        # flag on the last step
+    run(w, with_x0=True, with_gxT=True, mutate=flags)
+
+
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+def test_every_step_flagged_and_no_flags(io):
+    w = I.Workload("all", B=2, T=40, H=32, P=16, io_dtype=io, p_done=0.5, seed=5)
+    run(w, with_x0=True, mutate=lambda d: d["done"].fill(1))
+    run(w, with_x0=True, mutate=lambda d: d["done"].fill(0))
+    run(I.small_variant(w, p_done=0.0), with_gxT=True)
+
+
+def test_long_sequence_small_batch_fp32():
+    # long enough that the sequence is cut into many chunks with carries in between
+    w = I.Workload("long", B=2, T=2500, H=16, P=24, io_dtype="f32", p_done=0.003, seed=77)
+    run(w, with_x0=True, with_gxT=True)
+
+
+def test_forward_backward_twice_is_bitwise_repeatable_and_workspace_reusable():
+    import torch
+    from paper_2502_20168_b200 import harness
+    d = I.draw_layer(I.C1)
+    buf = harness.LayerBuffers(d, "f32")
+    buf.forward(); buf.backward()
+    first = buf.results()
+    buf.forward(); buf.backward()
+    torch.cuda.synchronize()
+    second = buf.results()
+    for k in ("y", "du", "dB", "dC", "dLambda", "dDelta", "dD"):
+        assert np.array_equal(first[k], second[k]), k
