@@ -164,10 +164,10 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
                       at<float2>(ws, p.Bbar), st);
-    launch_pack_operands(s.H, s.P, bf16, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.Bp),
+    launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.Bp),
                          at<void>(ws, p.Bq), at<void>(ws, p.Cp), at<void>(ws, p.Cq), st);
     // Bu[m, 2p+c] = sum_h u[m,h] Bp[2p+c, h]
-    GemmTN g1{u, bf16, s.H, at<void>(ws, p.Bp), bf16, s.H, BT, P2, s.H, Epi::StoreF32,
+    GemmTN g1{u, bf16, s.H, at<void>(ws, p.Bp), false, s.H, BT, P2, s.H, Epi::StoreF32,
               at<void>(ws, p.xs), false, nullptr, nullptr, nullptr};
     launch_gemm_tn(g1, st);
     int rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.xs), done,
@@ -175,7 +175,7 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
                              at<char>(ws, p.scan), st);
     if (rc) return rc;
     // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
-    GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.Cp), bf16, P2, BT, s.H, P2, Epi::AddDiagIo,
+    GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.Cp), false, P2, BT, s.H, P2, Epi::AddDiagIo,
               y, bf16, D, u, nullptr};
     launch_gemm_tn(g2, st);
     SSM_RETURN_IF_CUDA_ERROR();
@@ -202,7 +202,7 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     const int BT = s.B * s.T, P2 = 2 * s.P;
 
     // gx[m, 2p+c] = sum_h gy[m,h] Cq[2p+c, h]          (= gy conj(C))
-    GemmTN g3{gy, bf16, s.H, at<void>(ws, p.Cq), bf16, s.H, BT, P2, s.H, Epi::StoreF32,
+    GemmTN g3{gy, bf16, s.H, at<void>(ws, p.Cq), false, s.H, BT, P2, s.H, Epi::StoreF32,
               at<void>(ws, p.gs), false, nullptr, nullptr, nullptr};
     launch_gemm_tn(g3, st);
     int rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
@@ -211,7 +211,7 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
                              at<WsHeader>(ws, p.hdr), at<char>(ws, p.scan), st);
     if (rc) return rc;
     // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]      (= Re(Bbar^H s) + D gy)
-    GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.Bq), bf16, P2, BT, s.H, P2, Epi::AddDiagIo,
+    GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.Bq), false, P2, BT, s.H, P2, Epi::AddDiagIo,
               du, bf16, D, gy, nullptr};
     launch_gemm_tn(g4, st);
     // gBbar[p,h] = sum_m s[m,p] u[m,h]
