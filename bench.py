@@ -1,0 +1,313 @@
+#!/usr/bin/env python
+"""Benchmark of the SSM layer forward + backward (timesteps per second) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step is one forward + backward pass of the layer over one synthetic batch.  With N > 1
+(launched by torch.distributed.run) every rank runs the same workload on its own seeded
+batch: sequences are independent, so the path shards over the batch with no collective on
+the data path; the reported value is the sum over ranks divided by the slowest rank's time.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2502_20168_b200 import inputs as I  # noqa: E402
+
+METRIC = "ssm_layer_fwd_bwd_timesteps_per_sec"
+UNIT = "timesteps/s"
+DEFAULT_WORKLOAD = "c4_sweep_T1024_bf16"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# Algorithmic work of each internal stage per timestep (one (b,t) row): bytes for the
+# HBM-bound scans, flops for the projections (a real GEMM with K*N = 2*H*P per row).
+STAGE_MODEL = {
+    "gemm_Bu": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "scan_fwd": ("hbm", lambda H, P, s: 16.0 * P),
+    "gemm_y": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "gemm_gx": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "scan_bwd": ("hbm", lambda H, P, s: 24.0 * P),
+    "gemm_du": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "gemm_gBbar": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "gemm_gC": ("tensor", lambda H, P, s: 4.0 * H * P),
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu = gpu_index
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        hi = [v for v in sm if v >= 0.5 * max(sm)]
+        return {"sm_mhz": statistics.median(hi), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample_run(d, n_seq):
+    """Forward + backward of the float64 oracle on the first n_seq sequences; returns seconds."""
+    from oracle import ssm_oracle as O
+    done = None if d["done"] is None else d["done"][:n_seq]
+    u, gy = d["u"][:n_seq], d["gy"][:n_seq]
+    t0 = time.perf_counter()
+    O.ssm_layer_fwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], u, done, None)
+    O.ssm_layer_bwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], u, done, None, gy)
+    return time.perf_counter() - t0
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(w, d, budget_s=15.0):
+    """The oracle, as it stands, timed on a bounded sample of the workload's sequences."""
+    n = 1
+    dt = oracle_sample_run(d, n)
+    rate = n * w.T / dt
+    n = int(max(1, min(w.B, budget_s * rate / w.T)))
+    if n > 1:
+        dt = oracle_sample_run(d, n)
+    return {"value": n * w.T / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"first {n} of {w.B} sequences of {w.name} (T={w.T}, H={w.H}, P={w.P}), "
+                      f"float64 forward+backward once, {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = I.WORKLOADS[args.workload]
+    small = I.small_variant(w, B=min(w.B, 64))
+    d = I.draw_layer(small)
+    n = 1
+    dt = oracle_sample_run(d, 1)
+    per_step_budget = max(2.0, 120.0 / max(1, args.steps + args.warmup))
+    n = int(max(1, min(small.B, per_step_budget * (w.T / dt) / w.T)))
+    for _ in range(args.warmup):
+        oracle_sample_run(d, n)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_run(d, n)
+    total = time.perf_counter() - t0
+    value = n * w.T * args.steps / total
+    sample = f"first {n} sequences of {w.name} per step, float64 oracle forward+backward"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
+                   "sampled_sequences_per_step": n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2502_20168_b200 import binding as sb, harness
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = I.WORKLOADS[args.workload]
+    if w.n_layers != 1:
+        raise SystemExit("bench.py times single-layer workloads")
+    wr = I.small_variant(w, seed=w.seed + 1000 * rank)
+    d = I.draw_layer(wr)
+    buf = harness.LayerBuffers(d, w.io_dtype)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        buf.forward(stream)
+        buf.backward(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    sb.ssm_check(buf.ws)
+    barrier()
+
+    # ---- timed region: device-resident inputs, per-stage events recorded by the library ----
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = sb.ssm_launch_count()
+    sb.ssm_profile_begin()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    stages = sb.ssm_profile_end()
+    launches = sb.ssm_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    sb.ssm_check(buf.ws)
+
+    # ---- end to end: pinned host inputs in, results out, every step ----
+    host_in = {k: getattr(buf, k).cpu().pin_memory() for k in ("u", "gy")}
+    if buf.done is not None:
+        host_in["done"] = buf.done.cpu().pin_memory()
+    out_names = ("y", "du", "dLambda", "dDelta", "dB", "dC", "dD")
+    host_out = {k: torch.empty_like(getattr(buf, k), device="cpu").pin_memory() for k in out_names}
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def e2e_step():
+        for k, t in host_in.items():
+            getattr(buf, k).copy_(t, non_blocking=True)
+        step()
+        for k, t in host_out.items():
+            t.copy_(getattr(buf, k), non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        total_ts = w.timesteps * world
+        value = total_ts * args.steps / (ms * 1e-3)
+        s_io = 2 if w.io_dtype == "bf16" else 4
+        top = max((k for k in stages if k in STAGE_MODEL), key=lambda k: stages[k][1])
+        bound, work = STAGE_MODEL[top]
+        n_launch, top_ms = stages[top]
+        per_launch_s = top_ms * 1e-3 / n_launch
+        alg = work(w.H, w.P, s_io) * w.timesteps
+        if bound == "hbm":
+            achieved, peak, runit = alg / per_launch_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"
+        else:
+            achieved = alg / per_launch_s / 1e12
+            peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+            runit = "TFLOP/s"
+        stage_share = {k: round(v[1] / ms, 4) for k, v in stages.items()}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
+                       "p_done": w.p_done, "l2": "inputs larger than L2 (no flush)"
+                       if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}"},
+            "e2e": {"value": total_ts * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
+                         "frac": achieved / peak, "traffic": None, "peak_source": peak_kind,
+                         "ms_per_launch": per_launch_s * 1e3},
+            "stage_ms_per_step": {k: round(v[1] / args.steps, 4) for k, v in stages.items()},
+            "stage_share": stage_share,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, 64))))
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

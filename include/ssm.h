@@ -132,6 +132,17 @@ int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* De
                   ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
                   ssm_c64* dx0, void* stream);
 
+/* ---- measurement helpers (no counterpart in the paper; they never change results) ----
+ * ssm_launch_count: kernels this library has launched in this process so far.
+ * ssm_profile_begin / ssm_profile_end: between the two, every internal stage of the
+ * entry points above is bracketed by CUDA events on its stream.  ssm_profile_end
+ * synchronises the device and writes one line per stage, "name launches total_ms\n",
+ * into the HOST buffer `buf` (truncated to buf_bytes, NUL-terminated).  Process-wide,
+ * not thread-safe; creates CUDA events, allocates no device memory. */
+long long ssm_launch_count(void);
+int ssm_profile_begin(void);
+int ssm_profile_end(char* buf, size_t buf_bytes);
+
 #ifdef __cplusplus
 }
 #endif

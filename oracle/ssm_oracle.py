@@ -162,13 +162,14 @@ def ssm_layer_bwd(Lambda, Delta, Bc, Cc, D, u, done, x0, gy, gxT=None):
     x, _ = ssm_scan(Abar, u @ Bbar.T, done, x0)
     # y = Re(C x) + D u
     gx = gy @ np.conj(Cc)                                # [B,T,P]
-    dC = np.einsum("bth,btp->hp", gy, np.conj(x))
+    P = x.shape[-1]
+    dC = gy.reshape(-1, H).T @ np.conj(x).reshape(-1, P)      # dC[h,p] = sum_{b,t} gy[b,t,h] conj(x[b,t,p])
     dD = np.sum(gy * u, axis=(0, 1))
     # x = scan(Abar, Bu)
     s, gAbar, gx0 = ssm_scan_bwd(Abar, x, done, x0, gx, gxT)
     # Bu = Bbar u  (u real)
     du = D * gy + (s @ np.conj(Bbar)).real
-    gBbar = np.einsum("btp,bth->ph", s, u.astype(C128))
+    gBbar = s.reshape(-1, P).T @ u.reshape(-1, H)             # gBbar[p,h] = sum_{b,t} s[b,t,p] u[b,t,h]
     dLambda, dDelta, dB = zoh_discretize_bwd(Lambda, Delta, Bc, gAbar, gBbar)
     return {"du": du, "dLambda": dLambda, "dDelta": dDelta, "dB": dB, "dC": dC,
             "dD": dD, "dx0": gx0}

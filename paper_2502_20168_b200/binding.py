@@ -25,6 +25,7 @@ EXPORTS = (
     "ssm_status_string", "ssm_check", "ssm_discretize", "ssm_discretize_bwd",
     "ssm_scan_workspace_bytes", "ssm_scan_fwd", "ssm_scan_bwd",
     "ssm_layer_workspace_bytes", "ssm_layer_fwd", "ssm_layer_bwd",
+    "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end",
 )
 
 
@@ -67,6 +68,12 @@ def _load() -> ctypes.CDLL:
     lib.ssm_layer_fwd.argtypes = [S] + [P] * 11 + [c_size_t, P]
     lib.ssm_layer_bwd.restype = c_int
     lib.ssm_layer_bwd.argtypes = [S] + [P] * 11 + [c_size_t] + [P] * 8
+    lib.ssm_launch_count.restype = ctypes.c_longlong
+    lib.ssm_launch_count.argtypes = []
+    lib.ssm_profile_begin.restype = c_int
+    lib.ssm_profile_begin.argtypes = []
+    lib.ssm_profile_end.restype = c_int
+    lib.ssm_profile_end.argtypes = [ctypes.c_char_p, c_size_t]
     return lib
 
 
@@ -160,6 +167,25 @@ def ssm_layer_bwd(shape, Lambda, Delta, Bc, Cc, D, u, done, x0, gy, gxT, ws, du,
                            _ptr(done), _ptr(x0), _ptr(gy), _ptr(gxT), _ptr(ws), _nbytes(ws), _ptr(du),
                            _ptr(dLambda), _ptr(dDelta), _ptr(dB), _ptr(dC), _ptr(dD), _ptr(dx0),
                            _stream(stream)), "ssm_layer_bwd")
+
+
+def ssm_launch_count() -> int:
+    return int(_lib.ssm_launch_count())
+
+
+def ssm_profile_begin() -> None:
+    _ok(_lib.ssm_profile_begin(), "ssm_profile_begin")
+
+
+def ssm_profile_end() -> dict:
+    """Stage name -> (launches, total milliseconds) recorded since ssm_profile_begin."""
+    buf = ctypes.create_string_buffer(1 << 16)
+    _ok(_lib.ssm_profile_end(buf, len(buf)), "ssm_profile_end")
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, count, ms = line.split()
+        out[name] = (int(count), float(ms))
+    return out
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:

@@ -162,22 +162,27 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     const int BT = s.B * s.T, P2 = 2 * s.P;
 
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    {
+    StageTimer tm("discretize_pack", st);
     launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
                       at<float2>(ws, p.Bbar), st);
     launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.Bp),
                          at<void>(ws, p.Bq), at<void>(ws, p.Cp), at<void>(ws, p.Cq), st);
+    }
     // Bu[m, 2p+c] = sum_h u[m,h] Bp[2p+c, h]
     GemmTN g1{u, bf16, s.H, at<void>(ws, p.Bp), false, s.H, BT, P2, s.H, Epi::StoreF32,
               at<void>(ws, p.xs), false, nullptr, nullptr, nullptr};
-    launch_gemm_tn(g1, st);
+    { StageTimer tm("gemm_Bu", st); launch_gemm_tn(g1, st); }
+    StageTimer* tscan = new StageTimer("scan_fwd", st);
     int rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.xs), done,
                              (const float2*)x0, at<float2>(ws, p.xs), (float2*)xT, at<WsHeader>(ws, p.hdr),
                              at<char>(ws, p.scan), st);
+    delete tscan;
     if (rc) return rc;
     // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
     GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.Cp), false, P2, BT, s.H, P2, Epi::AddDiagIo,
               y, bf16, D, u, nullptr};
-    launch_gemm_tn(g2, st);
+    { StageTimer tm("gemm_y", st); launch_gemm_tn(g2, st); }
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;
 }
@@ -204,26 +209,35 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     // gx[m, 2p+c] = sum_h gy[m,h] Cq[2p+c, h]          (= gy conj(C))
     GemmTN g3{gy, bf16, s.H, at<void>(ws, p.Cq), false, s.H, BT, P2, s.H, Epi::StoreF32,
               at<void>(ws, p.gs), false, nullptr, nullptr, nullptr};
-    launch_gemm_tn(g3, st);
+    { StageTimer tm("gemm_gx", st); launch_gemm_tn(g3, st); }
+    StageTimer* tscan = new StageTimer("scan_bwd", st);
     int rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
                              at<float2>(ws, p.xs), at<float2>(ws, p.gs), (const float2*)gxT,
                              at<float2>(ws, p.gs), at<float2>(ws, p.gAbar), (float2*)dx0,
                              at<WsHeader>(ws, p.hdr), at<char>(ws, p.scan), st);
+    delete tscan;
     if (rc) return rc;
     // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]      (= Re(Bbar^H s) + D gy)
     GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.Bq), false, P2, BT, s.H, P2, Epi::AddDiagIo,
               du, bf16, D, gy, nullptr};
-    launch_gemm_tn(g4, st);
+    { StageTimer tm("gemm_du", st); launch_gemm_tn(g4, st); }
     // gBbar[p,h] = sum_m s[m,p] u[m,h]
     const int splits = gemm_nt_splits(BT);
     GemmNT g5{u, bf16, s.H, at<void>(ws, p.gs), false, P2, BT, splits, at<float>(ws, p.part)};
-    launch_gemm_nt(g5, st);
-    launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
+    {
+        StageTimer tm("gemm_gBbar", st);
+        launch_gemm_nt(g5, st);
+        launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
+    }
     // dC[h,p] = sum_m gy[m,h] conj(x[m,p])
     GemmNT g6{gy, bf16, s.H, at<void>(ws, p.xs), false, P2, BT, splits, at<float>(ws, p.part)};
-    launch_gemm_nt(g6, st);
-    launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 1, (float2*)dC, st);
+    {
+        StageTimer tm("gemm_gC", st);
+        launch_gemm_nt(g6, st);
+        launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 1, (float2*)dC, st);
+    }
     // dD[h] = sum_m gy[m,h] u[m,h]
+    StageTimer tm("gD_and_discretize_bwd", st);
     launch_dot_columns(bf16, gy, u, BT, s.H, dD, at<float>(ws, p.dot), st);
     launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
                           at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);

@@ -50,6 +50,17 @@ inline int check_shape(const ssm_shape* s) {
 }
 inline bool misaligned(const void* p, size_t a = 16) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
+// Measurement hooks (profile.cu): launch counter and optional per-stage event timing.
+void count_launch(int n = 1);
+class StageTimer {
+  public:
+    StageTimer(const char* name, cudaStream_t st);
+    ~StageTimer();
+  private:
+    cudaStream_t st_;
+    int idx_;
+};
+
 #define SSM_RETURN_IF_CUDA_ERROR()                              \
     do {                                                        \
         if (cudaPeekAtLastError() != cudaSuccess) {             \

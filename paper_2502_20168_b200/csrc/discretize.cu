@@ -134,12 +134,14 @@ __global__ void pack_operands_kernel(int H, int P, const float2* __restrict__ Bb
 
 void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc, float2* Abar,
                        float2* Bbar, cudaStream_t st) {
+    count_launch();
     discretize_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, Abar, Bbar);
 }
 
 void launch_discretize_bwd(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
                            const float2* gAbar, const float2* gBbar, float2* dLambda, float* dDelta, float2* dB,
                            cudaStream_t st) {
+    count_launch();
     discretize_bwd_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, gAbar, gBbar, dLambda, dDelta, dB);
 }
 
@@ -147,6 +149,7 @@ void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const flo
                           void* Cp, void* Cq, cudaStream_t st) {
     const int threads = 256;
     const int blocks = (int)(((size_t)P * H + threads - 1) / threads);
+    count_launch();
     if (bf16)
         pack_operands_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>(
             H, P, Bbar, Cc, (__nv_bfloat16*)Bp, (__nv_bfloat16*)Bq, (__nv_bfloat16*)Cp, (__nv_bfloat16*)Cq);

@@ -89,6 +89,7 @@ gemm_tn_kernel(const TA* __restrict__ A, int lda, const TB* __restrict__ Bm, int
 template <typename TA, typename TB>
 static void dispatch_tn(const GemmTN& g, cudaStream_t st) {
     dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM);
+    count_launch();
     EpiArgs e{g.out, g.diag, g.skip, g.add, g.N};
     const TA* A = (const TA*)g.A;
     const TB* Bm = (const TB*)g.Bm;
@@ -164,6 +165,7 @@ void launch_gemm_nt(const GemmNT& g, cudaStream_t st) {
     int kps = (g.K + g.splits - 1) / g.splits;
     kps = (kps + TK - 1) / TK * TK;
     dim3 grid((g.J + TN - 1) / TN, (g.I + TM - 1) / TM, g.splits);
+    count_launch();
     if (g.a_bf16 && g.b_bf16)
         gemm_nt_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, kGemmThreads, 0, st>>>((const __nv_bfloat16*)g.A, g.I, (const __nv_bfloat16*)g.Bm, g.J, g.K, kps, g.part);
     else if (g.a_bf16)
@@ -191,6 +193,7 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
 void launch_splitk_reduce(const float* part, int splits, int I, int J, int mode, float2* out, cudaStream_t st) {
     const int threads = 256;
     const int blocks = (int)(((size_t)I * J + threads - 1) / threads);
+    count_launch();
     splitk_reduce_kernel<<<blocks, threads, 0, st>>>(part, splits, I, J, mode, (float*)out);
 }
 

@@ -32,10 +32,12 @@ void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaSt
     dim3 blk(32, 8);
     const int gx = (C + 31) / 32;
     if (R <= kRowsPerBlock * 2) {
+        count_launch();
         colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(in, R, C, R, out);
         return;
     }
     const int groups = (R + kRowsPerBlock - 1) / kRowsPerBlock;
+    count_launch(2);
     colsum_kernel<<<dim3(gx, groups), blk, 0, st>>>(in, R, C, kRowsPerBlock, tmp);
     colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(tmp, groups, C, groups, out);
 }
@@ -74,6 +76,7 @@ void launch_dot_columns(bool bf16, const void* a, const void* b, int M, int C, f
                         cudaStream_t st) {
     const int g = dot_groups(M);
     dim3 blk(32, 8), grid((C + 31) / 32, g);
+    count_launch();
     if (bf16)
         dot_columns_kernel<__nv_bfloat16><<<grid, blk, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, M, C, tmp);
     else

@@ -132,6 +132,7 @@ int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Bu, c
     (void)scratch;
     const int P2 = P / 2;
     const int blocks = (int)(((size_t)B * P2 + kScanThreads - 1) / kScanThreads);
+    count_launch();
     scan_fwd_seq_kernel<<<blocks, kScanThreads, 0, st>>>(B, T, P2, (const float4*)Abar, (const float4*)Bu, done,
                                                          (const float4*)x0, (float4*)x, (float4*)xT);
     return SSM_OK;
@@ -145,6 +146,7 @@ int launch_scan_bwd(int B, int T, int P, const float2* Abar, const uint8_t* done
     float* part = (float*)scratch;
     float* tmp = part + (size_t)B * P * 2;
     const int blocks = (int)(((size_t)B * P2 + kScanThreads - 1) / kScanThreads);
+    count_launch();
     scan_bwd_seq_kernel<<<blocks, kScanThreads, 0, st>>>(B, T, P2, (const float4*)Abar, done, (const float4*)x0,
                                                          (const float4*)x, (const float4*)gx, (const float4*)gxT,
                                                          (float4*)gBu, (float4*)part, (float4*)gx0);
