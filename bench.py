@@ -125,12 +125,12 @@ def blas_threads() -> int:
 
 def cpu_baseline(w, d, budget_s=15.0):
     """The oracle, as it stands, timed on a bounded sample of the workload's sequences."""
-    n = 1
+    have = d["u"].shape[0]
+    n = min(have, 4)
     dt = oracle_sample_run(d, n)
     rate = n * w.T / dt
-    n = int(max(1, min(w.B, budget_s * rate / w.T)))
-    if n > 1:
-        dt = oracle_sample_run(d, n)
+    n = int(max(1, min(have, budget_s * rate / w.T)))
+    dt = oracle_sample_run(d, n)
     return {"value": n * w.T / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "sample": f"first {n} of {w.B} sequences of {w.name} (T={w.T}, H={w.H}, P={w.P}), "
                       f"float64 forward+backward once, {dt:.1f} s"}
@@ -141,12 +141,12 @@ def run_reference(args):
     if rank != 0:
         return
     w = I.WORKLOADS[args.workload]
-    small = I.small_variant(w, B=min(w.B, 64))
+    small = I.small_variant(w, B=min(w.B, max(1, 65536 // w.T)))
     d = I.draw_layer(small)
-    n = 1
-    dt = oracle_sample_run(d, 1)
-    per_step_budget = max(2.0, 120.0 / max(1, args.steps + args.warmup))
-    n = int(max(1, min(small.B, per_step_budget * (w.T / dt) / w.T)))
+    n0 = min(small.B, 4)
+    dt = oracle_sample_run(d, n0)
+    per_step_budget = max(1.0, 120.0 / max(1, args.steps + args.warmup))
+    n = int(max(1, min(small.B, per_step_budget * n0 / dt)))
     for _ in range(args.warmup):
         oracle_sample_run(d, n)
     t0 = time.perf_counter()
@@ -303,7 +303,7 @@ def main():
             "stage_share": stage_share,
         }
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, 64))))
+            line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, max(1, 262144 // w.T)))))
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
