@@ -58,7 +58,8 @@ enum {
     SSM_ERR_DTYPE = -4,      /* io_dtype is neither SSM_F32 nor SSM_BF16           */
     SSM_ERR_WORKSPACE = -5,  /* workspace missing or too small                     */
     SSM_ERR_CUDA = -6,       /* a CUDA runtime call or launch reported an error    */
-    SSM_ERR_TIMEOUT = -7     /* a bounded device-side wait gave up                 */
+    SSM_ERR_TIMEOUT = -7,    /* a bounded device-side wait gave up                 */
+    SSM_ERR_TOO_LARGE = -8   /* problem exceeds a built-in fixed-size buffer       */
 };
 
 typedef struct {
@@ -111,6 +112,29 @@ int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* don
                  const ssm_c64* gx /*[B,T,P]*/, const ssm_c64* gxT /*[B,P] or NULL*/,
                  ssm_c64* gBu /*[B,T,P] out*/, ssm_c64* gAbar /*[P] out*/,
                  ssm_c64* gx0 /*[B,P] out or NULL*/, void* ws, size_t ws_bytes, void* stream);
+
+/* ---- reverse scan without a caller workspace (the paper has no counterpart) ---------
+ * Same result as ssm_scan_bwd, for callers that have no scratch buffer to pass and are
+ * not in a position to get one: code running where device allocation is off limits, for
+ * example a plug-in inside a host framework that owns all device memory through its own
+ * pool and forbids cudaMalloc (which also stalls the whole device while it runs), a
+ * real-time loop with a memory budget fixed at start-up, or a callback that may not call
+ * allocating CUDA routines.  The scratch lives in a fixed array of
+ * SSM_STATIC_SCRATCH_BYTES inside the library's device image, so every GPU that loads the
+ * library gives up that much memory until the process ends.  The call allocates nothing.
+ *  - Limit: problems whose scan scratch (ssm_scan_workspace_bytes(shape)) exceeds
+ *    SSM_STATIC_SCRATCH_BYTES are refused with SSM_ERR_TOO_LARGE before anything runs.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  The library clears what has to start at
+ *    zero on every call, but two calls whose GPU work overlaps (different streams) race on
+ *    it: issue them on one stream or order them yourself.
+ * Arguments are those of ssm_scan_bwd minus the workspace. */
+#define SSM_STATIC_SCRATCH_BYTES (8u << 20)
+int ssm_scan_bwd_static(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* done,
+                        const ssm_c64* x0, const ssm_c64* x, const ssm_c64* gx,
+                        const ssm_c64* gxT, ssm_c64* gBu, ssm_c64* gAbar, ssm_c64* gx0,
+                        void* stream);
 
 /* ---- the whole layer: Sec. III-B Eq. 3 with the resets of Sec. IV-A ----------------
  * Forward: discretise, Bu = Bbar u, scan, y = Re(C x) + D u.  u, y are [B,T,H] in

@@ -25,8 +25,10 @@ EXPORTS = (
     "ssm_status_string", "ssm_check", "ssm_discretize", "ssm_discretize_bwd",
     "ssm_scan_workspace_bytes", "ssm_scan_fwd", "ssm_scan_bwd",
     "ssm_layer_workspace_bytes", "ssm_layer_fwd", "ssm_layer_bwd",
-    "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end",
+    "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static",
 )
+SSM_ERR_TOO_LARGE = -8
+SSM_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class ssm_shape(Structure):
@@ -68,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.ssm_layer_fwd.argtypes = [S] + [P] * 11 + [c_size_t, P]
     lib.ssm_layer_bwd.restype = c_int
     lib.ssm_layer_bwd.argtypes = [S] + [P] * 11 + [c_size_t] + [P] * 8
+    lib.ssm_scan_bwd_static.restype = c_int
+    lib.ssm_scan_bwd_static.argtypes = [S] + [P] * 10
     lib.ssm_launch_count.restype = ctypes.c_longlong
     lib.ssm_launch_count.argtypes = []
     lib.ssm_profile_begin.restype = c_int
@@ -149,6 +153,14 @@ def ssm_scan_bwd(shape, Abar, done, x0, x, gx, gxT, gBu, gAbar, gx0, ws, stream=
     _ok(_lib.ssm_scan_bwd(byref(shape), _ptr(Abar), _ptr(done), _ptr(x0), _ptr(x), _ptr(gx), _ptr(gxT),
                           _ptr(gBu), _ptr(gAbar), _ptr(gx0), _ptr(ws), _nbytes(ws), _stream(stream)),
         "ssm_scan_bwd")
+
+
+def ssm_scan_bwd_static(shape, Abar, done, x0, x, gx, gxT, gBu, gAbar, gx0, stream=None) -> None:
+    """ssm_scan_bwd for callers that cannot allocate a workspace: the library's own fixed
+    scratch array is used instead (shared by all calls on the device, so do not overlap them;
+    raises SsmError(SSM_ERR_TOO_LARGE) when the shape needs more than SSM_STATIC_SCRATCH_BYTES)."""
+    _ok(_lib.ssm_scan_bwd_static(byref(shape), _ptr(Abar), _ptr(done), _ptr(x0), _ptr(x), _ptr(gx), _ptr(gxT),
+                                 _ptr(gBu), _ptr(gAbar), _ptr(gx0), _stream(stream)), "ssm_scan_bwd_static")
 
 
 def ssm_layer_workspace_bytes(shape) -> int:

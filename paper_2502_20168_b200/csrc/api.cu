@@ -61,6 +61,7 @@ SSM_API const char* ssm_status_string(int status) {
         case SSM_ERR_WORKSPACE: return "workspace missing or too small";
         case SSM_ERR_CUDA: return "a CUDA call or kernel launch failed";
         case SSM_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case SSM_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in static buffer holds";
         default: return "unknown status";
     }
 }
