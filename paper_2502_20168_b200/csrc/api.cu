@@ -7,8 +7,14 @@ using namespace ssm;
 
 namespace {
 
+// Workspace of one layer.  Two paths:
+//  * tensor-core path (bf16 I/O and tile-sized H, P): projections on tcgen05, states Bu / g_x
+//    in one fp32 buffer, x and s kept as bf16 pairs;
+//  * CUDA-core path (fp32 I/O, or odd shapes): fp32 weights and states throughout.
 struct LayerPlan {
-    size_t hdr, Abar, Bbar, Bp, Bq, Cp, Cq, xs, gs, gAbar, gBbar, scan, part, dot, total;
+    bool tc;
+    int splits;
+    size_t hdr, Abar, Bbar, W0, W1, W2, W3, f32buf, xs, gs, gAbar, gBbar, scan, part, dot, total;
 };
 
 size_t take(size_t& off, size_t bytes) {
@@ -21,19 +27,34 @@ LayerPlan plan_layer(const ssm_shape& s) {
     LayerPlan p{};
     size_t off = 0;
     const size_t BT = (size_t)s.B * s.T, PH = (size_t)s.P * s.H;
+    const int P2 = 2 * s.P;
+    p.tc = s.io_dtype == SSM_BF16 && tc_tn_supported((int)BT, P2, s.H, true) &&
+           tc_tn_supported((int)BT, s.H, P2, false) && tc_nt_supported(s.H, P2);
+    p.splits = p.tc ? tc_nt_splits((int)BT, s.H, P2) : gemm_nt_splits((int)BT);
     p.hdr = take(off, sizeof(WsHeader));
     p.Abar = take(off, (size_t)s.P * 8);
     p.Bbar = take(off, PH * 8);
-    p.Bp = take(off, 2 * PH * 4);
-    p.Bq = take(off, 2 * PH * 4);
-    p.Cp = take(off, 2 * PH * 4);
-    p.Cq = take(off, 2 * PH * 4);
-    p.xs = take(off, BT * s.P * 8);
-    p.gs = take(off, BT * s.P * 8);
+    if (p.tc) {
+        p.W0 = take(off, 4 * PH * 2);   // hi/lo stacked Bbar operand  [4P, H] bf16
+        p.W1 = take(off, 4 * PH * 2);   // hi/lo stacked conj(C) operand [4P, H] bf16
+        p.W2 = take(off, 2 * PH * 2);   // Cp [H, 2P] bf16
+        p.W3 = take(off, 2 * PH * 2);   // Bq [H, 2P] bf16
+        p.f32buf = take(off, BT * s.P * 8);   // Bu (forward), then g_x (backward)
+        p.xs = take(off, BT * s.P * 8);       // x as two bf16 planes (hi, lo)
+        p.gs = take(off, BT * s.P * 8);       // s as two bf16 planes (hi, lo)
+    } else {
+        p.W0 = take(off, 2 * PH * 4);   // Bp [2P, H]
+        p.W1 = take(off, 2 * PH * 4);   // Cq [2P, H]
+        p.W2 = take(off, 2 * PH * 4);   // Cp [H, 2P]
+        p.W3 = take(off, 2 * PH * 4);   // Bq [H, 2P]
+        p.f32buf = off;                 // unused
+        p.xs = take(off, BT * s.P * 8); // Bu, overwritten in place by x
+        p.gs = take(off, BT * s.P * 8); // g_x, overwritten in place by s
+    }
     p.gAbar = take(off, (size_t)s.P * 8);
     p.gBbar = take(off, PH * 8);
     p.scan = take(off, scan_scratch_bytes(s.B, s.T, s.P));
-    p.part = take(off, (size_t)gemm_nt_splits((int)BT) * 2 * PH * 4);
+    p.part = take(off, (size_t)p.splits * 2 * PH * 4);
     p.dot = take(off, dot_columns_tmp_floats((int)BT, s.H) * 4);
     p.total = off;
     return p;
@@ -115,8 +136,9 @@ SSM_API int ssm_scan_fwd(const ssm_shape* shape, const ssm_c64* Abar, const ssm_
     if (int rc = check_ws(ws, ws_bytes, ssm_scan_workspace_bytes(shape))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    StageTimer tm("scan_fwd", st);
     int rc = launch_scan_fwd(shape->B, shape->T, shape->P, (const float2*)Abar, (const float2*)Bu, done,
-                             (const float2*)x0, (float2*)x, (float2*)xT, at<WsHeader>(ws, 0),
+                             (const float2*)x0, x, false, (float2*)xT, at<WsHeader>(ws, 0),
                              at<char>(ws, sizeof(WsHeader)), st);
     if (rc) return rc;
     SSM_RETURN_IF_CUDA_ERROR();
@@ -134,9 +156,10 @@ SSM_API int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint
     if (int rc = check_ws(ws, ws_bytes, ssm_scan_workspace_bytes(shape))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
-    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, done, (const float2*)x0,
-                             (const float2*)x, (const float2*)gx, (const float2*)gxT, (float2*)gBu,
-                             (float2*)gAbar, (float2*)gx0, at<WsHeader>(ws, 0), at<char>(ws, sizeof(WsHeader)), st);
+    StageTimer tm("scan_bwd", st);
+    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, done, (const float2*)x0, x, false,
+                             (const float2*)gx, (const float2*)gxT, gBu, false, (float2*)gAbar, (float2*)gx0,
+                             at<WsHeader>(ws, 0), at<char>(ws, sizeof(WsHeader)), st);
     if (rc) return rc;
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;
@@ -161,29 +184,61 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     cudaStream_t st = (cudaStream_t)stream;
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T, P2 = 2 * s.P;
+    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    int rc = SSM_OK;
 
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     {
-    StageTimer tm("discretize_pack", st);
-    launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
-                      at<float2>(ws, p.Bbar), st);
-    launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.Bp),
-                         at<void>(ws, p.Bq), at<void>(ws, p.Cp), at<void>(ws, p.Cq), st);
+        StageTimer tm("discretize_pack", st);
+        launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
+                          at<float2>(ws, p.Bbar), st);
+        if (p.tc)
+            launch_pack_operands_tc(s.H, s.P, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+                                    at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
+        else
+            launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+                                 at<void>(ws, p.W3), at<void>(ws, p.W2), at<void>(ws, p.W1), st);
     }
-    // Bu[m, 2p+c] = sum_h u[m,h] Bp[2p+c, h]
-    GemmTN g1{u, bf16, s.H, at<void>(ws, p.Bp), false, s.H, BT, P2, s.H, Epi::StoreF32,
-              at<void>(ws, p.xs), false, nullptr, nullptr, nullptr};
-    { StageTimer tm("gemm_Bu", st); launch_gemm_tn(g1, st); }
-    StageTimer* tscan = new StageTimer("scan_fwd", st);
-    int rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.xs), done,
-                             (const float2*)x0, at<float2>(ws, p.xs), (float2*)xT, at<WsHeader>(ws, p.hdr),
-                             at<char>(ws, p.scan), st);
-    delete tscan;
-    if (rc) return rc;
-    // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
-    GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.Cp), false, P2, BT, s.H, P2, Epi::AddDiagIo,
-              y, bf16, D, u, nullptr};
-    { StageTimer tm("gemm_y", st); launch_gemm_tn(g2, st); }
+    if (p.tc) {
+        {   // Bu[m, 2p+c] = sum_h u[m,h] Bbar_c[p,h]     (weights as hi + lo bf16)
+            StageTimer tm("gemm_Bu", st);
+            GemmTcTN g{u, at<void>(ws, p.W0), BT, P2, s.H, true, true, at<void>(ws, p.f32buf),
+                       nullptr, nullptr, nullptr, hdr};
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+        {
+            StageTimer tm("scan_fwd", st);
+            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.f32buf), done,
+                                 (const float2*)x0, at<void>(ws, p.xs), true, (float2*)xT, hdr,
+                                 at<char>(ws, p.scan), st);
+            if (rc) return rc;
+        }
+        {   // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
+            StageTimer tm("gemm_y", st);
+            GemmTcTN g{at<void>(ws, p.xs), at<void>(ws, p.W2), BT, s.H, P2, false, false, y, D, u, nullptr, hdr};
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+    } else {
+        {
+            StageTimer tm("gemm_Bu", st);
+            GemmTN g1{u, bf16, s.H, at<void>(ws, p.W0), false, s.H, BT, P2, s.H, Epi::StoreF32,
+                      at<void>(ws, p.xs), false, nullptr, nullptr, nullptr};
+            launch_gemm_tn(g1, st);
+        }
+        {
+            StageTimer tm("scan_fwd", st);
+            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.xs), done,
+                                 (const float2*)x0, at<void>(ws, p.xs), false, (float2*)xT, hdr,
+                                 at<char>(ws, p.scan), st);
+            if (rc) return rc;
+        }
+        {
+            StageTimer tm("gemm_y", st);
+            GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.W2), false, P2, BT, s.H, P2, Epi::AddDiagIo,
+                      y, bf16, D, u, nullptr};
+            launch_gemm_tn(g2, st);
+        }
+    }
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;
 }
@@ -206,42 +261,83 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     cudaStream_t st = (cudaStream_t)stream;
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T, P2 = 2 * s.P;
+    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    float* part = at<float>(ws, p.part);
+    const size_t plane = (size_t)BT * s.P * 4;   // bytes of one bf16 plane of a state tensor
+    int rc = SSM_OK;
 
-    // gx[m, 2p+c] = sum_h gy[m,h] Cq[2p+c, h]          (= gy conj(C))
-    GemmTN g3{gy, bf16, s.H, at<void>(ws, p.Cq), false, s.H, BT, P2, s.H, Epi::StoreF32,
-              at<void>(ws, p.gs), false, nullptr, nullptr, nullptr};
-    { StageTimer tm("gemm_gx", st); launch_gemm_tn(g3, st); }
-    StageTimer* tscan = new StageTimer("scan_bwd", st);
-    int rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
-                             at<float2>(ws, p.xs), at<float2>(ws, p.gs), (const float2*)gxT,
-                             at<float2>(ws, p.gs), at<float2>(ws, p.gAbar), (float2*)dx0,
-                             at<WsHeader>(ws, p.hdr), at<char>(ws, p.scan), st);
-    delete tscan;
-    if (rc) return rc;
-    // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]      (= Re(Bbar^H s) + D gy)
-    GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.Bq), false, P2, BT, s.H, P2, Epi::AddDiagIo,
-              du, bf16, D, gy, nullptr};
-    { StageTimer tm("gemm_du", st); launch_gemm_tn(g4, st); }
-    // gBbar[p,h] = sum_m s[m,p] u[m,h]
-    const int splits = gemm_nt_splits(BT);
-    GemmNT g5{u, bf16, s.H, at<void>(ws, p.gs), false, P2, BT, splits, at<float>(ws, p.part)};
-    {
-        StageTimer tm("gemm_gBbar", st);
-        launch_gemm_nt(g5, st);
-        launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
+    if (p.tc) {
+        {   // gx[m, 2p+c] = sum_h gy[m,h] conj(C)_c[h,p]   (weights as hi + lo bf16)
+            StageTimer tm("gemm_gx", st);
+            GemmTcTN g{gy, at<void>(ws, p.W1), BT, P2, s.H, true, true, at<void>(ws, p.f32buf),
+                       nullptr, nullptr, nullptr, hdr};
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+        {
+            StageTimer tm("scan_bwd", st);
+            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+                                 at<void>(ws, p.xs), true, at<float2>(ws, p.f32buf), (const float2*)gxT,
+                                 at<void>(ws, p.gs), true, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
+                                 at<char>(ws, p.scan), st);
+            if (rc) return rc;
+        }
+        {   // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]
+            StageTimer tm("gemm_du", st);
+            GemmTcTN g{at<void>(ws, p.gs), at<void>(ws, p.W3), BT, s.H, P2, false, false, du, D, gy, nullptr, hdr};
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+        {   // gBbar[p,h] = sum_m s[m,p] u[m,h]
+            StageTimer tm("gemm_gBbar", st);
+            GemmTcNT g{u, s.H, at<void>(ws, p.gs), at<void>(ws, p.gs + plane), P2, BT, p.splits, part, hdr};
+            if ((rc = launch_gemm_tc_nt(g, st))) return rc;
+            launch_splitk_reduce(part, p.splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
+        }
+        {   // dC[h,p] = sum_m gy[m,h] conj(x[m,p])
+            StageTimer tm("gemm_gC", st);
+            GemmTcNT g{gy, s.H, at<void>(ws, p.xs), at<void>(ws, p.xs + plane), P2, BT, p.splits, part, hdr};
+            if ((rc = launch_gemm_tc_nt(g, st))) return rc;
+            launch_splitk_reduce(part, p.splits, s.H, P2, 1, (float2*)dC, st);
+        }
+    } else {
+        {
+            StageTimer tm("gemm_gx", st);
+            GemmTN g3{gy, bf16, s.H, at<void>(ws, p.W1), false, s.H, BT, P2, s.H, Epi::StoreF32,
+                      at<void>(ws, p.gs), false, nullptr, nullptr, nullptr};
+            launch_gemm_tn(g3, st);
+        }
+        {
+            StageTimer tm("scan_bwd", st);
+            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+                                 at<void>(ws, p.xs), false, at<float2>(ws, p.gs), (const float2*)gxT,
+                                 at<void>(ws, p.gs), false, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
+                                 at<char>(ws, p.scan), st);
+            if (rc) return rc;
+        }
+        {
+            StageTimer tm("gemm_du", st);
+            GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.W3), false, P2, BT, s.H, P2, Epi::AddDiagIo,
+                      du, bf16, D, gy, nullptr};
+            launch_gemm_tn(g4, st);
+        }
+        {
+            StageTimer tm("gemm_gBbar", st);
+            GemmNT g5{u, bf16, s.H, at<void>(ws, p.gs), false, P2, BT, p.splits, part};
+            launch_gemm_nt(g5, st);
+            launch_splitk_reduce(part, p.splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
+        }
+        {
+            StageTimer tm("gemm_gC", st);
+            GemmNT g6{gy, bf16, s.H, at<void>(ws, p.xs), false, P2, BT, p.splits, part};
+            launch_gemm_nt(g6, st);
+            launch_splitk_reduce(part, p.splits, s.H, P2, 1, (float2*)dC, st);
+        }
     }
-    // dC[h,p] = sum_m gy[m,h] conj(x[m,p])
-    GemmNT g6{gy, bf16, s.H, at<void>(ws, p.xs), false, P2, BT, splits, at<float>(ws, p.part)};
-    {
-        StageTimer tm("gemm_gC", st);
-        launch_gemm_nt(g6, st);
-        launch_splitk_reduce(at<float>(ws, p.part), splits, s.H, P2, 1, (float2*)dC, st);
+    {   // dD[h] = sum_m gy[m,h] u[m,h];  then the adjoint of the discretisation
+        StageTimer tm("gD_and_discretize_bwd", st);
+        launch_dot_columns(bf16, gy, u, BT, s.H, dD, at<float>(ws, p.dot), st);
+        launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
+                              at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);
     }
-    // dD[h] = sum_m gy[m,h] u[m,h]
-    StageTimer tm("gD_and_discretize_bwd", st);
-    launch_dot_columns(bf16, gy, u, BT, s.H, dD, at<float>(ws, p.dot), st);
-    launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
-                          at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;
 }

@@ -132,6 +132,52 @@ __global__ void pack_operands_kernel(int H, int P, const float2* __restrict__ Bb
     }
 }
 
+// Operands of the tensor-core path.  A weight w is carried as hi = bf16(w), lo = bf16(w - hi)
+// in the two projections that feed the states (Bu and g_x), so that the states see ~16
+// mantissa bits of the parameters.  Logical row n of the [2P, H] operand goes to rows
+// (n/128)*256 + n%128 (hi) and (n/128)*256 + 128 + n%128 (lo) of the stacked [4P, H] matrix.
+__device__ __forceinline__ void store_split(__nv_bfloat16* W, int H, int n, int h, float w) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+    const size_t r = (size_t)(n >> 7) * 256 + (n & 127);
+    W[r * H + h] = hi;
+    W[(r + 128) * H + h] = lo;
+}
+
+__global__ void pack_operands_tc_kernel(int H, int P, const float2* __restrict__ Bbar, const float2* __restrict__ Cc,
+                                        __nv_bfloat16* __restrict__ WsB, __nv_bfloat16* __restrict__ WsC,
+                                        __nv_bfloat16* __restrict__ Cp, __nv_bfloat16* __restrict__ Bq) {
+    const size_t n = (size_t)P * H;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        {   // i indexes Bbar[p, h]
+            const int p = (int)(i / H), h = (int)(i % H);
+            const float2 v = Bbar[i];
+            store_split(WsB, H, 2 * p, h, v.x);
+            store_split(WsB, H, 2 * p + 1, h, v.y);
+            Bq[(size_t)h * 2 * P + 2 * p] = __float2bfloat16_rn(v.x);
+            Bq[(size_t)h * 2 * P + 2 * p + 1] = __float2bfloat16_rn(v.y);
+        }
+        {   // i indexes C[h, p]
+            const int h = (int)(i / P), p = (int)(i % P);
+            const float2 v = Cc[i];
+            Cp[(size_t)h * 2 * P + 2 * p] = __float2bfloat16_rn(v.x);
+            Cp[(size_t)h * 2 * P + 2 * p + 1] = __float2bfloat16_rn(-v.y);
+            store_split(WsC, H, 2 * p, h, v.x);
+            store_split(WsC, H, 2 * p + 1, h, -v.y);
+        }
+    }
+}
+
+void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
+                             void* Cp, void* Bq, cudaStream_t st) {
+    const int threads = 256;
+    const int blocks = (int)(((size_t)P * H + threads - 1) / threads);
+    count_launch();
+    pack_operands_tc_kernel<<<blocks, threads, 0, st>>>(H, P, Bbar, Cc, (__nv_bfloat16*)Wsplit_B,
+                                                        (__nv_bfloat16*)Wsplit_C, (__nv_bfloat16*)Cp,
+                                                        (__nv_bfloat16*)Bq);
+}
+
 void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc, float2* Abar,
                        float2* Bbar, cudaStream_t st) {
     count_launch();

@@ -1,0 +1,594 @@
+// bf16 projections on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
+// memory, operands staged in shared memory by TMA).  Two kernels:
+//
+//  * gemm_tc_tn_kernel: out[m, n] = sum_k A[m, k] * W[n, k]  (both operands K-contiguous).
+//    Persistent, one CTA per SM walking 128 x 256 accumulator tiles.  A = activations or states
+//    [B*T, K]; W = packed parameters.  With kSplitW the 256 accumulator columns of a tile hold
+//    the products with the high and the low bf16 halves of 128 weight rows, summed in the
+//    epilogue (weights then carry ~16 mantissa bits; see pack_operands_tc_kernel).
+//  * gemm_tc_nt_kernel: part[s, i, j] = sum_{m in slice s} A[m, i] * Bm[m, j]  (both operands
+//    contiguous in the output index, i.e. MN-major), split over the B*T rows.
+//
+// Warp roles in both: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
+// warps 2..5 drain accumulators (one TMEM lane quarter each).  Every mbarrier wait is bounded;
+// a wait that gives up raises a CTA-wide abort flag, the status word of the workspace header
+// is set, tensor memory is released and the kernel returns.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "kernels.h"
+
+namespace ssm {
+namespace tc {
+
+constexpr int BM = 128;   // accumulator rows per tile = TMEM lanes
+constexpr int BN = 256;   // accumulator columns per tile
+constexpr int BK = 64;    // bf16 elements per shared-memory row: 128 bytes, one swizzle span
+constexpr int UK = 16;    // K extent of one tcgen05.mma of kind::f16
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;
+constexpr int kBBytes = BN * BK * 2;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;  // two accumulator buffers of BN columns
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (base lane + i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (128-byte swizzle).  Fields: start address >> 4 in bits
+// [0,14), leading byte offset >> 4 in [16,30), stride byte offset >> 4 in [32,46), descriptor
+// version 1 in [46,48), swizzle mode 2 (128 B) in [61,64).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// K-major tile: rows of 128 bytes, groups of 8 rows 1024 bytes apart (leading offset unused).
+__device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr) { return smem_desc(addr, 16, 1024); }
+// MN-major tile made of [BK rows][64 elements] blocks: 64-element blocks 8192 bytes apart,
+// groups of 8 k-rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_mnmajor(uint32_t addr) { return smem_desc(addr, BK * 128, 1024); }
+
+// Instruction descriptor: D = f32 (bits [4,6) = 1), A = B = bf16 (bits [7,10), [10,13) = 1),
+// operand majors in bits 15 / 16 (0 = K), N >> 3 in [17,23), M >> 4 in [24,29).
+__host__ __device__ constexpr uint32_t instr_desc(int m, int n, int a_mn, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct Smem {
+    uint8_t* tiles;       // 1024-byte aligned
+    uint32_t full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_slot;   // where tcgen05.alloc writes the base address
+    volatile int* abort_flag;
+    volatile uint32_t* tmem_slot_ptr;
+};
+
+__device__ __forceinline__ Smem carve_smem(uint8_t* raw) {
+    Smem s;
+    uintptr_t base = (reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023;
+    s.tiles = reinterpret_cast<uint8_t*>(base);
+    uint8_t* bars = s.tiles + (size_t)kStages * kStageBytes;
+    for (int i = 0; i < kStages; ++i) {
+        s.full[i] = smem_u32(bars + 8 * i);
+        s.empty[i] = smem_u32(bars + 8 * (kStages + i));
+    }
+    for (int i = 0; i < 2; ++i) {
+        s.tmem_full[i] = smem_u32(bars + 8 * (2 * kStages + i));
+        s.tmem_empty[i] = smem_u32(bars + 8 * (2 * kStages + 2 + i));
+    }
+    s.tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(bars + 8 * (2 * kStages + 4));
+    s.tmem_slot = smem_u32(bars + 8 * (2 * kStages + 4));
+    s.abort_flag = reinterpret_cast<volatile int*>(bars + 8 * (2 * kStages + 4) + 4);
+    return s;
+}
+
+// Common prologue: barriers, tensor memory.  Returns the TMEM base address.
+__device__ __forceinline__ uint32_t prologue(const Smem& s, int warp, int lane) {
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(s.full[i], 1);
+            mbar_init(s.empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s.tmem_full[i], 1);
+            mbar_init(s.tmem_empty[i], 128);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(s.tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    (void)lane;
+    return *s.tmem_slot_ptr;
+}
+
+__device__ __forceinline__ void epilogue_exit(const Smem& s, int warp, uint32_t tmem_base, WsHeader* hdr) {
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && *s.abort_flag && hdr) hdr->status = SSM_ERR_TIMEOUT;
+}
+
+// ---------------------------------------------------------------------------------------------
+// TN kernel
+// ---------------------------------------------------------------------------------------------
+struct TnParams {
+    int M;            // rows of A / out
+    int n_tiles;      // accumulator tiles along N (each BN columns of W rows)
+    int k_blocks;     // K / BK
+    int ldo;          // leading dimension of out (and skip/add)
+    void* out;        // fp32 (kEpi == 0) or bf16 (kEpi == 1)
+    const float* diag;
+    const __nv_bfloat16* skip;
+    const __nv_bfloat16* add;
+    WsHeader* hdr;
+};
+
+// kEpi 0: store fp32;  kEpi 1: out = bf16(acc + diag[n] * skip[m, n] (+ add[m, n])).
+// kSplitW: columns [0,128) and [128,256) of the accumulator tile are the hi and lo weight
+// halves of the same 128 output columns.
+template <int kEpi, bool kSplitW>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tmem_base = prologue(s, warp, lane);
+    const int m_tiles = (p.M + BM - 1) / BM;
+    const int total = m_tiles * p.n_tiles;
+    constexpr int kOutCols = kSplitW ? BN / 2 : BN;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmW);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+                const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag))) break;
+                    mbar_expect_tx(s.full[stage], kStageBytes);
+                    const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
+                    tma_load_2d(a_dst, &tmA, s.full[stage], kb * BK, m0);
+                    tma_load_2d(a_dst + kABytes, &tmW, s.full[stage], kb * BK, n0);
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(BM, BN, 0, 0);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+                if (!(ok = mbar_wait(s.tmem_empty[acc], acc_phase ^ 1u, s.abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageBytes);
+                    const uint64_t adesc = smem_desc_kmajor(a_addr);
+                    const uint64_t bdesc = smem_desc_kmajor(a_addr + kABytes);
+#pragma unroll
+                    for (int k = 0; k < BK / UK; ++k) {
+                        // 16 bf16 = 32 bytes further along the 128-byte row: +2 in the address field
+                        umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                  (uint32_t)((kb | k) != 0));
+                    }
+                    umma_commit(s.empty[stage]);
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit(s.tmem_full[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1u;
+            }
+        }
+    } else {
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+            const int m0 = (tile / p.n_tiles) * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
+            if (!(ok = mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag))) break;
+            tc_fence_after();
+            const int row = m0 + q * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+            for (int c = 0; c < kOutCols; c += 32) {
+                uint32_t r[32];
+                tmem_ld32(t_row + (uint32_t)c, r);
+                tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                if (kSplitW) {
+                    tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r[i]);
+                }
+                if (row < p.M) {
+                    const size_t off = (size_t)row * p.ldo + n_out0 + c;
+                    if (kEpi == 0) {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    } else {
+                        const uint4* sk = reinterpret_cast<const uint4*>(p.skip + off);
+                        const uint4* ad = p.add ? reinterpret_cast<const uint4*>(p.add + off) : nullptr;
+                        const float4* dg = reinterpret_cast<const float4*>(p.diag + n_out0 + c);
+                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {  // 8 outputs per iteration
+                            const uint4 sv = sk[i];
+                            const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
+                            const float4 d0 = dg[2 * i], d1 = dg[2 * i + 1];
+                            const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                            float o[8];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 sf = __bfloat1622float2(s2[j]);
+                                o[2 * j] = fmaf(dd[2 * j], sf.x, v[8 * i + 2 * j]);
+                                o[2 * j + 1] = fmaf(dd[2 * j + 1], sf.y, v[8 * i + 2 * j + 1]);
+                            }
+                            if (ad) {
+                                const uint4 av = ad[i];
+                                const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&av);
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const float2 af = __bfloat1622float2(a2[j]);
+                                    o[2 * j] += af.x;
+                                    o[2 * j + 1] += af.y;
+                                }
+                            }
+                            uint4 ov;
+                            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(o[2 * j], o[2 * j + 1]);
+                            dst[i] = ov;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(s.tmem_empty[acc]);
+            if ((acc ^= 1) == 0) acc_phase ^= 1u;
+        }
+    }
+    epilogue_exit(s, warp, tmem_base, p.hdr);
+}
+
+// ---------------------------------------------------------------------------------------------
+// NT kernel (weight gradients): one 128 x 256 output tile and one slice of the rows per CTA
+// ---------------------------------------------------------------------------------------------
+struct NtParams {
+    int K;              // rows of A and Bm (the reduction index)
+    int J;              // columns of Bm = leading dimension of a partial
+    int I;              // columns of A
+    int j_tiles;        // J / BN
+    int blocks_per_split;  // k-blocks (of BK rows) per slice
+    float* part;        // [splits, I, J]
+    WsHeader* hdr;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBhi,
+                  const __grid_constant__ CUtensorMap tmBlo, NtParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tmem_base = prologue(s, warp, lane);
+    const int tile = blockIdx.x, split = blockIdx.y;
+    constexpr int kOutCols = BN / 2;   // accumulator columns [0,128): hi plane, [128,256): lo plane
+    const int i0 = (tile / p.j_tiles) * BM, j0 = (tile % p.j_tiles) * kOutCols;
+    const int total_blocks = (p.K + BK - 1) / BK;
+    const int kb0 = split * p.blocks_per_split;
+    const int kb1 = min(total_blocks, kb0 + p.blocks_per_split);
+    const int nkb = max(0, kb1 - kb0);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmBhi);
+            prefetch_tmap(&tmBlo);
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag)) break;
+                mbar_expect_tx(s.full[stage], kStageBytes);
+                const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
+                const int row = (kb0 + kb) * BK;
+#pragma unroll
+                for (int h = 0; h < BM / 64; ++h) tma_load_2d(a_dst + h * (BK * 128), &tmA, s.full[stage], i0 + 64 * h, row);
+#pragma unroll
+                for (int h = 0; h < kOutCols / 64; ++h) {
+                    tma_load_2d(a_dst + kABytes + h * (BK * 128), &tmBhi, s.full[stage], j0 + 64 * h, row);
+                    tma_load_2d(a_dst + kABytes + (kOutCols / 64 + h) * (BK * 128), &tmBlo, s.full[stage],
+                                j0 + 64 * h, row);
+                }
+                if (++stage == kStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && nkb > 0) {
+            constexpr uint32_t idesc = instr_desc(BM, BN, 1, 1);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageBytes);
+                const uint64_t adesc = smem_desc_mnmajor(a_addr);
+                const uint64_t bdesc = smem_desc_mnmajor(a_addr + kABytes);
+#pragma unroll
+                for (int k = 0; k < BK / UK; ++k) {
+                    // 16 k-rows of 128 bytes further: +2048 bytes = +128 in the address field
+                    umma_bf16(tmem_base, adesc + (uint64_t)(128 * k), bdesc + (uint64_t)(128 * k), idesc,
+                              (uint32_t)((kb | k) != 0));
+                }
+                umma_commit(s.empty[stage]);
+                if (++stage == kStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+            if (ok) umma_commit(s.tmem_full[0]);
+        }
+    } else {
+        const int q = warp & 3;
+        const int row = i0 + q * 32 + lane;
+        float* dst_row = p.part + ((size_t)split * p.I + row) * p.J + j0;
+        bool ok = true;
+        if (nkb > 0) {
+            ok = mbar_wait(s.tmem_full[0], 0, s.abort_flag);
+            tc_fence_after();
+        }
+        if (ok) {
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < kOutCols; c += 32) {
+                float v[32];
+                if (nkb > 0) {
+                    uint32_t r[32];
+                    tmem_ld32(t_row + (uint32_t)c, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                    tmem_ld32(t_row + (uint32_t)(kOutCols + c), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r[i]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0.f;
+                }
+                if (row < p.I) {
+                    float4* dst = reinterpret_cast<float4*>(dst_row + c);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+            }
+        }
+    }
+    epilogue_exit(s, warp, tmem_base, p.hdr);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+static PFN_cuTensorMapEncodeTiled encode_fn() {
+    static PFN_cuTensorMapEncodeTiled fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(p);
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows, cols] (cols contiguous), boxes of box_cols x box_rows, 128-byte swizzle.
+static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_cols,
+                     uint32_t box_rows) {
+    PFN_cuTensorMapEncodeTiled fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <typename K>
+static bool set_smem(K kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) == cudaSuccess;
+}
+
+}  // namespace tc
+
+bool tc_tn_supported(int M, int N_out, int K, bool split_w) {
+    const int out_cols = split_w ? tc::BN / 2 : tc::BN;
+    return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % out_cols) == 0;
+}
+
+int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
+    using namespace tc;
+    const int out_cols = g.split_w ? BN / 2 : BN;
+    const int n_tiles = g.N_out / out_cols;
+    CUtensorMap ma, mw;
+    if (!make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, BK, BM)) return SSM_ERR_CUDA;
+    if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN)) return SSM_ERR_CUDA;
+    TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.out, g.diag, (const __nv_bfloat16*)g.skip,
+               (const __nv_bfloat16*)g.add, g.hdr};
+    const int m_tiles = (g.M + BM - 1) / BM;
+    const int grid = min(sm_count(), m_tiles * n_tiles);
+    count_launch();
+    bool ok;
+    if (g.store_f32) {
+        if (g.split_w) {
+            ok = set_smem(gemm_tc_tn_kernel<0, true>);
+            gemm_tc_tn_kernel<0, true><<<grid, kThreads, kSmemBytes, st>>>(ma, mw, p);
+        } else {
+            ok = set_smem(gemm_tc_tn_kernel<0, false>);
+            gemm_tc_tn_kernel<0, false><<<grid, kThreads, kSmemBytes, st>>>(ma, mw, p);
+        }
+    } else {
+        ok = set_smem(gemm_tc_tn_kernel<1, false>);
+        gemm_tc_tn_kernel<1, false><<<grid, kThreads, kSmemBytes, st>>>(ma, mw, p);
+    }
+    return ok ? SSM_OK : SSM_ERR_CUDA;
+}
+
+bool tc_nt_supported(int I, int J) { return (I % tc::BM) == 0 && (J % (tc::BN / 2)) == 0; }
+
+int tc_nt_splits(int K, int I, int J) {
+    const int tiles = (I / tc::BM) * (J / (tc::BN / 2));
+    const int blocks = (K + tc::BK - 1) / tc::BK;
+    int s = tc::sm_count() / (tiles > 0 ? tiles : 1);
+    if (s < 1) s = 1;
+    if (s > blocks) s = blocks;
+    if (s > 64) s = 64;
+    return s;
+}
+
+int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
+    using namespace tc;
+    CUtensorMap ma, mbh, mbl;
+    if (!make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.I, 64, BK)) return SSM_ERR_CUDA;
+    if (!make_map(&mbh, g.Bm_hi, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
+    if (!make_map(&mbl, g.Bm_lo, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
+    const int blocks = (g.K + BK - 1) / BK;
+    const int bps = (blocks + g.splits - 1) / g.splits;
+    const int j_tiles = g.J / (BN / 2);
+    NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr};
+    dim3 grid((g.I / BM) * j_tiles, g.splits);
+    count_launch();
+    const bool ok = set_smem(gemm_tc_nt_kernel);
+    gemm_tc_nt_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mbh, mbl, p);
+    return ok ? SSM_OK : SSM_ERR_CUDA;
+}
+
+}  // namespace ssm

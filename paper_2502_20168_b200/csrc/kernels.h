@@ -18,10 +18,12 @@ void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const flo
 // Scratch the scans need for a [B,T,P] problem: look-back records and the partial sums of gAbar.
 size_t scan_scratch_bytes(int B, int T, int P);
 int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Bu, const uint8_t* done,
-                    const float2* x0, float2* x, float2* xT, WsHeader* hdr, void* scratch, cudaStream_t st);
+                    const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr, void* scratch,
+                    cudaStream_t st);
+// x and gBu are stored both as fp32 pairs or both as bf16 pairs (x_bf16 == s_bf16).
 int launch_scan_bwd(int B, int T, int P, const float2* Abar, const uint8_t* done, const float2* x0,
-                    const float2* x, const float2* gx, const float2* gxT, float2* gBu, float2* gAbar,
-                    float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st);
+                    const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
+                    float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st);
 
 // reduce.cu
 // out[c] = sum_r in[r, c]; `tmp` must hold colsum_tmp_floats(R, C) floats.  Deterministic.
@@ -59,5 +61,39 @@ void launch_gemm_nt(const GemmNT& g, cudaStream_t st);
 // mode 0: complex out[J/2, I]: out[j/2, i].(re if j even else im) = sum_s part[s,i,j]
 // mode 1: complex out[I, J/2]: out[i, j/2] likewise, with the imaginary part negated
 void launch_splitk_reduce(const float* part, int splits, int I, int J, int mode, float2* out, cudaStream_t st);
+
+// gemm_tc.cu: bf16 projections on tcgen05 tensor cores (operands by TMA, accumulators in TMEM).
+struct GemmTcTN {
+    // out[m, n] = sum_k A[m, k] * W[n, k];  A bf16 [M, K];  W bf16 packed by pack_operands_tc:
+    // [N_out, K], or with split_w [2 * N_out, K] where each group of 256 rows holds the high
+    // halves of 128 output columns followed by their low halves.
+    const void* A; const void* W;
+    int M, N_out, K;
+    bool split_w;
+    bool store_f32;                      // true: out fp32 [M, N_out]; false: out bf16 with the epilogue below
+    void* out;
+    const float* diag; const void* skip; const void* add;   // out = acc + diag[n] * skip[m, n] (+ add[m, n])
+    WsHeader* hdr;
+};
+bool tc_tn_supported(int M, int N_out, int K, bool split_w);
+int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st);
+
+struct GemmTcNT {
+    // part[s, i, j] = sum_{m in slice s} A[m, i] * (Bm_hi[m, j] + Bm_lo[m, j]);  A bf16 [K, I],
+    // Bm_hi / Bm_lo bf16 [K, J]: the two planes of a state tensor
+    const void* A; int I;
+    const void* Bm_hi; const void* Bm_lo; int J;
+    int K; int splits;
+    float* part;
+    WsHeader* hdr;
+};
+bool tc_nt_supported(int I, int J);
+int tc_nt_splits(int K, int I, int J);
+int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
+
+// discretize.cu: operands of the tensor-core path (bf16).  Wsplit_B / Wsplit_C: [4P, H] hi/lo
+// stacked forms of Bp / Cq (see GemmTcTN);  Cp, Bq: [H, 2P] single bf16.
+void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
+                             void* Cp, void* Bq, cudaStream_t st);
 
 }  // namespace ssm

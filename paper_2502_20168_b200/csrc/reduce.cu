@@ -42,26 +42,52 @@ void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaSt
     colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(tmp, groups, C, groups, out);
 }
 
-// part[g, c] = sum_{m in group g} a[m, c] * b[m, c]
-constexpr int kDotRows = 256;
+// part[g, c] = sum_{m in group g} a[m, c] * b[m, c].  A thread owns 4 neighbouring columns
+// (16 bytes of fp32, 8 bytes of bf16 per load); block = 32 column quads x 8 row lanes.
+constexpr int kDotRows = 128;
 template <typename T>
-__global__ void dot_columns_kernel(const T* __restrict__ a, const T* __restrict__ b, int M, int C,
-                                   float* __restrict__ part) {
-    __shared__ float sm[8][33];
-    const int c = blockIdx.x * 32 + threadIdx.x;
+__device__ __forceinline__ void load_quad(const T* p, float (&v)[4]);
+template <>
+__device__ __forceinline__ void load_quad<float>(const float* p, float (&v)[4]) {
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+template <>
+__device__ __forceinline__ void load_quad<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[4]) {
+    const uint2 t = __ldcs(reinterpret_cast<const uint2*>(p));
+    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&t.x));
+    const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&t.y));
+    v[0] = lo.x; v[1] = lo.y; v[2] = hi.x; v[3] = hi.y;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+dot_columns_kernel(const T* __restrict__ a, const T* __restrict__ b, int M, int C, float* __restrict__ part) {
+    __shared__ float4 sm[8][33];
+    const int c = (blockIdx.x * 32 + threadIdx.x) * 4;
     const int r0 = blockIdx.y * kDotRows;
     const int r1 = min(M, r0 + kDotRows);
-    float acc = 0.f;
-    if (c < C)
-        for (int r = r0 + threadIdx.y; r < r1; r += 8)
-            acc = fmaf(to_f32<T>(a[(size_t)r * C + c]), to_f32<T>(b[(size_t)r * C + c]), acc);
-    sm[threadIdx.y][threadIdx.x] = acc;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    if (c < C) {
+#pragma unroll 4
+        for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+            float va[4], vb[4];
+            load_quad<T>(a + (size_t)r * C + c, va);
+            load_quad<T>(b + (size_t)r * C + c, vb);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[i] = fmaf(va[i], vb[i], acc[i]);
+        }
+    }
+    sm[threadIdx.y][threadIdx.x] = make_float4(acc[0], acc[1], acc[2], acc[3]);
     __syncthreads();
     if (threadIdx.y == 0 && c < C) {
-        float t = 0.f;
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x];
-        part[(size_t)blockIdx.y * C + c] = t;
+        for (int i = 0; i < 8; ++i) {
+            const float4 v = sm[i][threadIdx.x];
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        *reinterpret_cast<float4*>(part + (size_t)blockIdx.y * C + c) = t;
     }
 }
 
@@ -75,7 +101,7 @@ size_t dot_columns_tmp_floats(int M, int C) {
 void launch_dot_columns(bool bf16, const void* a, const void* b, int M, int C, float* out, float* tmp,
                         cudaStream_t st) {
     const int g = dot_groups(M);
-    dim3 blk(32, 8), grid((C + 31) / 32, g);
+    dim3 blk(32, 8), grid((C + 127) / 128, g);
     count_launch();
     if (bf16)
         dot_columns_kernel<__nv_bfloat16><<<grid, blk, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, M, C, tmp);
