@@ -32,7 +32,10 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;  // two accumulator buffers of BN columns
 constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kStagingBytes = 4 * 32 * 32 * 4;  // per epilogue warp: 32 rows x 32 fp32 columns
+constexpr int kMaxDiag = 4096;                  // widest output whose diagonal fits the shared copy
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kStagingBytes + kMaxDiag * 4 +
+                              1024 /*alignment slack*/ + 256 /*barriers*/;
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -144,6 +147,8 @@ __host__ __device__ constexpr uint32_t instr_desc(int m, int n, int a_mn, int b_
 
 struct Smem {
     uint8_t* tiles;       // 1024-byte aligned
+    uint8_t* staging;     // epilogue transpose buffers
+    float* diag;          // copy of the epilogue's diagonal
     uint32_t full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
     uint32_t tmem_slot;   // where tcgen05.alloc writes the base address
     volatile int* abort_flag;
@@ -154,7 +159,9 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* raw) {
     Smem s;
     uintptr_t base = (reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023;
     s.tiles = reinterpret_cast<uint8_t*>(base);
-    uint8_t* bars = s.tiles + (size_t)kStages * kStageBytes;
+    s.staging = s.tiles + (size_t)kStages * kStageBytes;
+    s.diag = reinterpret_cast<float*>(s.staging + kStagingBytes);
+    uint8_t* bars = s.staging + kStagingBytes + kMaxDiag * 4;
     for (int i = 0; i < kStages; ++i) {
         s.full[i] = smem_u32(bars + 8 * i);
         s.empty[i] = smem_u32(bars + 8 * (kStages + i));
@@ -227,6 +234,8 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (kEpi == 1)
+        for (int i = threadIdx.x; i < p.ldo; i += kThreads) s.diag[i] = p.diag[i];
     const uint32_t tmem_base = prologue(s, warp, lane);
     const int m_tiles = (p.M + BM - 1) / BM;
     const int total = m_tiles * p.n_tiles;
@@ -294,50 +303,88 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
             const int m0 = (tile / p.n_tiles) * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
+            const int row0 = m0 + q * 32;   // first of this warp's 32 rows
+            // skip[m, n] slabs are fetched kPre slabs ahead of their use (the first ones while the
+            // tile's MMAs are still running): lane -> (row i*8 + lane/4, 8 columns) per slab
+            constexpr int kSlabs = kOutCols / 32, kPre = 3;
+            uint4 skb[kPre + 1][4];
+            auto load_skip = [&](int slab, uint4 (&dst)[4]) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int rr = i * 8 + (lane >> 2);
+                    if (row0 + rr < p.M)
+                        dst[i] = __ldg(reinterpret_cast<const uint4*>(
+                            p.skip + (size_t)(row0 + rr) * p.ldo + n_out0 + slab * 32 + (lane & 3) * 8));
+                }
+            };
+            if (kEpi == 1) {
+#pragma unroll
+                for (int d = 0; d < kPre; ++d) load_skip(d, skb[d]);
+            }
             if (!(ok = mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag))) break;
             tc_fence_after();
-            const int row = m0 + q * 32 + lane;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-#pragma unroll 1
-            for (int c = 0; c < kOutCols; c += 32) {
-                uint32_t r[32];
+            float4* stg = reinterpret_cast<float4*>(s.staging) + (size_t)(warp - 2) * (32 * 8);
+#pragma unroll
+            for (int sl = 0; sl < kSlabs; ++sl) {
+                const int c = sl * 32;
+                if (kEpi == 1 && sl + kPre < kSlabs) load_skip(sl + kPre, skb[(sl + kPre) % (kPre + 1)]);
+                // TMEM -> registers: lane = row, 32 consecutive columns
+                uint32_t r[32], r2[32];
                 tmem_ld32(t_row + (uint32_t)c, r);
+                if (kSplitW) tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
                 tmem_ld_wait();
-                float v[32];
+                // registers -> staging (16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7))
+                __syncwarp();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                if (kSplitW) {
-                    tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r[i]);
+                for (int j = 0; j < 8; ++j) {
+                    float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                           __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                    if (kSplitW) {
+                        v.x += __uint_as_float(r2[4 * j]);
+                        v.y += __uint_as_float(r2[4 * j + 1]);
+                        v.z += __uint_as_float(r2[4 * j + 2]);
+                        v.w += __uint_as_float(r2[4 * j + 3]);
+                    }
+                    stg[lane * 8 + (j ^ (lane & 7))] = v;
                 }
-                if (row < p.M) {
-                    const size_t off = (size_t)row * p.ldo + n_out0 + c;
-                    if (kEpi == 0) {
-                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off);
+                __syncwarp();
+                // staging -> global with full-line accesses
+                if (kEpi == 0) {
+                    // each instruction covers 4 rows x 128 bytes: lane -> (row i*4 + lane/8, chunk lane%8)
+                    float* out = reinterpret_cast<float*>(p.out);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                    } else {
-                        const uint4* sk = reinterpret_cast<const uint4*>(p.skip + off);
-                        const uint4* ad = p.add ? reinterpret_cast<const uint4*>(p.add + off) : nullptr;
-                        const float4* dg = reinterpret_cast<const float4*>(p.diag + n_out0 + c);
-                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off);
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr = i * 4 + (lane >> 3), ch = lane & 7;
+                        const float4 v = stg[rr * 8 + (ch ^ (rr & 7))];
+                        if (row0 + rr < p.M)
+                            *reinterpret_cast<float4*>(out + (size_t)(row0 + rr) * p.ldo + n_out0 + c + ch * 4) = v;
+                    }
+                } else {
+                    // each instruction covers 8 rows x 64 bytes of bf16: lane -> (row i*8 + lane/4, 8 columns)
+                    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+                    const int cq = lane & 3;
+                    const float4 d0 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8);
+                    const float4 d1 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8 + 4);
+                    const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {  // 8 outputs per iteration
-                            const uint4 sv = sk[i];
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = i * 8 + (lane >> 2);
+                        const float4 a0 = stg[rr * 8 + ((2 * cq) ^ (rr & 7))];
+                        const float4 a1 = stg[rr * 8 + ((2 * cq + 1) ^ (rr & 7))];
+                        if (row0 + rr < p.M) {
+                            const size_t off = (size_t)(row0 + rr) * p.ldo + n_out0 + c + cq * 8;
+                            const uint4 sv = skb[sl % (kPre + 1)][i];
                             const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
-                            const float4 d0 = dg[2 * i], d1 = dg[2 * i + 1];
-                            const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-                            float o[8];
+                            float o[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const float2 sf = __bfloat1622float2(s2[j]);
-                                o[2 * j] = fmaf(dd[2 * j], sf.x, v[8 * i + 2 * j]);
-                                o[2 * j + 1] = fmaf(dd[2 * j + 1], sf.y, v[8 * i + 2 * j + 1]);
+                                o[2 * j] = fmaf(dd[2 * j], sf.x, o[2 * j]);
+                                o[2 * j + 1] = fmaf(dd[2 * j + 1], sf.y, o[2 * j + 1]);
                             }
-                            if (ad) {
-                                const uint4 av = ad[i];
+                            if (p.add) {
+                                const uint4 av = *reinterpret_cast<const uint4*>(p.add + off);
                                 const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&av);
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
@@ -350,7 +397,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                             __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
 #pragma unroll
                             for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(o[2 * j], o[2 * j + 1]);
-                            dst[i] = ov;
+                            *reinterpret_cast<uint4*>(out + off) = ov;
                         }
                     }
                 }
@@ -531,7 +578,7 @@ static bool set_smem(K kernel) {
 
 bool tc_tn_supported(int M, int N_out, int K, bool split_w) {
     const int out_cols = split_w ? tc::BN / 2 : tc::BN;
-    return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % out_cols) == 0;
+    return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % out_cols) == 0 && N_out <= tc::kMaxDiag;
 }
 
 int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {

@@ -123,8 +123,30 @@ scan_fwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
     if (xT) xT[(size_t)b * P2 + pp] = c2_pack(s);
 }
 
+// Undecoded state loads, so that a whole batch of them can be in flight while the previous
+// batch is being processed.
+template <typename ST> struct RawState;
+template <> struct RawState<float4> {
+    float4 v;
+    __device__ __forceinline__ void load(const float4* p, size_t) { v = __ldcs(p); }
+    __device__ __forceinline__ C2 get() const { return c2_from(v); }
+};
+template <> struct RawState<uint2> {
+    uint2 hi, lo;
+    __device__ __forceinline__ void load(const uint2* p, size_t plane) {
+        hi = __ldcs(p);
+        lo = __ldcs(p + plane);
+    }
+    __device__ __forceinline__ C2 get() const {
+        const C2 h = unpack_bf16x4(hi), l = unpack_bf16x4(lo);
+        return C2{cadd(h.a, l.a), cadd(h.b, l.b)};
+    }
+};
+
 // s_t = gx_t + c_t,  c_{t-1} = keep_t conj(Abar) s_t  (c_{T-1} = gxT);
 // gAbar partial = sum_t keep_t s_t conj(x_{t-1}).  gBu may alias gx.
+// Two register batches of kUnrollBwd steps alternate: the loads of one are issued before the
+// other is processed.
 template <typename XT, typename ST>
 __global__ void __launch_bounds__(kSeqThreads)
 scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const uint8_t* __restrict__ done,
@@ -144,34 +166,52 @@ scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
     ST* dst = gBu + (size_t)b * T * P2 + pp;
     const uint8_t* dn = done ? done + (size_t)b * T : nullptr;
     const C2 xinit = x0 ? c2_from(x0[(size_t)b * P2 + pp]) : c2_zero();
-    for (int t0 = T - 1; t0 >= 0; t0 -= kUnrollBwd) {
-        C2 v[kUnrollBwd], xp[kUnrollBwd];
-        bool d[kUnrollBwd];
+
+    struct Batch {
+        float4 v[kUnrollBwd];
+        RawState<XT> xp[kUnrollBwd];
+        uint32_t flags;
+    };
+    // steps t0, t0-1, ..., t0-kUnrollBwd+1 (those that exist)
+    auto fetch = [&](int t0, Batch& q) {
+        q.flags = 0u;
 #pragma unroll
         for (int i = 0; i < kUnrollBwd; ++i) {
             const int t = t0 - i;
             if (t >= 0) {
-                v[i] = StateIO<float4>::load(gsrc + (size_t)t * P2, 0);
-                xp[i] = (t > 0) ? StateIO<XT>::load(xsrc + (size_t)(t - 1) * P2, plane) : xinit;
-                d[i] = dn ? (dn[t] != 0) : false;
+                q.v[i] = __ldcs(gsrc + (size_t)t * P2);
+                if (t > 0) q.xp[i].load(xsrc + (size_t)(t - 1) * P2, plane);
+                if (dn && dn[t] != 0) q.flags |= 1u << i;
             }
         }
+    };
+    auto process = [&](int t0, const Batch& q) {
 #pragma unroll
         for (int i = 0; i < kUnrollBwd; ++i) {
             const int t = t0 - i;
             if (t >= 0) {
-                const C2 s{cadd(v[i].a, c.a), cadd(v[i].b, c.b)};
+                const C2 vi = c2_from(q.v[i]);
+                const C2 s{cadd(vi.a, c.a), cadd(vi.b, c.b)};
                 StateIO<ST>::store(dst + (size_t)t * P2, s, plane);
-                if (d[i]) {
+                if ((q.flags >> i) & 1u) {
                     c = c2_zero();
                 } else {
-                    g.a = cfma(s.a, cconj(xp[i].a), g.a);
-                    g.b = cfma(s.b, cconj(xp[i].b), g.b);
+                    const C2 xprev = t > 0 ? q.xp[i].get() : xinit;
+                    g.a = cfma(s.a, cconj(xprev.a), g.a);
+                    g.b = cfma(s.b, cconj(xprev.b), g.b);
                     c.a = cmul(ac0, s.a);
                     c.b = cmul(ac1, s.b);
                 }
             }
         }
+    };
+    Batch q0, q1;
+    fetch(T - 1, q0);
+    for (int t0 = T - 1; t0 >= 0; t0 -= 2 * kUnrollBwd) {
+        fetch(t0 - kUnrollBwd, q1);
+        process(t0, q0);
+        fetch(t0 - 2 * kUnrollBwd, q0);
+        process(t0 - kUnrollBwd, q1);
     }
     gA_part[(size_t)b * P2 + pp] = c2_pack(g);
     if (gx0) gx0[(size_t)b * P2 + pp] = c2_pack(c);
