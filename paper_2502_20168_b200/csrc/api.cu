@@ -14,7 +14,7 @@ namespace {
 struct LayerPlan {
     bool tc;
     int splits;
-    size_t hdr, Abar, Bbar, W0, W1, W2, W3, f32buf, xs, gs, gAbar, gBbar, scan, part, dot, total;
+    size_t hdr, Abar, Alo, Bbar, W0, W1, W2, W3, f32buf, xs, gs, gAbar, gBbar, scan, part, dot, total;
 };
 
 size_t take(size_t& off, size_t bytes) {
@@ -33,6 +33,7 @@ LayerPlan plan_layer(const ssm_shape& s) {
     p.splits = p.tc ? tc_nt_splits((int)BT, s.H, P2) : gemm_nt_splits((int)BT);
     p.hdr = take(off, sizeof(WsHeader));
     p.Abar = take(off, (size_t)s.P * 8);
+    p.Alo = take(off, (size_t)s.P * 8);
     p.Bbar = take(off, PH * 8);
     if (p.tc) {
         p.W0 = take(off, 4 * PH * 2);   // hi/lo stacked Bbar operand  [4P, H] bf16
@@ -102,7 +103,7 @@ SSM_API int ssm_discretize(const ssm_shape* shape, const ssm_c64* Lambda, const 
     if (!Lambda || !Delta || !Bc || !Abar || !Bbar) return SSM_ERR_NULL;
     if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Abar) || misaligned(Bbar))
         return SSM_ERR_ALIGN;
-    launch_discretize(shape->H, shape->P, (const float2*)Lambda, Delta, (const float2*)Bc, (float2*)Abar,
+    launch_discretize(shape->H, shape->P, (const float2*)Lambda, Delta, (const float2*)Bc, (float2*)Abar, nullptr,
                       (float2*)Bbar, (cudaStream_t)stream);
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;
@@ -137,7 +138,7 @@ SSM_API int ssm_scan_fwd(const ssm_shape* shape, const ssm_c64* Abar, const ssm_
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     StageTimer tm("scan_fwd", st);
-    int rc = launch_scan_fwd(shape->B, shape->T, shape->P, (const float2*)Abar, (const float2*)Bu, done,
+    int rc = launch_scan_fwd(shape->B, shape->T, shape->P, (const float2*)Abar, nullptr, (const float2*)Bu, done,
                              (const float2*)x0, x, false, (float2*)xT, at<WsHeader>(ws, 0),
                              at<char>(ws, sizeof(WsHeader)), st);
     if (rc) return rc;
@@ -157,7 +158,7 @@ SSM_API int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     StageTimer tm("scan_bwd", st);
-    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, done, (const float2*)x0, x, false,
+    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, nullptr, done, (const float2*)x0, x, false,
                              (const float2*)gx, (const float2*)gxT, gBu, false, (float2*)gAbar, (float2*)gx0,
                              at<WsHeader>(ws, 0), at<char>(ws, sizeof(WsHeader)), st);
     if (rc) return rc;
@@ -191,7 +192,7 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     {
         StageTimer tm("discretize_pack", st);
         launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
-                          at<float2>(ws, p.Bbar), st);
+                          at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
         if (p.tc)
             launch_pack_operands_tc(s.H, s.P, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
                                     at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
@@ -208,7 +209,7 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         }
         {
             StageTimer tm("scan_fwd", st);
-            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.f32buf), done,
+            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), at<float2>(ws, p.f32buf), done,
                                  (const float2*)x0, at<void>(ws, p.xs), true, (float2*)xT, hdr,
                                  at<char>(ws, p.scan), st);
             if (rc) return rc;
@@ -227,7 +228,7 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         }
         {
             StageTimer tm("scan_fwd", st);
-            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.xs), done,
+            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), at<float2>(ws, p.xs), done,
                                  (const float2*)x0, at<void>(ws, p.xs), false, (float2*)xT, hdr,
                                  at<char>(ws, p.scan), st);
             if (rc) return rc;
@@ -275,7 +276,7 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         }
         {
             StageTimer tm("scan_bwd", st);
-            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done, (const float2*)x0,
                                  at<void>(ws, p.xs), true, at<float2>(ws, p.f32buf), (const float2*)gxT,
                                  at<void>(ws, p.gs), true, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
                                  at<char>(ws, p.scan), st);
@@ -307,7 +308,7 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         }
         {
             StageTimer tm("scan_bwd", st);
-            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done, (const float2*)x0,
                                  at<void>(ws, p.xs), false, at<float2>(ws, p.gs), (const float2*)gxT,
                                  at<void>(ws, p.gs), false, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
                                  at<char>(ws, p.scan), st);

@@ -34,12 +34,14 @@ __device__ __forceinline__ ZohTerms zoh_terms(float2 lam, float dt) {
 // One block per state p: Abar[p], Bbar[p, :] = gamma_p * B[p, :].
 __global__ void discretize_kernel(int H, const float2* __restrict__ Lambda, const float* __restrict__ Delta,
                                   const float2* __restrict__ Bc, float2* __restrict__ Abar,
-                                  float2* __restrict__ Bbar) {
+                                  float2* __restrict__ Abar_lo, float2* __restrict__ Bbar) {
     __shared__ float2 gamma_s;
     const int p = blockIdx.x;
     if (threadIdx.x == 0) {
         ZohTerms z = zoh_terms(Lambda[p], Delta[p]);
-        Abar[p] = make_float2((float)z.ar, (float)z.ai);
+        const float2 ah = make_float2((float)z.ar, (float)z.ai);
+        Abar[p] = ah;
+        if (Abar_lo) Abar_lo[p] = make_float2((float)(z.ar - (double)ah.x), (float)(z.ai - (double)ah.y));
         gamma_s = make_float2((float)z.gr, (float)z.gi);
     }
     __syncthreads();
@@ -179,9 +181,9 @@ void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc,
 }
 
 void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc, float2* Abar,
-                       float2* Bbar, cudaStream_t st) {
+                       float2* Abar_lo, float2* Bbar, cudaStream_t st) {
     count_launch();
-    discretize_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, Abar, Bbar);
+    discretize_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, Abar, Abar_lo, Bbar);
 }
 
 void launch_discretize_bwd(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,

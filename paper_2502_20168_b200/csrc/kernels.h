@@ -6,8 +6,9 @@
 namespace ssm {
 
 // discretize.cu
+// Abar_lo (may be NULL): Abar's rounding residual, exp(Lambda Delta) - Abar, as fp32.
 void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc, float2* Abar,
-                       float2* Bbar, cudaStream_t st);
+                       float2* Abar_lo, float2* Bbar, cudaStream_t st);
 void launch_discretize_bwd(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
                            const float2* gAbar, const float2* gBbar, float2* dLambda, float* dDelta, float2* dB,
                            cudaStream_t st);
@@ -17,11 +18,12 @@ void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const flo
 // scan.cu
 // Scratch the scans need for a [B,T,P] problem: look-back records and the partial sums of gAbar.
 size_t scan_scratch_bytes(int B, int T, int P);
-int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Bu, const uint8_t* done,
+// Alo (may be NULL): low part of Abar, so that Abar + Alo carries the multiplier to ~48 bits.
+int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu, const uint8_t* done,
                     const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr, void* scratch,
                     cudaStream_t st);
 // x and gBu are stored both as fp32 pairs or both as bf16 pairs (x_bf16 == s_bf16).
-int launch_scan_bwd(int B, int T, int P, const float2* Abar, const uint8_t* done, const float2* x0,
+int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done, const float2* x0,
                     const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
                     float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st);
 

@@ -29,7 +29,7 @@ constexpr int kUnrollBwd = 8;
 constexpr int kSeqThreads = 64;   // small blocks spread a few hundred thousand threads evenly over the SMs
 constexpr int kScanThreads = 128;
 constexpr int kFwdChunk = 32;     // steps per chunk, forward
-constexpr int kBwdChunk = 16;     // steps per chunk, backward (it also holds x)
+constexpr int kBwdChunk = 16;     // steps per chunk, backward (its buffers also hold x)
 constexpr uint32_t kPollLimit = 1u << 22;
 
 // ---- two complex states as stored in memory ----------------------------------------------
@@ -77,6 +77,24 @@ template <> struct StateIO<uint2> {
         p[plane] = pack_bf16x4(r);
     }
 };
+// (a + alo) * x + b with the small product added first: a step of the recurrence whose multiplier
+// is carried as an fp32 pair (hi, lo), i.e. to about 48 bits.
+__device__ __forceinline__ float2 cfma2(float2 a, float2 alo, float2 x, float2 b) {
+    return cfma(a, x, cfma(alo, x, b));
+}
+// (a + alo)^n for n a power of two, evaluated in double and returned as an fp32 pair.
+template <int N>
+__device__ __forceinline__ void cpow2_pair(float2 a, float2 alo, float2& hi, float2& lo) {
+    double re = (double)a.x + (double)alo.x, im = (double)a.y + (double)alo.y;
+#pragma unroll
+    for (int n = 1; n < N; n *= 2) {
+        const double r2 = re * re - im * im, i2 = 2.0 * re * im;
+        re = r2;
+        im = i2;
+    }
+    hi = make_float2((float)re, (float)im);
+    lo = make_float2((float)(re - (double)hi.x), (float)(im - (double)hi.y));
+}
 __device__ __forceinline__ C2 c2_from(const float4 v) { return C2{make_float2(v.x, v.y), make_float2(v.z, v.w)}; }
 __device__ __forceinline__ float4 c2_pack(const C2& v) { return make_float4(v.a.x, v.a.y, v.b.x, v.b.y); }
 
@@ -86,7 +104,8 @@ __device__ __forceinline__ float4 c2_pack(const C2& v) { return make_float4(v.a.
 // grid: ceil(B * P/2 / kSeqThreads); thread -> (b, pair of states).  x may alias Bu.
 template <typename XT>
 __global__ void __launch_bounds__(kSeqThreads)
-scan_fwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const float4* Bu,
+scan_fwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const float4* __restrict__ Alo,
+                    const float4* Bu,
                     const uint8_t* __restrict__ done, const float4* __restrict__ x0, XT* x,
                     float4* __restrict__ xT) {
     const int idx = blockIdx.x * kSeqThreads + threadIdx.x;
@@ -94,6 +113,7 @@ scan_fwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
     const int b = idx / P2, pp = idx - b * P2;
     const size_t plane = (size_t)B * T * P2;
     const C2 a = c2_from(Abar[pp]);
+    const C2 al = Alo ? c2_from(Alo[pp]) : c2_zero();
     C2 s = x0 ? c2_from(x0[(size_t)b * P2 + pp]) : c2_zero();
     const float4* src = Bu + (size_t)b * T * P2 + pp;
     XT* dst = x + (size_t)b * T * P2 + pp;
@@ -114,8 +134,8 @@ scan_fwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
             const int t = t0 + i;
             if (t < T) {
                 if (d[i]) s = c2_zero();
-                s.a = cfma(a.a, s.a, v[i].a);
-                s.b = cfma(a.b, s.b, v[i].b);
+                s.a = cfma2(a.a, al.a, s.a, v[i].a);
+                s.b = cfma2(a.b, al.b, s.b, v[i].b);
                 StateIO<XT>::store(dst + (size_t)t * P2, s, plane);
             }
         }
@@ -149,7 +169,8 @@ template <> struct RawState<uint2> {
 // other is processed.
 template <typename XT, typename ST>
 __global__ void __launch_bounds__(kSeqThreads)
-scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const uint8_t* __restrict__ done,
+scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const float4* __restrict__ Alo,
+                    const uint8_t* __restrict__ done,
                     const float4* __restrict__ x0, const XT* __restrict__ x, const float4* gx,
                     const float4* __restrict__ gxT, ST* gBu, float4* __restrict__ gA_part,
                     float4* __restrict__ gx0) {
@@ -159,6 +180,9 @@ scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
     const size_t plane = (size_t)B * T * P2;
     const C2 a = c2_from(Abar[pp]);
     const float2 ac0 = cconj(a.a), ac1 = cconj(a.b);
+    const C2 al = Alo ? c2_from(Alo[pp]) : c2_zero();
+    const float2 al0 = cconj(al.a), al1 = cconj(al.b);
+    const float2 zero2 = make_float2(0.f, 0.f);
     C2 c = gxT ? c2_from(gxT[(size_t)b * P2 + pp]) : c2_zero();
     C2 g = c2_zero();
     const float4* gsrc = gx + (size_t)b * T * P2 + pp;
@@ -199,8 +223,8 @@ scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
                     const C2 xprev = t > 0 ? q.xp[i].get() : xinit;
                     g.a = cfma(s.a, cconj(xprev.a), g.a);
                     g.b = cfma(s.b, cconj(xprev.b), g.b);
-                    c.a = cmul(ac0, s.a);
-                    c.b = cmul(ac1, s.b);
+                    c.a = cfma2(ac0, al0, s.a, zero2);
+                    c.b = cfma2(ac1, al1, s.b, zero2);
                 }
             }
         }
@@ -220,8 +244,17 @@ scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
 // =============================================================================================
 // Chunked, with decoupled look-back
 // =============================================================================================
-// Scratch layout: [ScanCounters (256 B)][status: items*128 int][agg: items*128 float4]
-// [incl: items*128 float4][gA partials (backward): items * P2 float4][column-sum scratch].
+// Here a thread owns ONE state (8-byte accesses; twice the threads of the whole-sequence
+// kernels, half the registers per buffered step) and a CTA of 128 threads is persistent: it
+// takes chunk ids from an atomic ticket and always has the loads of its next chunk in flight
+// while it folds, publishes, looks back and stores the current one.
+//
+// Items are numbered chunk-major (item = chunk * nchains + chain, a chain being one
+// (sequence, group of 128 states)), so the chunks in flight at any moment are spread over all
+// chains and the carry of every chain advances at the same time.
+//
+// Scratch layout: [ScanCounters (256 B)][status: one int per item][agg: items*128 float2]
+// [incl: items*128 float2][gA partials (backward): grid rows of P float2][column-sum scratch].
 // Everything up to the end of `status` is zeroed before each launch.
 struct ScanCounters {
     int ticket;
@@ -229,243 +262,325 @@ struct ScanCounters {
 };
 
 struct ChunkArgs {
-    int B, T, P2, nchunks, npg;
-    const float4* Abar;
+    int B, T, P, nchunks, npg, nchains, items;
+    const float2* Abar;
+    const float2* Alo;     // low part of Abar as an fp32 pair, or NULL
     const uint8_t* done;
     int* ticket;
     int* status;
-    float4* agg;
-    float4* incl;
+    float2* agg;
+    float2* incl;
     WsHeader* hdr;
 };
 
-// m^n for n a power of two
-template <int N>
-__device__ __forceinline__ float2 cpow2(float2 m) {
-#pragma unroll
-    for (int n = 1; n < N; n *= 2) m = cmul(m, m);
-    return m;
-}
+// Storage of one state: float2 (fp32 pair) or uint32_t (bf16 pair) in two planes hi / lo.
+template <typename XS> struct Raw1;
+template <> struct Raw1<float2> {
+    float2 v;
+    __device__ __forceinline__ void load(const float2* p, size_t) { v = __ldcs(p); }
+    __device__ __forceinline__ float2 get() const { return v; }
+    static __device__ __forceinline__ void store(float2* p, float2 s, size_t) { *p = s; }
+};
+template <> struct Raw1<uint32_t> {
+    uint32_t hi, lo;
+    __device__ __forceinline__ void load(const uint32_t* p, size_t plane) {
+        hi = __ldcs(p);
+        lo = __ldcs(p + plane);
+    }
+    __device__ __forceinline__ float2 get() const {
+        const float2 h = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hi));
+        const float2 l = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&lo));
+        return cadd(h, l);
+    }
+    static __device__ __forceinline__ void store(uint32_t* p, float2 s, size_t plane) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(s.x, s.y);
+        const float2 hf = __bfloat1622float2(h);
+        const __nv_bfloat162 l = __floats2bfloat162_rn(s.x - hf.x, s.y - hf.y);
+        p[0] = *reinterpret_cast<const uint32_t*>(&h);
+        p[plane] = *reinterpret_cast<const uint32_t*>(&l);
+    }
+};
 
-__device__ __forceinline__ void publish(float4* slot, int* status, const C2& v, int state) {
-    *slot = c2_pack(v);
+// The CTA publishes one record (128 values, then the item's state word).  All threads call it.
+__device__ __forceinline__ void publish(const ChunkArgs& k, float2* values, int item, float2 v, int state) {
+    values[(size_t)item * kScanThreads + threadIdx.x] = v;
     __threadfence();
-    *reinterpret_cast<volatile int*>(status) = state;
+    __syncthreads();
+    if (threadIdx.x == 0) *reinterpret_cast<volatile int*>(k.status + item) = state;
 }
 
-// State entering this chunk, from the records of the chunks processed before it (items
-// item-1, item-2, ... in ticket order).  `mult` is the per-chunk multiplier (Abar^L or its
-// conjugate).  Bounded: gives up into hdr->status.
-__device__ __forceinline__ C2 look_back(const ChunkArgs& k, int item, int tid, float2 mult_a, float2 mult_b) {
-    C2 carry = c2_zero();
-    float2 ma = make_float2(1.f, 0.f), mb = ma;
-    for (int j = item - 1;; --j) {
-        const size_t r = (size_t)j * kScanThreads + tid;
-        volatile int* st = k.status + r;
-        int state = *st;
-        uint32_t polls = 0;
-        while (state == 0) {
+// State entering chunk `ci` of a chain, from the records of the chain's earlier chunks (items
+// item - nchains, item - 2 nchains, ...).  `mult` is the per-chunk multiplier (Abar^L or its
+// conjugate).  A window of kWindow predecessors is inspected at a time, their state words and
+// values fetched with independent loads, so a long run of aggregates costs a few round trips
+// instead of one per chunk.  Control flow is uniform over the CTA (state words are per item).
+// Bounded: gives up into hdr->status.
+constexpr int kWindow = 8;
+__device__ __forceinline__ float2 look_back(const ChunkArgs& k, int item, int ci, float2 mult, float2 mult_lo) {
+    float2 carry = make_float2(0.f, 0.f);
+    float2 m = make_float2(1.f, 0.f);
+    int back = 1;             // next predecessor to absorb: chunk ci - back
+    uint32_t polls = 0;
+    for (;;) {
+        int st[kWindow];
+#pragma unroll
+        for (int i = 0; i < kWindow; ++i) {
+            const int d = back + i;
+            st[i] = d <= ci ? *reinterpret_cast<volatile int*>(k.status + (item - d * k.nchains)) : 0;
+        }
+        int n = 0;            // predecessors usable now: a ready prefix, cut after the first inclusive one
+        bool closed = false;
+#pragma unroll
+        for (int i = 0; i < kWindow; ++i)
+            if (n == i && !closed && st[i] != 0) {
+                n = i + 1;
+                closed = st[i] == 2;
+            }
+        if (n == 0) {
             if (++polls > kPollLimit) {
                 k.hdr->status = SSM_ERR_TIMEOUT;
                 return carry;
             }
-            __nanosleep(40);
-            state = *st;
+            __nanosleep(20);
+            continue;
         }
         __threadfence();
-        const C2 v = c2_from(__ldcg((state == 2 ? k.incl : k.agg) + r));
-        carry.a = cfma(ma, v.a, carry.a);
-        carry.b = cfma(mb, v.b, carry.b);
-        if (state == 2) return carry;
-        ma = cmul(ma, mult_a);
-        mb = cmul(mb, mult_b);
+        float2 v[kWindow];
+#pragma unroll
+        for (int i = 0; i < kWindow; ++i)
+            if (i < n)
+                v[i] = __ldcg((st[i] == 2 ? k.incl : k.agg) +
+                              (size_t)(item - (back + i) * k.nchains) * kScanThreads + threadIdx.x);
+#pragma unroll
+        for (int i = 0; i < kWindow; ++i)
+            if (i < n) {
+                carry = cfma(m, v[i], carry);
+                m = cfma2(mult, mult_lo, m, make_float2(0.f, 0.f));
+            }
+        if (closed) return carry;
+        back += n;
     }
 }
 
-// Decodes the ticket: chunks of one (sequence, state group) are consecutive items.
-struct Item {
-    int item, c, pg, b;
-};
-__device__ __forceinline__ Item take_item(const ChunkArgs& k) {
+// One ticket for the CTA.  All threads call it.
+__device__ __forceinline__ int take_ticket(const ChunkArgs& k) {
     __shared__ int s_item;
+    __syncthreads();   // everybody has read the previous ticket
     if (threadIdx.x == 0) s_item = atomicAdd(k.ticket, 1);
     __syncthreads();
-    Item it;
-    it.item = s_item;
-    it.c = it.item % k.nchunks;
-    const int rest = it.item / k.nchunks;
-    it.pg = rest % k.npg;
-    it.b = rest / k.npg;
-    return it;
+    return s_item;
 }
 
-// Bit i of the result: step t0 + i carries a done flag (i < len <= 32).
-__device__ __forceinline__ uint32_t done_mask(const uint8_t* done, size_t row0, int len) {
-    if (!done) return 0u;
-    const int lane = threadIdx.x & 31;
-    const bool f = lane < len && done[row0 + lane] != 0;
-    return __ballot_sync(0xffffffffu, f);
+struct Where {
+    int item, ci, c, b, p, len;   // ci: position in processing order; c: chunk index in time
+    size_t row0;       // (b * T + t0)
+    uint32_t mask;     // bit i: step t0 + i carries a done flag
+    bool active;       // this thread's state exists
+};
+
+// `from_end`: items count chunks from the end of the sequence (backward pass).
+template <int L>
+__device__ __forceinline__ Where locate(const ChunkArgs& k, int item, bool from_end) {
+    Where w;
+    w.item = item;
+    const int ci = item / k.nchains;      // position in processing order
+    const int chain = item - ci * k.nchains;
+    const int pg = chain % k.npg;
+    w.b = chain / k.npg;
+    w.ci = ci;
+    w.c = from_end ? k.nchunks - 1 - ci : ci;
+    w.p = pg * kScanThreads + threadIdx.x;
+    w.active = w.p < k.P;
+    const int t0 = w.c * L;
+    w.len = min(L, k.T - t0);
+    w.row0 = (size_t)w.b * k.T + t0;
+    w.mask = 0u;
+    if (k.done) {
+        const int lane = threadIdx.x & 31;
+        const bool f = lane < w.len && k.done[w.row0 + lane] != 0;
+        w.mask = __ballot_sync(0xffffffffu, f);
+    }
+    return w;
 }
 
-template <int L, typename XT>
+template <int L, typename XS>
 __global__ void __launch_bounds__(kScanThreads)
-scan_fwd_chunk_kernel(ChunkArgs k, const float4* Bu, const float4* __restrict__ x0, XT* x,
-                      float4* __restrict__ xT) {
+scan_fwd_chunk_kernel(ChunkArgs k, const float2* Bu, const float2* __restrict__ x0, XS* x,
+                      float2* __restrict__ xT) {
     static_assert(L <= 32 && (L & (L - 1)) == 0, "chunk length: power of two, at most 32");
-    const Item it = take_item(k);
     const int tid = threadIdx.x;
-    const int pp = it.pg * kScanThreads + tid;
-    const size_t plane = (size_t)k.B * k.T * k.P2;
-    const int t0 = it.c * L;
-    const int len = min(L, k.T - t0);
-    const size_t row0 = (size_t)it.b * k.T + t0;
-    const uint32_t mask = done_mask(k.done, row0, len);
-    if (pp >= k.P2) return;
-    const C2 a = c2_from(k.Abar[pp]);
-    const float4* src = Bu + row0 * k.P2 + pp;
-    C2 v[L];
+    const size_t plane = (size_t)k.B * k.T * k.P;
+    struct Buf {
+        Where w;
+        float2 v[L];
+    };
+    auto fetch = [&](int item, Buf& q) {
+        q.w = locate<L>(k, item, false);
+        if (!q.w.active) return;
+        const float2* src = Bu + q.w.row0 * k.P + q.w.p;
 #pragma unroll
-    for (int i = 0; i < L; ++i)
-        if (i < len) v[i] = StateIO<float4>::load(src + (size_t)i * k.P2, 0);
-    // fold from a zero state: the chunk's aggregate
-    C2 e = c2_zero();
+        for (int i = 0; i < L; ++i)
+            if (i < q.w.len) q.v[i] = __ldcs(src + (size_t)i * k.P);
+    };
+    auto process = [&](const Buf& q) {
+        const Where& w = q.w;
+        const float2 a = w.active ? k.Abar[w.p] : make_float2(0.f, 0.f);
+        const float2 al = (w.active && k.Alo) ? k.Alo[w.p] : make_float2(0.f, 0.f);
+        // fold from a zero state: the chunk's aggregate
+        float2 e = make_float2(0.f, 0.f);
+        if (w.active) {
 #pragma unroll
-    for (int i = 0; i < L; ++i)
-        if (i < len) {
-            if ((mask >> i) & 1u) e = c2_zero();
-            e.a = cfma(a.a, e.a, v[i].a);
-            e.b = cfma(a.b, e.b, v[i].b);
+            for (int i = 0; i < L; ++i)
+                if (i < w.len) {
+                    if ((w.mask >> i) & 1u) e = make_float2(0.f, 0.f);
+                    e = cfma2(a, al, e, q.v[i]);
+                }
         }
-    const bool has_reset = mask != 0u;
-    const bool last = it.c == k.nchunks - 1;
-    const float2 aLa = cpow2<L>(a.a), aLb = cpow2<L>(a.b);
-    const size_t rec = (size_t)it.item * kScanThreads + tid;
-    C2 carry;
-    if (it.c == 0) {
-        carry = x0 ? c2_from(x0[(size_t)it.b * k.P2 + pp]) : c2_zero();
-    } else {
-        if (!last) {
-            if (has_reset) publish(k.incl + rec, k.status + rec, e, 2);
-            else publish(k.agg + rec, k.status + rec, e, 1);
+        const bool has_reset = w.mask != 0u;
+        const bool last = w.c == k.nchunks - 1;
+        float2 aL, aLlo;
+        cpow2_pair<L>(a, al, aL, aLlo);
+        float2 carry;
+        if (w.c == 0) {
+            carry = (x0 && w.active) ? x0[(size_t)w.b * k.P + w.p] : make_float2(0.f, 0.f);
+        } else {
+            if (!last) publish(k, has_reset ? k.incl : k.agg, w.item, e, has_reset ? 2 : 1);
+            carry = look_back(k, w.item, w.ci, aL, aLlo);
         }
-        carry = look_back(k, it.item, tid, aLa, aLb);
+        if (!last && (w.c == 0 || !has_reset))
+            publish(k, k.incl, w.item, has_reset ? e : cfma2(aL, aLlo, carry, e), 2);
+        if (!w.active) return;
+        // fold again from the true entering state and store
+        float2 s = carry;
+        XS* dst = x + w.row0 * k.P + w.p;
+#pragma unroll
+        for (int i = 0; i < L; ++i)
+            if (i < w.len) {
+                if ((w.mask >> i) & 1u) s = make_float2(0.f, 0.f);
+                s = cfma2(a, al, s, q.v[i]);
+                Raw1<XS>::store(dst + (size_t)i * k.P, s, plane);
+            }
+        if (last && xT) xT[(size_t)w.b * k.P + w.p] = s;
+    };
+    Buf q0, q1;
+    int cur = take_ticket(k);
+    if (cur >= k.items) return;
+    fetch(cur, q0);
+    for (;;) {
+        int nxt = take_ticket(k);
+        if (nxt < k.items) fetch(nxt, q1);
+        process(q0);
+        if (nxt >= k.items) break;
+        nxt = take_ticket(k);
+        if (nxt < k.items) fetch(nxt, q0);
+        process(q1);
+        if (nxt >= k.items) break;
     }
-    if (!last && (it.c == 0 || !has_reset)) {
-        C2 inc = e;
-        if (!has_reset) {
-            inc.a = cfma(aLa, carry.a, e.a);
-            inc.b = cfma(aLb, carry.b, e.b);
-        }
-        publish(k.incl + rec, k.status + rec, inc, 2);
-    }
-    // fold again from the true entering state and store
-    C2 s = carry;
-    XT* dst = x + row0 * k.P2 + pp;
-#pragma unroll
-    for (int i = 0; i < L; ++i)
-        if (i < len) {
-            if ((mask >> i) & 1u) s = c2_zero();
-            s.a = cfma(a.a, s.a, v[i].a);
-            s.b = cfma(a.b, s.b, v[i].b);
-            StateIO<XT>::store(dst + (size_t)i * k.P2, s, plane);
-        }
-    if (last && xT) xT[(size_t)it.b * k.P2 + pp] = c2_pack(s);
 }
 
 // Backward: chunks are taken from the end of the sequence; the carried quantity is
 // c_{t-1} = keep_t conj(Abar) (gx_t + c_t), a recurrence of the same form run in reverse.
-template <int L, typename XT, typename ST>
+// gAbar: each CTA keeps one row of partial sums (one entry per state), zeroed by itself first.
+template <int L, typename XS>
 __global__ void __launch_bounds__(kScanThreads)
-scan_bwd_chunk_kernel(ChunkArgs k, const float4* __restrict__ x0, const XT* __restrict__ x, const float4* gx,
-                      const float4* __restrict__ gxT, ST* gBu, float4* __restrict__ gA_part,
-                      float4* __restrict__ gx0) {
+scan_bwd_chunk_kernel(ChunkArgs k, const float2* __restrict__ x0, const XS* __restrict__ x, const float2* gx,
+                      const float2* __restrict__ gxT, XS* gBu, float2* __restrict__ gA_part,
+                      float2* __restrict__ gx0) {
     static_assert(L <= 32 && (L & (L - 1)) == 0, "chunk length: power of two, at most 32");
-    const Item it = take_item(k);
     const int tid = threadIdx.x;
-    const int pp = it.pg * kScanThreads + tid;
-    const size_t plane = (size_t)k.B * k.T * k.P2;
-    const int c = k.nchunks - 1 - it.c;          // chunk index in time; it.c counts from the end
-    const int t0 = c * L;
-    const int len = min(L, k.T - t0);
-    const size_t row0 = (size_t)it.b * k.T + t0;
-    const uint32_t mask = done_mask(k.done, row0, len);
-    if (pp >= k.P2) return;
-    const C2 a = c2_from(k.Abar[pp]);
-    const float2 ac0 = cconj(a.a), ac1 = cconj(a.b);
-    const float4* gsrc = gx + row0 * k.P2 + pp;
-    const XT* xsrc = x + row0 * k.P2 + pp;
-    C2 v[L], xp[L];
+    const size_t plane = (size_t)k.B * k.T * k.P;
+    float2* my_part = gA_part + (size_t)blockIdx.x * k.P;
+    for (int p = tid; p < k.P; p += kScanThreads) my_part[p] = make_float2(0.f, 0.f);
+    struct Buf {
+        Where w;
+        float2 v[L];
+        Raw1<XS> xp[L];
+    };
+    auto fetch = [&](int item, Buf& q) {
+        q.w = locate<L>(k, item, true);
+        if (!q.w.active) return;
+        const float2* gsrc = gx + q.w.row0 * k.P + q.w.p;
+        const XS* xsrc = x + q.w.row0 * k.P + q.w.p;
+        const bool at_start = q.w.c == 0;
 #pragma unroll
-    for (int i = 0; i < L; ++i)
-        if (i < len) {
-            v[i] = StateIO<float4>::load(gsrc + (size_t)i * k.P2, 0);
-            if (t0 + i > 0) xp[i] = StateIO<XT>::load(xsrc + ((ptrdiff_t)i - 1) * k.P2, plane);
-            else xp[i] = x0 ? c2_from(x0[(size_t)it.b * k.P2 + pp]) : c2_zero();
-        }
-    // fold from a zero carry: aggregate = c_{t0-1} given c_{t1-1} = 0
-    C2 e = c2_zero();
-#pragma unroll
-    for (int i = L - 1; i >= 0; --i)
-        if (i < len) {
-            if ((mask >> i) & 1u) {
-                e = c2_zero();
-            } else {
-                e.a = cmul(ac0, cadd(v[i].a, e.a));
-                e.b = cmul(ac1, cadd(v[i].b, e.b));
+        for (int i = 0; i < L; ++i)
+            if (i < q.w.len) {
+                q.v[i] = __ldcs(gsrc + (size_t)i * k.P);
+                if (!(at_start && i == 0)) q.xp[i].load(xsrc + ((ptrdiff_t)i - 1) * k.P, plane);
             }
+    };
+    auto process = [&](const Buf& q) {
+        const Where& w = q.w;
+        const float2 ac = w.active ? cconj(k.Abar[w.p]) : make_float2(0.f, 0.f);
+        const float2 acl = (w.active && k.Alo) ? cconj(k.Alo[w.p]) : make_float2(0.f, 0.f);
+        const float2 zero2 = make_float2(0.f, 0.f);
+        // fold from a zero carry: aggregate = c_{t0-1} given c_{t1-1} = 0
+        float2 e = make_float2(0.f, 0.f);
+        if (w.active) {
+#pragma unroll
+            for (int i = L - 1; i >= 0; --i)
+                if (i < w.len) e = ((w.mask >> i) & 1u) ? zero2 : cfma2(ac, acl, cadd(q.v[i], e), zero2);
         }
-    const bool has_reset = mask != 0u;
-    const bool first_item = it.c == 0;           // the chunk at the end of the sequence
-    const bool final_item = it.c == k.nchunks - 1;  // the chunk at t = 0: nobody looks at it
-    const float2 aLa = cpow2<L>(ac0), aLb = cpow2<L>(ac1);
-    const size_t rec = (size_t)it.item * kScanThreads + tid;
-    C2 carry;
-    if (first_item) {
-        carry = gxT ? c2_from(gxT[(size_t)it.b * k.P2 + pp]) : c2_zero();
-    } else {
-        if (!final_item) {
-            if (has_reset) publish(k.incl + rec, k.status + rec, e, 2);
-            else publish(k.agg + rec, k.status + rec, e, 1);
+        const bool has_reset = w.mask != 0u;
+        const bool first_item = w.c == k.nchunks - 1;   // the chunk at the end of the sequence
+        const bool final_item = w.c == 0;               // the chunk at t = 0: nobody looks at it
+        float2 aL, aLlo;
+        cpow2_pair<L>(ac, acl, aL, aLlo);
+        float2 carry;
+        if (first_item) {
+            carry = (gxT && w.active) ? gxT[(size_t)w.b * k.P + w.p] : make_float2(0.f, 0.f);
+        } else {
+            if (!final_item) publish(k, has_reset ? k.incl : k.agg, w.item, e, has_reset ? 2 : 1);
+            carry = look_back(k, w.item, w.ci, aL, aLlo);
         }
-        carry = look_back(k, it.item, tid, aLa, aLb);
-    }
-    if (!final_item && (first_item || !has_reset)) {
-        C2 inc = e;
-        if (!has_reset) {
-            // a short chunk at the end of the sequence multiplies by conj(Abar)^len
-            float2 pa = aLa, pb = aLb;
-            if (len != L) {
-                pa = make_float2(1.f, 0.f);
-                pb = pa;
-                for (int i = 0; i < len; ++i) {
-                    pa = cmul(pa, ac0);
-                    pb = cmul(pb, ac1);
+        if (!final_item && (first_item || !has_reset)) {
+            float2 inc = e;
+            if (!has_reset) {
+                float2 pw = aL, pwl = aLlo;   // a short chunk at the end multiplies by conj(Abar)^len
+                if (w.len != L) {
+                    pw = make_float2(1.f, 0.f);
+                    pwl = zero2;
+                    for (int i = 0; i < w.len; ++i) pw = cfma2(ac, acl, pw, zero2);
+                }
+                inc = cfma2(pw, pwl, carry, e);
+            }
+            publish(k, k.incl, w.item, inc, 2);
+        }
+        if (!w.active) return;
+        // true pass
+        float2 cc = carry, g = make_float2(0.f, 0.f);
+        XS* dst = gBu + w.row0 * k.P + w.p;
+        const float2 xinit = (final_item && x0) ? x0[(size_t)w.b * k.P + w.p] : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = L - 1; i >= 0; --i)
+            if (i < w.len) {
+                const float2 s = cadd(q.v[i], cc);
+                Raw1<XS>::store(dst + (size_t)i * k.P, s, plane);
+                if ((w.mask >> i) & 1u) {
+                    cc = make_float2(0.f, 0.f);
+                } else {
+                    const float2 xprev = (final_item && i == 0) ? xinit : q.xp[i].get();
+                    g = cfma(s, cconj(xprev), g);
+                    cc = cfma2(ac, acl, s, zero2);
                 }
             }
-            inc.a = cfma(pa, carry.a, e.a);
-            inc.b = cfma(pb, carry.b, e.b);
-        }
-        publish(k.incl + rec, k.status + rec, inc, 2);
+        my_part[w.p] = cadd(my_part[w.p], g);   // only this thread touches this entry of this row
+        if (final_item && gx0) gx0[(size_t)w.b * k.P + w.p] = cc;
+    };
+    Buf q0, q1;
+    int cur = take_ticket(k);
+    if (cur >= k.items) return;
+    fetch(cur, q0);
+    for (;;) {
+        int nxt = take_ticket(k);
+        if (nxt < k.items) fetch(nxt, q1);
+        process(q0);
+        if (nxt >= k.items) break;
+        nxt = take_ticket(k);
+        if (nxt < k.items) fetch(nxt, q0);
+        process(q1);
+        if (nxt >= k.items) break;
     }
-    // true pass
-    C2 cc = carry, g = c2_zero();
-    ST* dst = gBu + row0 * k.P2 + pp;
-#pragma unroll
-    for (int i = L - 1; i >= 0; --i)
-        if (i < len) {
-            const C2 s{cadd(v[i].a, cc.a), cadd(v[i].b, cc.b)};
-            StateIO<ST>::store(dst + (size_t)i * k.P2, s, plane);
-            if ((mask >> i) & 1u) {
-                cc = c2_zero();
-            } else {
-                g.a = cfma(s.a, cconj(xp[i].a), g.a);
-                g.b = cfma(s.b, cconj(xp[i].b), g.b);
-                cc.a = cmul(ac0, s.a);
-                cc.b = cmul(ac1, s.b);
-            }
-        }
-    gA_part[((size_t)it.b * k.nchunks + c) * k.P2 + pp] = c2_pack(g);
-    if (final_item && gx0) gx0[(size_t)it.b * k.P2 + pp] = c2_pack(cc);
 }
 
 // =============================================================================================
@@ -473,12 +588,27 @@ scan_bwd_chunk_kernel(ChunkArgs k, const float4* __restrict__ x0, const XT* __re
 // =============================================================================================
 namespace {
 
+constexpr int kChunkCtasPerSm = 4;
+
 struct ScanPlan {
     bool chunked;
-    int L, nchunks, npg, items;
+    int L, nchunks, npg, items, grid;
     size_t off_status, off_agg, off_incl, off_part, off_tmp, zero_bytes, total;
     int part_rows;
 };
+
+int scan_sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = 148;
+        }
+    }
+    return n;
+}
 
 ScanPlan plan_scan(int B, int T, int P, int L) {
     ScanPlan s{};
@@ -487,39 +617,44 @@ ScanPlan plan_scan(int B, int T, int P, int L) {
     s.chunked = T >= 2 * L && (size_t)B * P2 < (size_t)16 * 1024;
     s.L = L;
     s.nchunks = s.chunked ? (T + L - 1) / L : 1;
-    s.npg = (P2 + kScanThreads - 1) / kScanThreads;
+    s.npg = (P + kScanThreads - 1) / kScanThreads;
     s.items = B * s.npg * s.nchunks;
+    const int max_grid = scan_sm_count() * kChunkCtasPerSm;
+    s.grid = s.items < max_grid ? s.items : max_grid;
     size_t off = sizeof(ScanCounters);
     s.off_status = off;
-    off += s.chunked ? align_up((size_t)s.items * kScanThreads * 4, 256) : 0;
+    off += s.chunked ? align_up((size_t)s.items * 4, 256) : 0;
     s.zero_bytes = off;
     s.off_agg = off;
-    off += s.chunked ? (size_t)s.items * kScanThreads * 16 : 0;
+    off += s.chunked ? (size_t)s.items * kScanThreads * 8 : 0;
     s.off_incl = off;
-    off += s.chunked ? (size_t)s.items * kScanThreads * 16 : 0;
-    s.part_rows = B * s.nchunks;
+    off += s.chunked ? (size_t)s.items * kScanThreads * 8 : 0;
+    s.part_rows = s.chunked ? 148 * 2 * kChunkCtasPerSm : B;   // upper bound on the grid, any device
     s.off_part = off;
-    off += align_up((size_t)s.part_rows * P2 * 16, 256);
+    off += align_up((size_t)s.part_rows * P * 8, 256);
     s.off_tmp = off;
     off += align_up(colsum_tmp_floats(s.part_rows, 2 * P) * 4, 256);
     s.total = off;
     return s;
 }
 
-ChunkArgs chunk_args(const ScanPlan& s, int B, int T, int P, const float2* Abar, const uint8_t* done,
+ChunkArgs chunk_args(const ScanPlan& s, int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done,
                      WsHeader* hdr, char* scratch) {
     ChunkArgs k;
     k.B = B;
     k.T = T;
-    k.P2 = P / 2;
+    k.P = P;
     k.nchunks = s.nchunks;
     k.npg = s.npg;
-    k.Abar = (const float4*)Abar;
+    k.nchains = B * s.npg;
+    k.items = s.items;
+    k.Abar = Abar;
+    k.Alo = Alo;
     k.done = done;
     k.ticket = &reinterpret_cast<ScanCounters*>(scratch)->ticket;
     k.status = reinterpret_cast<int*>(scratch + s.off_status);
-    k.agg = reinterpret_cast<float4*>(scratch + s.off_agg);
-    k.incl = reinterpret_cast<float4*>(scratch + s.off_incl);
+    k.agg = reinterpret_cast<float2*>(scratch + s.off_agg);
+    k.incl = reinterpret_cast<float2*>(scratch + s.off_incl);
     k.hdr = hdr;
     return k;
 }
@@ -531,7 +666,7 @@ size_t scan_scratch_bytes(int B, int T, int P) {
     return align_up(f > b ? f : b, 256);
 }
 
-int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Bu, const uint8_t* done,
+int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu, const uint8_t* done,
                     const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr, void* scratch,
                     cudaStream_t st) {
     const int P2 = P / 2;
@@ -540,59 +675,57 @@ int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Bu, c
         const int blocks = (int)(((size_t)B * P2 + kSeqThreads - 1) / kSeqThreads);
         count_launch();
         if (x_bf16)
-            scan_fwd_seq_kernel<uint2><<<blocks, kSeqThreads, 0, st>>>(B, T, P2, (const float4*)Abar, (const float4*)Bu,
+            scan_fwd_seq_kernel<uint2><<<blocks, kSeqThreads, 0, st>>>(B, T, P2, (const float4*)Abar, (const float4*)Alo, (const float4*)Bu,
                                                                        done, (const float4*)x0, (uint2*)x, (float4*)xT);
         else
-            scan_fwd_seq_kernel<float4><<<blocks, kSeqThreads, 0, st>>>(B, T, P2, (const float4*)Abar, (const float4*)Bu,
+            scan_fwd_seq_kernel<float4><<<blocks, kSeqThreads, 0, st>>>(B, T, P2, (const float4*)Abar, (const float4*)Alo, (const float4*)Bu,
                                                                         done, (const float4*)x0, (float4*)x, (float4*)xT);
         return SSM_OK;
     }
     if (cudaMemsetAsync(scratch, 0, s.zero_bytes, st) != cudaSuccess) return SSM_ERR_CUDA;
-    const ChunkArgs k = chunk_args(s, B, T, P, Abar, done, hdr, (char*)scratch);
+    const ChunkArgs k = chunk_args(s, B, T, P, Abar, Alo, done, hdr, (char*)scratch);
     count_launch();
     if (x_bf16)
-        scan_fwd_chunk_kernel<kFwdChunk, uint2><<<s.items, kScanThreads, 0, st>>>(k, (const float4*)Bu, (const float4*)x0,
-                                                                                 (uint2*)x, (float4*)xT);
+        scan_fwd_chunk_kernel<kFwdChunk, uint32_t><<<s.grid, kScanThreads, 0, st>>>(k, Bu, x0, (uint32_t*)x, xT);
     else
-        scan_fwd_chunk_kernel<kFwdChunk, float4><<<s.items, kScanThreads, 0, st>>>(k, (const float4*)Bu, (const float4*)x0,
-                                                                                  (float4*)x, (float4*)xT);
+        scan_fwd_chunk_kernel<kFwdChunk, float2><<<s.grid, kScanThreads, 0, st>>>(k, Bu, x0, (float2*)x, xT);
     return SSM_OK;
 }
 
-int launch_scan_bwd(int B, int T, int P, const float2* Abar, const uint8_t* done, const float2* x0,
+int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done, const float2* x0,
                     const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
                     float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st) {
     const int P2 = P / 2;
     const ScanPlan s = plan_scan(B, T, P, kBwdChunk);
     char* base = (char*)scratch;
-    float4* part = reinterpret_cast<float4*>(base + s.off_part);
+    float* part = reinterpret_cast<float*>(base + s.off_part);
     float* tmp = reinterpret_cast<float*>(base + s.off_tmp);
     if (x_bf16 != s_bf16) return SSM_ERR_DTYPE;
+    int rows = B;
     if (!s.chunked) {
         const int blocks = (int)(((size_t)B * P2 + kSeqThreads - 1) / kSeqThreads);
         count_launch();
         if (x_bf16)
             scan_bwd_seq_kernel<uint2, uint2><<<blocks, kSeqThreads, 0, st>>>(
-                B, T, P2, (const float4*)Abar, done, (const float4*)x0, (const uint2*)x, (const float4*)gx,
-                (const float4*)gxT, (uint2*)gBu, part, (float4*)gx0);
+                B, T, P2, (const float4*)Abar, (const float4*)Alo, done, (const float4*)x0, (const uint2*)x, (const float4*)gx,
+                (const float4*)gxT, (uint2*)gBu, (float4*)part, (float4*)gx0);
         else
             scan_bwd_seq_kernel<float4, float4><<<blocks, kSeqThreads, 0, st>>>(
-                B, T, P2, (const float4*)Abar, done, (const float4*)x0, (const float4*)x, (const float4*)gx,
-                (const float4*)gxT, (float4*)gBu, part, (float4*)gx0);
+                B, T, P2, (const float4*)Abar, (const float4*)Alo, done, (const float4*)x0, (const float4*)x, (const float4*)gx,
+                (const float4*)gxT, (float4*)gBu, (float4*)part, (float4*)gx0);
     } else {
         if (cudaMemsetAsync(scratch, 0, s.zero_bytes, st) != cudaSuccess) return SSM_ERR_CUDA;
-        const ChunkArgs k = chunk_args(s, B, T, P, Abar, done, hdr, base);
+        const ChunkArgs k = chunk_args(s, B, T, P, Abar, Alo, done, hdr, base);
+        rows = s.grid < s.part_rows ? s.grid : s.part_rows;
         count_launch();
         if (x_bf16)
-            scan_bwd_chunk_kernel<kBwdChunk, uint2, uint2><<<s.items, kScanThreads, 0, st>>>(
-                k, (const float4*)x0, (const uint2*)x, (const float4*)gx, (const float4*)gxT, (uint2*)gBu, part,
-                (float4*)gx0);
+            scan_bwd_chunk_kernel<kBwdChunk, uint32_t><<<rows, kScanThreads, 0, st>>>(
+                k, x0, (const uint32_t*)x, gx, gxT, (uint32_t*)gBu, (float2*)part, gx0);
         else
-            scan_bwd_chunk_kernel<kBwdChunk, float4, float4><<<s.items, kScanThreads, 0, st>>>(
-                k, (const float4*)x0, (const float4*)x, (const float4*)gx, (const float4*)gxT, (float4*)gBu, part,
-                (float4*)gx0);
+            scan_bwd_chunk_kernel<kBwdChunk, float2><<<rows, kScanThreads, 0, st>>>(
+                k, x0, (const float2*)x, gx, gxT, (float2*)gBu, (float2*)part, gx0);
     }
-    launch_colsum((const float*)part, s.part_rows, 2 * P, (float*)gAbar, tmp, st);
+    launch_colsum(part, rows, 2 * P, (float*)gAbar, tmp, st);
     return SSM_OK;
 }
 

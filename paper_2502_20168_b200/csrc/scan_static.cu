@@ -57,7 +57,7 @@ SSM_API int ssm_scan_bwd_static(const ssm_shape* shape, const ssm_c64* Abar, con
     // The array keeps whatever the previous call left; the header (status word, chunk
     // ticket) is the part that has to start at zero.
     if (cudaMemsetAsync(base, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
-    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, done, (const float2*)x0,
+    int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, nullptr, done, (const float2*)x0,
                              (const float2*)x, false, (const float2*)gx, (const float2*)gxT, (float2*)gBu, false,
                              (float2*)gAbar, (float2*)gx0, reinterpret_cast<WsHeader*>(base),
                              reinterpret_cast<char*>(base) + sizeof(WsHeader), st);
