@@ -20,6 +20,9 @@
 //
 // States are stored as fp32 pairs, or as bf16 pairs when they only feed bf16 tensor-core
 // operands (the arithmetic and the carried state stay fp32).
+#include <atomic>
+#include <chrono>
+
 #include "kernels.h"
 
 namespace ssm {
@@ -253,9 +256,14 @@ scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
 // (sequence, group of 128 states)), so the chunks in flight at any moment are spread over all
 // chains and the carry of every chain advances at the same time.
 //
-// Scratch layout: [ScanCounters (256 B)][status: one int per item][agg: items*128 float2]
-// [incl: items*128 float2][gA partials (backward): grid rows of P float2][column-sum scratch].
-// Everything up to the end of `status` is zeroed before each launch.
+// A chunk's record for one state is a single 16-byte word {value, launch tag, state}: it is
+// written and read with one 16-byte access, so no fence has to order a value against its flag
+// (a fence would also wait for the prefetched loads).  The 62-bit tag is unique to the launch;
+// whatever an earlier launch or nobody left in the scratch memory does not match it, so the
+// records need no clearing.  state: 1 = aggregate of the chunk alone, 2 = inclusive.
+//
+// Scratch layout: [ScanCounters (256 B), zeroed before each launch][records: items*128 x 16 B]
+// [gA partials (backward): grid rows of P float2][column-sum scratch].
 struct ScanCounters {
     int ticket;
     int pad[63];
@@ -267,9 +275,8 @@ struct ChunkArgs {
     const float2* Alo;     // low part of Abar as an fp32 pair, or NULL
     const uint8_t* done;
     int* ticket;
-    int* status;
-    float2* agg;
-    float2* incl;
+    uint4* rec;
+    uint32_t tag_hi, tag_lo;   // tag_lo has its two low bits clear
     WsHeader* hdr;
 };
 
@@ -301,19 +308,19 @@ template <> struct Raw1<uint32_t> {
     }
 };
 
-// The CTA publishes one record (128 values, then the item's state word).  All threads call it.
-__device__ __forceinline__ void publish(const ChunkArgs& k, float2* values, int item, float2 v, int state) {
-    values[(size_t)item * kScanThreads + threadIdx.x] = v;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) *reinterpret_cast<volatile int*>(k.status + item) = state;
+__device__ __forceinline__ void publish(const ChunkArgs& k, int item, float2 v, uint32_t state) {
+    uint4 r;
+    r.x = __float_as_uint(v.x);
+    r.y = __float_as_uint(v.y);
+    r.z = k.tag_hi;
+    r.w = k.tag_lo | state;
+    __stcg(k.rec + (size_t)item * kScanThreads + threadIdx.x, r);
 }
 
 // State entering chunk `ci` of a chain, from the records of the chain's earlier chunks (items
 // item - nchains, item - 2 nchains, ...).  `mult` is the per-chunk multiplier (Abar^L or its
-// conjugate).  A window of kWindow predecessors is inspected at a time, their state words and
-// values fetched with independent loads, so a long run of aggregates costs a few round trips
-// instead of one per chunk.  Control flow is uniform over the CTA (state words are per item).
+// conjugate) as an fp32 pair.  A window of kWindow predecessors is fetched with independent
+// loads, so a long run of aggregates costs a few round trips instead of one per chunk.
 // Bounded: gives up into hdr->status.
 constexpr int kWindow = 8;
 __device__ __forceinline__ float2 look_back(const ChunkArgs& k, int item, int ci, float2 mult, float2 mult_lo) {
@@ -322,20 +329,23 @@ __device__ __forceinline__ float2 look_back(const ChunkArgs& k, int item, int ci
     int back = 1;             // next predecessor to absorb: chunk ci - back
     uint32_t polls = 0;
     for (;;) {
-        int st[kWindow];
+        uint4 r[kWindow];
 #pragma unroll
         for (int i = 0; i < kWindow; ++i) {
             const int d = back + i;
-            st[i] = d <= ci ? *reinterpret_cast<volatile int*>(k.status + (item - d * k.nchains)) : 0;
+            r[i] = d <= ci ? __ldcv(k.rec + (size_t)(item - d * k.nchains) * kScanThreads + threadIdx.x)
+                           : make_uint4(0u, 0u, 0u, 0u);
         }
         int n = 0;            // predecessors usable now: a ready prefix, cut after the first inclusive one
         bool closed = false;
 #pragma unroll
-        for (int i = 0; i < kWindow; ++i)
-            if (n == i && !closed && st[i] != 0) {
+        for (int i = 0; i < kWindow; ++i) {
+            const bool ready = r[i].z == k.tag_hi && (r[i].w & ~3u) == k.tag_lo && (r[i].w & 3u) != 0u && back + i <= ci;
+            if (n == i && !closed && ready) {
                 n = i + 1;
-                closed = st[i] == 2;
+                closed = (r[i].w & 3u) == 2u;
             }
+        }
         if (n == 0) {
             if (++polls > kPollLimit) {
                 k.hdr->status = SSM_ERR_TIMEOUT;
@@ -344,17 +354,10 @@ __device__ __forceinline__ float2 look_back(const ChunkArgs& k, int item, int ci
             __nanosleep(20);
             continue;
         }
-        __threadfence();
-        float2 v[kWindow];
-#pragma unroll
-        for (int i = 0; i < kWindow; ++i)
-            if (i < n)
-                v[i] = __ldcg((st[i] == 2 ? k.incl : k.agg) +
-                              (size_t)(item - (back + i) * k.nchains) * kScanThreads + threadIdx.x);
 #pragma unroll
         for (int i = 0; i < kWindow; ++i)
             if (i < n) {
-                carry = cfma(m, v[i], carry);
+                carry = cfma(m, make_float2(__uint_as_float(r[i].x), __uint_as_float(r[i].y)), carry);
                 m = cfma2(mult, mult_lo, m, make_float2(0.f, 0.f));
             }
         if (closed) return carry;
@@ -408,7 +411,6 @@ __global__ void __launch_bounds__(kScanThreads)
 scan_fwd_chunk_kernel(ChunkArgs k, const float2* Bu, const float2* __restrict__ x0, XS* x,
                       float2* __restrict__ xT) {
     static_assert(L <= 32 && (L & (L - 1)) == 0, "chunk length: power of two, at most 32");
-    const int tid = threadIdx.x;
     const size_t plane = (size_t)k.B * k.T * k.P;
     struct Buf {
         Where w;
@@ -444,12 +446,12 @@ scan_fwd_chunk_kernel(ChunkArgs k, const float2* Bu, const float2* __restrict__ 
         if (w.c == 0) {
             carry = (x0 && w.active) ? x0[(size_t)w.b * k.P + w.p] : make_float2(0.f, 0.f);
         } else {
-            if (!last) publish(k, has_reset ? k.incl : k.agg, w.item, e, has_reset ? 2 : 1);
-            carry = look_back(k, w.item, w.ci, aL, aLlo);
+            if (!last && w.active) publish(k, w.item, e, has_reset ? 2u : 1u);
+            if (w.active) carry = look_back(k, w.item, w.ci, aL, aLlo);
+            else carry = make_float2(0.f, 0.f);
         }
-        if (!last && (w.c == 0 || !has_reset))
-            publish(k, k.incl, w.item, has_reset ? e : cfma2(aL, aLlo, carry, e), 2);
         if (!w.active) return;
+        if (!last && (w.c == 0 || !has_reset)) publish(k, w.item, has_reset ? e : cfma2(aL, aLlo, carry, e), 2u);
         // fold again from the true entering state and store
         float2 s = carry;
         XS* dst = x + w.row0 * k.P + w.p;
@@ -530,9 +532,11 @@ scan_bwd_chunk_kernel(ChunkArgs k, const float2* __restrict__ x0, const XS* __re
         if (first_item) {
             carry = (gxT && w.active) ? gxT[(size_t)w.b * k.P + w.p] : make_float2(0.f, 0.f);
         } else {
-            if (!final_item) publish(k, has_reset ? k.incl : k.agg, w.item, e, has_reset ? 2 : 1);
-            carry = look_back(k, w.item, w.ci, aL, aLlo);
+            if (!final_item && w.active) publish(k, w.item, e, has_reset ? 2u : 1u);
+            if (w.active) carry = look_back(k, w.item, w.ci, aL, aLlo);
+            else carry = zero2;
         }
+        if (!w.active) return;
         if (!final_item && (first_item || !has_reset)) {
             float2 inc = e;
             if (!has_reset) {
@@ -544,9 +548,8 @@ scan_bwd_chunk_kernel(ChunkArgs k, const float2* __restrict__ x0, const XS* __re
                 }
                 inc = cfma2(pw, pwl, carry, e);
             }
-            publish(k, k.incl, w.item, inc, 2);
+            publish(k, w.item, inc, 2u);
         }
-        if (!w.active) return;
         // true pass
         float2 cc = carry, g = make_float2(0.f, 0.f);
         XS* dst = gBu + w.row0 * k.P + w.p;
@@ -593,7 +596,7 @@ constexpr int kChunkCtasPerSm = 4;
 struct ScanPlan {
     bool chunked;
     int L, nchunks, npg, items, grid;
-    size_t off_status, off_agg, off_incl, off_part, off_tmp, zero_bytes, total;
+    size_t off_rec, off_part, off_tmp, zero_bytes, total;
     int part_rows;
 };
 
@@ -610,6 +613,16 @@ int scan_sm_count() {
     return n;
 }
 
+// A different 62-bit value for every launch of this process (splitmix64 over a counter that
+// starts from the clock).
+uint64_t next_launch_tag() {
+    static std::atomic<uint64_t> counter{(uint64_t)std::chrono::steady_clock::now().time_since_epoch().count()};
+    uint64_t z = counter.fetch_add(0x9E3779B97F4A7C15ull) + 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
 ScanPlan plan_scan(int B, int T, int P, int L) {
     ScanPlan s{};
     const int P2 = P / 2;
@@ -622,13 +635,9 @@ ScanPlan plan_scan(int B, int T, int P, int L) {
     const int max_grid = scan_sm_count() * kChunkCtasPerSm;
     s.grid = s.items < max_grid ? s.items : max_grid;
     size_t off = sizeof(ScanCounters);
-    s.off_status = off;
-    off += s.chunked ? align_up((size_t)s.items * 4, 256) : 0;
     s.zero_bytes = off;
-    s.off_agg = off;
-    off += s.chunked ? (size_t)s.items * kScanThreads * 8 : 0;
-    s.off_incl = off;
-    off += s.chunked ? (size_t)s.items * kScanThreads * 8 : 0;
+    s.off_rec = off;
+    off += s.chunked ? (size_t)s.items * kScanThreads * 16 : 0;
     s.part_rows = s.chunked ? 148 * 2 * kChunkCtasPerSm : B;   // upper bound on the grid, any device
     s.off_part = off;
     off += align_up((size_t)s.part_rows * P * 8, 256);
@@ -652,9 +661,10 @@ ChunkArgs chunk_args(const ScanPlan& s, int B, int T, int P, const float2* Abar,
     k.Alo = Alo;
     k.done = done;
     k.ticket = &reinterpret_cast<ScanCounters*>(scratch)->ticket;
-    k.status = reinterpret_cast<int*>(scratch + s.off_status);
-    k.agg = reinterpret_cast<float2*>(scratch + s.off_agg);
-    k.incl = reinterpret_cast<float2*>(scratch + s.off_incl);
+    k.rec = reinterpret_cast<uint4*>(scratch + s.off_rec);
+    const uint64_t tag = next_launch_tag();
+    k.tag_hi = (uint32_t)(tag >> 32);
+    k.tag_lo = (uint32_t)tag & ~3u;
     k.hdr = hdr;
     return k;
 }
