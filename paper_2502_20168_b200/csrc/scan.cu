@@ -407,7 +407,7 @@ __device__ __forceinline__ Where locate(const ChunkArgs& k, int item, bool from_
 }
 
 template <int L, typename XS>
-__global__ void __launch_bounds__(kScanThreads)
+__global__ void __launch_bounds__(kScanThreads, 4)
 scan_fwd_chunk_kernel(ChunkArgs k, const float2* Bu, const float2* __restrict__ x0, XS* x,
                       float2* __restrict__ xT) {
     static_assert(L <= 32 && (L & (L - 1)) == 0, "chunk length: power of two, at most 32");
@@ -464,19 +464,10 @@ scan_fwd_chunk_kernel(ChunkArgs k, const float2* Bu, const float2* __restrict__ 
             }
         if (last && xT) xT[(size_t)w.b * k.P + w.p] = s;
     };
-    Buf q0, q1;
-    int cur = take_ticket(k);
-    if (cur >= k.items) return;
-    fetch(cur, q0);
-    for (;;) {
-        int nxt = take_ticket(k);
-        if (nxt < k.items) fetch(nxt, q1);
-        process(q0);
-        if (nxt >= k.items) break;
-        nxt = take_ticket(k);
-        if (nxt < k.items) fetch(nxt, q0);
-        process(q1);
-        if (nxt >= k.items) break;
+    Buf q;
+    for (int item = take_ticket(k); item < k.items; item = take_ticket(k)) {
+        fetch(item, q);
+        process(q);
     }
 }
 
@@ -484,7 +475,7 @@ scan_fwd_chunk_kernel(ChunkArgs k, const float2* Bu, const float2* __restrict__ 
 // c_{t-1} = keep_t conj(Abar) (gx_t + c_t), a recurrence of the same form run in reverse.
 // gAbar: each CTA keeps one row of partial sums (one entry per state), zeroed by itself first.
 template <int L, typename XS>
-__global__ void __launch_bounds__(kScanThreads)
+__global__ void __launch_bounds__(kScanThreads, 4)
 scan_bwd_chunk_kernel(ChunkArgs k, const float2* __restrict__ x0, const XS* __restrict__ x, const float2* gx,
                       const float2* __restrict__ gxT, XS* gBu, float2* __restrict__ gA_part,
                       float2* __restrict__ gx0) {
@@ -570,19 +561,10 @@ scan_bwd_chunk_kernel(ChunkArgs k, const float2* __restrict__ x0, const XS* __re
         my_part[w.p] = cadd(my_part[w.p], g);   // only this thread touches this entry of this row
         if (final_item && gx0) gx0[(size_t)w.b * k.P + w.p] = cc;
     };
-    Buf q0, q1;
-    int cur = take_ticket(k);
-    if (cur >= k.items) return;
-    fetch(cur, q0);
-    for (;;) {
-        int nxt = take_ticket(k);
-        if (nxt < k.items) fetch(nxt, q1);
-        process(q0);
-        if (nxt >= k.items) break;
-        nxt = take_ticket(k);
-        if (nxt < k.items) fetch(nxt, q0);
-        process(q1);
-        if (nxt >= k.items) break;
+    Buf q;
+    for (int item = take_ticket(k); item < k.items; item = take_ticket(k)) {
+        fetch(item, q);
+        process(q);
     }
 }
 
@@ -591,7 +573,7 @@ scan_bwd_chunk_kernel(ChunkArgs k, const float2* __restrict__ x0, const XS* __re
 // =============================================================================================
 namespace {
 
-constexpr int kChunkCtasPerSm = 4;
+constexpr int kChunkCtasPerSm = 8;
 
 struct ScanPlan {
     bool chunked;
