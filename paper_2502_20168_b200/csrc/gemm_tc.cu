@@ -25,17 +25,21 @@ constexpr int BM = 128;   // accumulator rows per tile = TMEM lanes
 constexpr int BN = 256;   // accumulator columns per tile
 constexpr int BK = 64;    // bf16 elements per shared-memory row: 128 bytes, one swizzle span
 constexpr int UK = 16;    // K extent of one tcgen05.mma of kind::f16
-constexpr int kStages = 4;
+constexpr int kStages = 4;      // shared-memory stages of the NT kernel (and size of the barrier arrays)
+constexpr int kTnStages = 3;    // the TN kernel gives one stage up for its epilogue buffers
 constexpr int kABytes = BM * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;      // NT kernel: producer, MMA, 4 epilogue warps
+constexpr int kTnEpiWarps = 8;     // TN kernel: two epilogue warps per TMEM lane quarter
+constexpr int kTnThreads = 64 + 32 * kTnEpiWarps;
 constexpr int kTmemCols = 512;  // two accumulator buffers of BN columns
 constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr int kStagingBytes = 4 * 32 * 32 * 4;  // per epilogue warp: 32 rows x 32 fp32 columns
+constexpr int kStagingBytes = kTnEpiWarps * 32 * 32 * 4;  // per epilogue warp: 32 rows x 32 fp32 columns
 constexpr int kMaxDiag = 4096;                  // widest output whose diagonal fits the shared copy
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + kStagingBytes + kMaxDiag * 4 +
-                              1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr size_t kTnSmemBytes = (size_t)kTnStages * kStageBytes + kStagingBytes + kMaxDiag * 4 +
+                                1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr size_t kNtSmemBytes = (size_t)kStages * kStageBytes + 1024 + 256;
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -155,13 +159,14 @@ struct Smem {
     volatile uint32_t* tmem_slot_ptr;
 };
 
-__device__ __forceinline__ Smem carve_smem(uint8_t* raw) {
+// Layout: [stages][epilogue staging][diag copy][barriers]; the NT kernel has no staging / diag.
+__device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging_bytes, int diag_bytes) {
     Smem s;
     uintptr_t base = (reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023;
     s.tiles = reinterpret_cast<uint8_t*>(base);
-    s.staging = s.tiles + (size_t)kStages * kStageBytes;
-    s.diag = reinterpret_cast<float*>(s.staging + kStagingBytes);
-    uint8_t* bars = s.staging + kStagingBytes + kMaxDiag * 4;
+    s.staging = s.tiles + (size_t)stages * kStageBytes;
+    s.diag = reinterpret_cast<float*>(s.staging + staging_bytes);
+    uint8_t* bars = s.staging + staging_bytes + diag_bytes;
     for (int i = 0; i < kStages; ++i) {
         s.full[i] = smem_u32(bars + 8 * i);
         s.empty[i] = smem_u32(bars + 8 * (kStages + i));
@@ -177,7 +182,7 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* raw) {
 }
 
 // Common prologue: barriers, tensor memory.  Returns the TMEM base address.
-__device__ __forceinline__ uint32_t prologue(const Smem& s, int warp, int lane) {
+__device__ __forceinline__ uint32_t prologue(const Smem& s, int warp, int lane, int epilogue_threads) {
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) {
             mbar_init(s.full[i], 1);
@@ -185,7 +190,7 @@ __device__ __forceinline__ uint32_t prologue(const Smem& s, int warp, int lane) 
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(s.tmem_full[i], 1);
-            mbar_init(s.tmem_empty[i], 128);
+            mbar_init(s.tmem_empty[i], epilogue_threads);
         }
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -229,14 +234,14 @@ struct TnParams {
 // kSplitW: columns [0,128) and [128,256) of the accumulator tile are the hi and lo weight
 // halves of the same 128 output columns.
 template <int kEpi, bool kSplitW>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kTnThreads, 1)
 gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw);
+    const Smem s = carve_smem(smem_raw, kTnStages, kStagingBytes, kMaxDiag * 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (kEpi == 1)
-        for (int i = threadIdx.x; i < p.ldo; i += kThreads) s.diag[i] = p.diag[i];
-    const uint32_t tmem_base = prologue(s, warp, lane);
+        for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
+    const uint32_t tmem_base = prologue(s, warp, lane, 32 * kTnEpiWarps);
     const int m_tiles = (p.M + BM - 1) / BM;
     const int total = m_tiles * p.n_tiles;
     constexpr int kOutCols = kSplitW ? BN / 2 : BN;
@@ -256,7 +261,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
                     tma_load_2d(a_dst, &tmA, s.full[stage], kb * BK, m0);
                     tma_load_2d(a_dst + kABytes, &tmW, s.full[stage], kb * BK, n0);
-                    if (++stage == kStages) {
+                    if (++stage == kTnStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -286,7 +291,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                   (uint32_t)((kb | k) != 0));
                     }
                     umma_commit(s.empty[stage]);
-                    if (++stage == kStages) {
+                    if (++stage == kTnStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -297,7 +302,8 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
         }
     } else {
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const int q = warp & 3;          // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp drains
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -306,7 +312,8 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int row0 = m0 + q * 32;   // first of this warp's 32 rows
             // skip[m, n] slabs are fetched kPre slabs ahead of their use (the first ones while the
             // tile's MMAs are still running): lane -> (row i*8 + lane/4, 8 columns) per slab
-            constexpr int kSlabs = kOutCols / 32, kPre = 3;
+            constexpr int kSlabs = kOutCols / 32 / 2, kPre = kSlabs - 1 < 3 ? kSlabs - 1 : 3;
+            const int slab0 = half * kSlabs;   // this warp's slabs: slab0 .. slab0 + kSlabs - 1
             uint4 skb[kPre + 1][4];
             auto load_skip = [&](int slab, uint4 (&dst)[4]) {
 #pragma unroll
@@ -314,7 +321,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const int rr = i * 8 + (lane >> 2);
                     if (row0 + rr < p.M)
                         dst[i] = __ldg(reinterpret_cast<const uint4*>(
-                            p.skip + (size_t)(row0 + rr) * p.ldo + n_out0 + slab * 32 + (lane & 3) * 8));
+                            p.skip + (size_t)(row0 + rr) * p.ldo + n_out0 + (slab0 + slab) * 32 + (lane & 3) * 8));
                 }
             };
             if (kEpi == 1) {
@@ -327,7 +334,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             float4* stg = reinterpret_cast<float4*>(s.staging) + (size_t)(warp - 2) * (32 * 8);
 #pragma unroll
             for (int sl = 0; sl < kSlabs; ++sl) {
-                const int c = sl * 32;
+                const int c = (slab0 + sl) * 32;
                 if (kEpi == 1 && sl + kPre < kSlabs) load_skip(sl + kPre, skb[(sl + kPre) % (kPre + 1)]);
                 // TMEM -> registers: lane = row, 32 consecutive columns
                 uint32_t r[32], r2[32];
@@ -427,9 +434,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBhi,
                   const __grid_constant__ CUtensorMap tmBlo, NtParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw);
+    const Smem s = carve_smem(smem_raw, kStages, 0, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t tmem_base = prologue(s, warp, lane);
+    const uint32_t tmem_base = prologue(s, warp, lane, 128);
     const int tile = blockIdx.x, split = blockIdx.y;
     constexpr int kOutCols = BN / 2;   // accumulator columns [0,128): hi plane, [128,256): lo plane
     const int i0 = (tile / p.j_tiles) * BM, j0 = (tile % p.j_tiles) * kOutCols;
@@ -570,8 +577,8 @@ static int sm_count() {
 }
 
 template <typename K>
-static bool set_smem(K kernel) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) == cudaSuccess;
+static bool set_smem(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
 }
 
 }  // namespace tc
@@ -596,15 +603,15 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     bool ok;
     if (g.store_f32) {
         if (g.split_w) {
-            ok = set_smem(gemm_tc_tn_kernel<0, true>);
-            gemm_tc_tn_kernel<0, true><<<grid, kThreads, kSmemBytes, st>>>(ma, mw, p);
+            ok = set_smem(gemm_tc_tn_kernel<0, true>, kTnSmemBytes);
+            gemm_tc_tn_kernel<0, true><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, p);
         } else {
-            ok = set_smem(gemm_tc_tn_kernel<0, false>);
-            gemm_tc_tn_kernel<0, false><<<grid, kThreads, kSmemBytes, st>>>(ma, mw, p);
+            ok = set_smem(gemm_tc_tn_kernel<0, false>, kTnSmemBytes);
+            gemm_tc_tn_kernel<0, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, p);
         }
     } else {
-        ok = set_smem(gemm_tc_tn_kernel<1, false>);
-        gemm_tc_tn_kernel<1, false><<<grid, kThreads, kSmemBytes, st>>>(ma, mw, p);
+        ok = set_smem(gemm_tc_tn_kernel<1, false>, kTnSmemBytes);
+        gemm_tc_tn_kernel<1, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, p);
     }
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
@@ -633,8 +640,8 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
     NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr};
     dim3 grid((g.I / BM) * j_tiles, g.splits);
     count_launch();
-    const bool ok = set_smem(gemm_tc_nt_kernel);
-    gemm_tc_nt_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mbh, mbl, p);
+    const bool ok = set_smem(gemm_tc_nt_kernel, kNtSmemBytes);
+    gemm_tc_nt_kernel<<<grid, kThreads, kNtSmemBytes, st>>>(ma, mbh, mbl, p);
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
 
