@@ -156,6 +156,33 @@ int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* De
                   ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
                   ssm_c64* dx0, void* stream);
 
+/* ---- stacked sequence model --------------------------------------------------------
+ * n_layers layers of   v = SSM_l(u_l);  u_{l+1} = LayerNorm(u_l + GELU(v)) * ln_weight + ln_bias
+ * (exact erf GELU, LayerNorm over the H features with eps 1e-5), the same done flags in every
+ * layer and a zero initial state.  The paper wraps its S5 SSM in a block of nonlinearity and
+ * gating (Appendix "S5 Sequence Layer", whose schematic is a half-GLU); this post-norm
+ * residual block is the stacked configuration the benchmark defines.  Tensors between layers
+ * (v, u_l and, in the backward pass, their gradients) are stored in io_dtype; arithmetic is fp32.
+ * `params` / `grads` are HOST arrays of n_layers structs holding DEVICE pointers.  The
+ * workspace filled by ssm_stack_fwd is read by ssm_stack_bwd.  Backward: from gout[B,T,H] to
+ * du[B,T,H] and every layer's parameter gradients (overwritten). */
+typedef struct {
+    const ssm_c64* Lambda; const float* Delta; const ssm_c64* Bc; const ssm_c64* Cc; const float* D;
+    const float* ln_weight; const float* ln_bias;   /* [H] each */
+} ssm_stack_params;
+typedef struct {
+    ssm_c64* dLambda; float* dDelta; ssm_c64* dB; ssm_c64* dC; float* dD;
+    float* dln_weight; float* dln_bias;
+} ssm_stack_grads;
+size_t ssm_stack_workspace_bytes(const ssm_shape* shape, int n_layers);
+int ssm_stack_fwd(const ssm_shape* shape, int n_layers, const ssm_stack_params* params,
+                  const void* u /*[B,T,H] io*/, const uint8_t* done /*[B,T] or NULL*/,
+                  void* out /*[B,T,H] io*/, void* ws, size_t ws_bytes, void* stream);
+int ssm_stack_bwd(const ssm_shape* shape, int n_layers, const ssm_stack_params* params,
+                  const void* u, const uint8_t* done, const void* gout /*[B,T,H] io*/,
+                  void* ws, size_t ws_bytes, void* du /*[B,T,H] io*/,
+                  const ssm_stack_grads* grads, void* stream);
+
 /* ---- measurement helpers (no counterpart in the paper; they never change results) ----
  * ssm_launch_count: kernels this library has launched in this process so far.
  * ssm_profile_begin / ssm_profile_end: between the two, every internal stage of the

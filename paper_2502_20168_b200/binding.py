@@ -26,6 +26,7 @@ EXPORTS = (
     "ssm_scan_workspace_bytes", "ssm_scan_fwd", "ssm_scan_bwd",
     "ssm_layer_workspace_bytes", "ssm_layer_fwd", "ssm_layer_bwd",
     "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static",
+    "ssm_stack_workspace_bytes", "ssm_stack_fwd", "ssm_stack_bwd",
 )
 SSM_ERR_TOO_LARGE = -8
 SSM_STATIC_SCRATCH_BYTES = 8 << 20
@@ -34,6 +35,14 @@ SSM_STATIC_SCRATCH_BYTES = 8 << 20
 class ssm_shape(Structure):
     _fields_ = [("B", c_int32), ("T", c_int32), ("H", c_int32), ("P", c_int32),
                 ("io_dtype", c_int32), ("reserved", c_int32)]
+
+
+class ssm_stack_params(Structure):
+    _fields_ = [(n, c_void_p) for n in ("Lambda", "Delta", "Bc", "Cc", "D", "ln_weight", "ln_bias")]
+
+
+class ssm_stack_grads(Structure):
+    _fields_ = [(n, c_void_p) for n in ("dLambda", "dDelta", "dB", "dC", "dD", "dln_weight", "dln_bias")]
 
 
 class SsmError(RuntimeError):
@@ -72,6 +81,13 @@ def _load() -> ctypes.CDLL:
     lib.ssm_layer_bwd.argtypes = [S] + [P] * 11 + [c_size_t] + [P] * 8
     lib.ssm_scan_bwd_static.restype = c_int
     lib.ssm_scan_bwd_static.argtypes = [S] + [P] * 10
+    lib.ssm_stack_workspace_bytes.restype = c_size_t
+    lib.ssm_stack_workspace_bytes.argtypes = [S, c_int]
+    lib.ssm_stack_fwd.restype = c_int
+    lib.ssm_stack_fwd.argtypes = [S, c_int, POINTER(ssm_stack_params), P, P, P, P, c_size_t, P]
+    lib.ssm_stack_bwd.restype = c_int
+    lib.ssm_stack_bwd.argtypes = [S, c_int, POINTER(ssm_stack_params), P, P, P, P, c_size_t, P,
+                                  POINTER(ssm_stack_grads), P]
     lib.ssm_launch_count.restype = ctypes.c_longlong
     lib.ssm_launch_count.argtypes = []
     lib.ssm_profile_begin.restype = c_int
@@ -179,6 +195,34 @@ def ssm_layer_bwd(shape, Lambda, Delta, Bc, Cc, D, u, done, x0, gy, gxT, ws, du,
                            _ptr(done), _ptr(x0), _ptr(gy), _ptr(gxT), _ptr(ws), _nbytes(ws), _ptr(du),
                            _ptr(dLambda), _ptr(dDelta), _ptr(dB), _ptr(dC), _ptr(dD), _ptr(dx0),
                            _stream(stream)), "ssm_layer_bwd")
+
+
+def _struct_array(cls, dicts):
+    """Host array of structs of device pointers, one per layer (dicts of name -> tensor)."""
+    arr = (cls * len(dicts))()
+    for i, d in enumerate(dicts):
+        for name, _ in cls._fields_:
+            setattr(arr[i], name, _ptr(d[name]).value)
+    return arr
+
+
+def ssm_stack_workspace_bytes(shape, n_layers: int) -> int:
+    return int(_lib.ssm_stack_workspace_bytes(byref(shape), int(n_layers)))
+
+
+def ssm_stack_fwd(shape, params, u, done, out, ws, stream=None) -> None:
+    """params: list (one per layer) of dicts Lambda, Delta, Bc, Cc, D, ln_weight, ln_bias of tensors."""
+    arr = _struct_array(ssm_stack_params, params)
+    _ok(_lib.ssm_stack_fwd(byref(shape), len(params), arr, _ptr(u), _ptr(done), _ptr(out), _ptr(ws), _nbytes(ws),
+                           _stream(stream)), "ssm_stack_fwd")
+
+
+def ssm_stack_bwd(shape, params, u, done, gout, ws, du, grads, stream=None) -> None:
+    """grads: list of dicts dLambda, dDelta, dB, dC, dD, dln_weight, dln_bias of output tensors."""
+    arr = _struct_array(ssm_stack_params, params)
+    garr = _struct_array(ssm_stack_grads, grads)
+    _ok(_lib.ssm_stack_bwd(byref(shape), len(params), arr, _ptr(u), _ptr(done), _ptr(gout), _ptr(ws), _nbytes(ws),
+                           _ptr(du), garr, _stream(stream)), "ssm_stack_bwd")
 
 
 def ssm_launch_count() -> int:

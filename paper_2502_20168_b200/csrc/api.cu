@@ -23,12 +23,12 @@ size_t take(size_t& off, size_t bytes) {
     return at;
 }
 
-LayerPlan plan_layer(const ssm_shape& s) {
+LayerPlan plan_layer(const ssm_shape& s, bool allow_tc = true) {
     LayerPlan p{};
     size_t off = 0;
     const size_t BT = (size_t)s.B * s.T, PH = (size_t)s.P * s.H;
     const int P2 = 2 * s.P;
-    p.tc = s.io_dtype == SSM_BF16 && tc_tn_supported((int)BT, P2, s.H, true) &&
+    p.tc = allow_tc && s.io_dtype == SSM_BF16 && tc_tn_supported((int)BT, P2, s.H, true) &&
            tc_tn_supported((int)BT, s.H, P2, false) && tc_nt_supported(s.H, P2);
     p.splits = p.tc ? tc_nt_splits((int)BT, s.H, P2) : gemm_nt_splits((int)BT);
     p.hdr = take(off, sizeof(WsHeader));
@@ -171,24 +171,13 @@ SSM_API size_t ssm_layer_workspace_bytes(const ssm_shape* shape) {
     return plan_layer(*shape).total;
 }
 
-SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
-                          const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
-                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, size_t ws_bytes, void* stream) {
-    if (int rc = check_shape(shape)) return rc;
-    if (!Lambda || !Delta || !Bc || !Cc || !D || !u || !y) return SSM_ERR_NULL;
-    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Cc) || misaligned(D) ||
-        misaligned(u) || misaligned(y) || misaligned(x0) || misaligned(xT))
-        return SSM_ERR_ALIGN;
-    const ssm_shape& s = *shape;
-    const LayerPlan p = plan_layer(s);
-    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
+// Launch sequence of one layer's forward pass.  `hdr` receives the status of bounded waits.
+static int layer_fwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
+                          const ssm_c64* Bc, const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
+                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr, cudaStream_t st) {
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T, P2 = 2 * s.P;
-    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
     int rc = SSM_OK;
-
-    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     {
         StageTimer tm("discretize_pack", st);
         launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
@@ -244,25 +233,33 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     return SSM_OK;
 }
 
-SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
+
+SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
                           const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
-                          const ssm_c64* x0, const void* gy, const ssm_c64* gxT, void* ws, size_t ws_bytes,
-                          void* du, ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
-                          ssm_c64* dx0, void* stream) {
+                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_shape(shape)) return rc;
-    if (!Lambda || !Delta || !Bc || !Cc || !D || !u || !gy || !du || !dLambda || !dDelta || !dB || !dC || !dD)
-        return SSM_ERR_NULL;
+    if (!Lambda || !Delta || !Bc || !Cc || !D || !u || !y) return SSM_ERR_NULL;
     if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Cc) || misaligned(D) ||
-        misaligned(u) || misaligned(gy) || misaligned(du) || misaligned(dLambda) || misaligned(dDelta) ||
-        misaligned(dB) || misaligned(dC) || misaligned(dD) || misaligned(x0) || misaligned(gxT) || misaligned(dx0))
+        misaligned(u) || misaligned(y) || misaligned(x0) || misaligned(xT))
         return SSM_ERR_ALIGN;
     const ssm_shape& s = *shape;
     const LayerPlan p = plan_layer(s);
     if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    return layer_fwd_impl(s, p, Lambda, Delta, Bc, Cc, D, u, done, x0, y, xT, ws, hdr, st);
+}
+
+// Launch sequence of one layer's backward pass.  du_add (io dtype, may be NULL) is added to du
+// before it is rounded (the residual branch of a stacked model).
+static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
+                          const ssm_c64* Bc, const float* D, const void* u, const uint8_t* done, const ssm_c64* x0,
+                          const void* gy, const ssm_c64* gxT, const void* du_add, void* ws, WsHeader* hdr, void* du,
+                          ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD, ssm_c64* dx0,
+                          cudaStream_t st) {
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T, P2 = 2 * s.P;
-    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
     float* part = at<float>(ws, p.part);
     const size_t plane = (size_t)BT * s.P * 4;   // bytes of one bf16 plane of a state tensor
     int rc = SSM_OK;
@@ -284,7 +281,7 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         }
         {   // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]
             StageTimer tm("gemm_du", st);
-            GemmTcTN g{at<void>(ws, p.gs), at<void>(ws, p.W3), BT, s.H, P2, false, false, du, D, gy, nullptr, hdr};
+            GemmTcTN g{at<void>(ws, p.gs), at<void>(ws, p.W3), BT, s.H, P2, false, false, du, D, gy, du_add, hdr};
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
         }
         {   // gBbar[p,h] = sum_m s[m,p] u[m,h]
@@ -317,7 +314,7 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         {
             StageTimer tm("gemm_du", st);
             GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.W3), false, P2, BT, s.H, P2, Epi::AddDiagIo,
-                      du, bf16, D, gy, nullptr};
+                      du, bf16, D, gy, du_add};
             launch_gemm_tn(g4, st);
         }
         {
@@ -338,6 +335,159 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
         launch_dot_columns(bf16, gy, u, BT, s.H, dD, at<float>(ws, p.dot), st);
         launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
                               at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);
+    }
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
+                          const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
+                          const ssm_c64* x0, const void* gy, const ssm_c64* gxT, void* ws, size_t ws_bytes,
+                          void* du, ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
+                          ssm_c64* dx0, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Lambda || !Delta || !Bc || !Cc || !D || !u || !gy || !du || !dLambda || !dDelta || !dB || !dC || !dD)
+        return SSM_ERR_NULL;
+    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Cc) || misaligned(D) ||
+        misaligned(u) || misaligned(gy) || misaligned(du) || misaligned(dLambda) || misaligned(dDelta) ||
+        misaligned(dB) || misaligned(dC) || misaligned(dD) || misaligned(x0) || misaligned(gxT) || misaligned(dx0))
+        return SSM_ERR_ALIGN;
+    const ssm_shape& s = *shape;
+    const LayerPlan p = plan_layer(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    return layer_bwd_impl(s, p, Lambda, Delta, Bc, D, u, done, x0, gy, gxT, nullptr, ws, hdr, du, dLambda, dDelta, dB,
+                          dC, dD, dx0, st);
+}
+
+// ---- stacked model -----------------------------------------------------------------------------
+namespace {
+
+// The layers of a stack run on the fp32 CUDA-core path: what is stored between and inside the
+// blocks is rounded to the I/O type, and a value that lands on the other side of a rounding
+// boundary than in an exact evaluation shifts the parameter-gradient sums by more than the
+// tolerance allows unless the arithmetic in front of every rounding is accurate to fp32 level.
+struct StackPlan {
+    size_t layer_ws;   // bytes of one layer workspace
+    size_t act;        // bytes of one [B,T,H] io tensor
+    size_t hdr, layers, acts, vs, stats, gzr, gv, g0, g1, tmp, total;
+};
+
+StackPlan plan_stack(const ssm_shape& s, int L) {
+    StackPlan p{};
+    size_t off = 0;
+    const size_t BT = (size_t)s.B * s.T;
+    p.layer_ws = align_up(plan_layer(s, false).total, 256);
+    p.act = align_up(BT * s.H * (s.io_dtype == SSM_BF16 ? 2 : 4), 256);
+    p.hdr = take(off, sizeof(WsHeader));
+    p.layers = take(off, p.layer_ws * L);
+    p.acts = take(off, p.act * (L > 1 ? L - 1 : 0));   // inputs of layers 1 .. L-1
+    p.vs = take(off, p.act * L);                       // SSM outputs
+    p.stats = take(off, align_up(BT * 4, 256) * 2 * L);   // mean and 1/std of every row, per layer
+    p.gzr = take(off, p.act);
+    p.gv = take(off, p.act);
+    p.g0 = take(off, p.act);
+    p.g1 = take(off, p.act);
+    p.tmp = take(off, stack_tmp_floats((int)BT, s.H) * 4);
+    p.total = off;
+    return p;
+}
+
+int check_stack_args(const ssm_shape* shape, int n_layers, const ssm_stack_params* params) {
+    if (int rc = check_shape(shape)) return rc;
+    if (n_layers < 1 || n_layers > 64) return SSM_ERR_SHAPE;
+    if (!params) return SSM_ERR_NULL;
+    for (int l = 0; l < n_layers; ++l) {
+        const ssm_stack_params& q = params[l];
+        if (!q.Lambda || !q.Delta || !q.Bc || !q.Cc || !q.D || !q.ln_weight || !q.ln_bias) return SSM_ERR_NULL;
+        if (misaligned(q.Lambda) || misaligned(q.Delta) || misaligned(q.Bc) || misaligned(q.Cc) || misaligned(q.D) ||
+            misaligned(q.ln_weight) || misaligned(q.ln_bias))
+            return SSM_ERR_ALIGN;
+    }
+    return SSM_OK;
+}
+
+}  // namespace
+
+SSM_API size_t ssm_stack_workspace_bytes(const ssm_shape* shape, int n_layers) {
+    if (check_shape(shape) != SSM_OK || n_layers < 1 || n_layers > 64) return 0;
+    return plan_stack(*shape, n_layers).total;
+}
+
+SSM_API int ssm_stack_fwd(const ssm_shape* shape, int n_layers, const ssm_stack_params* params, const void* u,
+                          const uint8_t* done, void* out, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_stack_args(shape, n_layers, params)) return rc;
+    if (!u || !out) return SSM_ERR_NULL;
+    if (misaligned(u) || misaligned(out)) return SSM_ERR_ALIGN;
+    const ssm_shape& s = *shape;
+    const StackPlan sp = plan_stack(s, n_layers);
+    if (int rc = check_ws(ws, ws_bytes, sp.total)) return rc;
+    const LayerPlan lp = plan_layer(s, false);
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf16 = s.io_dtype == SSM_BF16;
+    const int BT = s.B * s.T;
+    const size_t stat = align_up((size_t)BT * 4, 256);
+    WsHeader* hdr = at<WsHeader>(ws, sp.hdr);
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    const void* in = u;
+    for (int l = 0; l < n_layers; ++l) {
+        const ssm_stack_params& q = params[l];
+        void* lws = at<void>(ws, sp.layers + sp.layer_ws * l);
+        void* v = at<void>(ws, sp.vs + sp.act * l);
+        void* o = (l == n_layers - 1) ? out : at<void>(ws, sp.acts + sp.act * l);
+        if (int rc = layer_fwd_impl(s, lp, q.Lambda, q.Delta, q.Bc, q.Cc, q.D, in, done, nullptr, v, nullptr, lws, hdr, st))
+            return rc;
+        StageTimer tm("stack_gelu_ln_fwd", st);
+        launch_stack_fwd(bf16, BT, s.H, in, v, q.ln_weight, q.ln_bias, o, at<float>(ws, sp.stats + stat * (2 * l)),
+                         at<float>(ws, sp.stats + stat * (2 * l + 1)), st);
+        in = o;
+    }
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_stack_bwd(const ssm_shape* shape, int n_layers, const ssm_stack_params* params, const void* u,
+                          const uint8_t* done, const void* gout, void* ws, size_t ws_bytes, void* du,
+                          const ssm_stack_grads* grads, void* stream) {
+    if (int rc = check_stack_args(shape, n_layers, params)) return rc;
+    if (!u || !gout || !du || !grads) return SSM_ERR_NULL;
+    if (misaligned(u) || misaligned(gout) || misaligned(du)) return SSM_ERR_ALIGN;
+    for (int l = 0; l < n_layers; ++l) {
+        const ssm_stack_grads& g = grads[l];
+        if (!g.dLambda || !g.dDelta || !g.dB || !g.dC || !g.dD || !g.dln_weight || !g.dln_bias) return SSM_ERR_NULL;
+        if (misaligned(g.dLambda) || misaligned(g.dDelta) || misaligned(g.dB) || misaligned(g.dC) || misaligned(g.dD) ||
+            misaligned(g.dln_weight) || misaligned(g.dln_bias))
+            return SSM_ERR_ALIGN;
+    }
+    const ssm_shape& s = *shape;
+    const StackPlan sp = plan_stack(s, n_layers);
+    if (int rc = check_ws(ws, ws_bytes, sp.total)) return rc;
+    const LayerPlan lp = plan_layer(s, false);
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf16 = s.io_dtype == SSM_BF16;
+    const int BT = s.B * s.T;
+    const size_t stat = align_up((size_t)BT * 4, 256);
+    WsHeader* hdr = at<WsHeader>(ws, sp.hdr);
+    const void* g = gout;
+    for (int l = n_layers - 1; l >= 0; --l) {
+        const ssm_stack_params& q = params[l];
+        const ssm_stack_grads& gr = grads[l];
+        void* lws = at<void>(ws, sp.layers + sp.layer_ws * l);
+        const void* in = (l == 0) ? u : at<void>(ws, sp.acts + sp.act * (l - 1));
+        const void* v = at<void>(ws, sp.vs + sp.act * l);
+        void* gnext = (l == 0) ? du : at<void>(ws, (l & 1) ? sp.g1 : sp.g0);
+        {
+            StageTimer tm("stack_gelu_ln_bwd", st);
+            launch_stack_bwd(bf16, BT, s.H, g, in, v, q.ln_weight, at<float>(ws, sp.stats + stat * (2 * l)),
+                             at<float>(ws, sp.stats + stat * (2 * l + 1)), at<void>(ws, sp.gzr), at<void>(ws, sp.gv),
+                             gr.dln_weight, gr.dln_bias, at<float>(ws, sp.tmp), st);
+        }
+        if (int rc = layer_bwd_impl(s, lp, q.Lambda, q.Delta, q.Bc, q.D, in, done, nullptr, at<void>(ws, sp.gv), nullptr,
+                                    at<void>(ws, sp.gzr), lws, hdr, gnext, gr.dLambda, gr.dDelta, gr.dB, gr.dC, gr.dD,
+                                    nullptr, st))
+            return rc;
+        g = gnext;
     }
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;

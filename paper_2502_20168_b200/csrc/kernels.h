@@ -98,4 +98,13 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st);
 
+// stack.cu: out = LayerNorm(u + GELU(v)) * w + b per row of H features, and its backward
+// (gzr = round(LN'(g)), gv = round(gz * GELU'(v)), dw, db).  tmp: stack_tmp_floats(M, H) floats.
+size_t stack_tmp_floats(int M, int H);
+void launch_stack_fwd(bool bf16, int M, int H, const void* u, const void* v, const float* w, const float* b, void* out,
+                      float* mu, float* rstd, cudaStream_t st);
+void launch_stack_bwd(bool bf16, int M, int H, const void* g, const void* u, const void* v, const float* w,
+                      const float* mu, const float* rstd, void* gzr, void* gv, float* dw, float* db, float* tmp,
+                      cudaStream_t st);
+
 }  // namespace ssm

@@ -85,3 +85,56 @@ def run_layer(d: dict, io_dtype: str, with_x0=False, with_gxT=False) -> dict:
     sb.ssm_check(buf.ws)
     torch.cuda.synchronize()
     return buf.results()
+
+
+class StackBuffers:
+    """Device copies of a stacked model's inputs plus preallocated outputs and workspace."""
+
+    def __init__(self, d: dict, io_dtype: str, device="cuda"):
+        io = _IO[io_dtype]
+        B, T, H = d["u"].shape
+        P = d["params"][0]["Lambda"].shape[0]
+        L = len(d["params"])
+        self.shape = sb.make_shape(B, T, H, P, io_dtype)
+        self.params, self.grads = [], []
+        c64 = dict(dtype=torch.complex64, device=device)
+        f32 = dict(dtype=torch.float32, device=device)
+        for l in range(L):
+            q = d["params"][l]
+            self.params.append({
+                "Lambda": to_dev(q["Lambda"].astype(np.complex64), device=device),
+                "Delta": to_dev(q["Delta"].astype(np.float32), device=device),
+                "Bc": to_dev(q["Bc"].astype(np.complex64), device=device),
+                "Cc": to_dev(q["Cc"].astype(np.complex64), device=device),
+                "D": to_dev(q["D"].astype(np.float32), device=device),
+                "ln_weight": to_dev(np.asarray(d["ln_weight"][l], np.float32), device=device),
+                "ln_bias": to_dev(np.asarray(d["ln_bias"][l], np.float32), device=device)})
+            self.grads.append({
+                "dLambda": torch.empty(P, **c64), "dDelta": torch.empty(P, **f32),
+                "dB": torch.empty((P, H), **c64), "dC": torch.empty((H, P), **c64), "dD": torch.empty(H, **f32),
+                "dln_weight": torch.empty(H, **f32), "dln_bias": torch.empty(H, **f32)})
+        self.u = to_dev(d["u"], io, device)
+        self.gout = to_dev(d["gy"], io, device)
+        self.done = to_dev(d.get("done"), torch.uint8, device)
+        self.out = torch.empty((B, T, H), dtype=io, device=device)
+        self.du = torch.empty((B, T, H), dtype=io, device=device)
+        self.ws = sb.alloc_workspace(sb.ssm_stack_workspace_bytes(self.shape, L), device)
+
+    def forward(self, stream=None):
+        sb.ssm_stack_fwd(self.shape, self.params, self.u, self.done, self.out, self.ws, stream)
+
+    def backward(self, stream=None):
+        sb.ssm_stack_bwd(self.shape, self.params, self.u, self.done, self.gout, self.ws, self.du, self.grads, stream)
+
+    def results(self) -> dict:
+        return {"out": to_np(self.out), "du": to_np(self.du),
+                "grads": [{k: to_np(v) for k, v in g.items()} for g in self.grads]}
+
+
+def run_stack(d: dict, io_dtype: str) -> dict:
+    buf = StackBuffers(d, io_dtype)
+    buf.forward()
+    buf.backward()
+    sb.ssm_check(buf.ws)
+    torch.cuda.synchronize()
+    return buf.results()
