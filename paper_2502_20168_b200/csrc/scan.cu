@@ -28,7 +28,6 @@
 namespace ssm {
 
 constexpr int kUnrollFwd = 16;    // time steps whose loads are in flight per thread (seq kernels)
-constexpr int kUnrollBwd = 8;
 constexpr int kSeqThreads = 64;   // small blocks spread a few hundred thousand threads evenly over the SMs
 constexpr int kScanThreads = 128;
 constexpr int kFwdChunk = 32;     // steps per chunk, forward
@@ -146,104 +145,6 @@ scan_fwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const
     if (xT) xT[(size_t)b * P2 + pp] = c2_pack(s);
 }
 
-// Undecoded state loads, so that a whole batch of them can be in flight while the previous
-// batch is being processed.
-template <typename ST> struct RawState;
-template <> struct RawState<float4> {
-    float4 v;
-    __device__ __forceinline__ void load(const float4* p, size_t) { v = __ldcs(p); }
-    __device__ __forceinline__ C2 get() const { return c2_from(v); }
-};
-template <> struct RawState<uint2> {
-    uint2 hi, lo;
-    __device__ __forceinline__ void load(const uint2* p, size_t plane) {
-        hi = __ldcs(p);
-        lo = __ldcs(p + plane);
-    }
-    __device__ __forceinline__ C2 get() const {
-        const C2 h = unpack_bf16x4(hi), l = unpack_bf16x4(lo);
-        return C2{cadd(h.a, l.a), cadd(h.b, l.b)};
-    }
-};
-
-// s_t = gx_t + c_t,  c_{t-1} = keep_t conj(Abar) s_t  (c_{T-1} = gxT);
-// gAbar partial = sum_t keep_t s_t conj(x_{t-1}).  gBu may alias gx.
-// Two register batches of kUnrollBwd steps alternate: the loads of one are issued before the
-// other is processed.
-template <typename XT, typename ST>
-__global__ void __launch_bounds__(kSeqThreads)
-scan_bwd_seq_kernel(int B, int T, int P2, const float4* __restrict__ Abar, const float4* __restrict__ Alo,
-                    const uint8_t* __restrict__ done,
-                    const float4* __restrict__ x0, const XT* __restrict__ x, const float4* gx,
-                    const float4* __restrict__ gxT, ST* gBu, float4* __restrict__ gA_part,
-                    float4* __restrict__ gx0) {
-    const int idx = blockIdx.x * kSeqThreads + threadIdx.x;
-    if (idx >= B * P2) return;
-    const int b = idx / P2, pp = idx - b * P2;
-    const size_t plane = (size_t)B * T * P2;
-    const C2 a = c2_from(Abar[pp]);
-    const float2 ac0 = cconj(a.a), ac1 = cconj(a.b);
-    const C2 al = Alo ? c2_from(Alo[pp]) : c2_zero();
-    const float2 al0 = cconj(al.a), al1 = cconj(al.b);
-    const float2 zero2 = make_float2(0.f, 0.f);
-    C2 c = gxT ? c2_from(gxT[(size_t)b * P2 + pp]) : c2_zero();
-    C2 g = c2_zero();
-    const float4* gsrc = gx + (size_t)b * T * P2 + pp;
-    const XT* xsrc = x + (size_t)b * T * P2 + pp;
-    ST* dst = gBu + (size_t)b * T * P2 + pp;
-    const uint8_t* dn = done ? done + (size_t)b * T : nullptr;
-    const C2 xinit = x0 ? c2_from(x0[(size_t)b * P2 + pp]) : c2_zero();
-
-    struct Batch {
-        float4 v[kUnrollBwd];
-        RawState<XT> xp[kUnrollBwd];
-        uint32_t flags;
-    };
-    // steps t0, t0-1, ..., t0-kUnrollBwd+1 (those that exist)
-    auto fetch = [&](int t0, Batch& q) {
-        q.flags = 0u;
-#pragma unroll
-        for (int i = 0; i < kUnrollBwd; ++i) {
-            const int t = t0 - i;
-            if (t >= 0) {
-                q.v[i] = __ldcs(gsrc + (size_t)t * P2);
-                if (t > 0) q.xp[i].load(xsrc + (size_t)(t - 1) * P2, plane);
-                if (dn && dn[t] != 0) q.flags |= 1u << i;
-            }
-        }
-    };
-    auto process = [&](int t0, const Batch& q) {
-#pragma unroll
-        for (int i = 0; i < kUnrollBwd; ++i) {
-            const int t = t0 - i;
-            if (t >= 0) {
-                const C2 vi = c2_from(q.v[i]);
-                const C2 s{cadd(vi.a, c.a), cadd(vi.b, c.b)};
-                StateIO<ST>::store(dst + (size_t)t * P2, s, plane);
-                if ((q.flags >> i) & 1u) {
-                    c = c2_zero();
-                } else {
-                    const C2 xprev = t > 0 ? q.xp[i].get() : xinit;
-                    g.a = cfma(s.a, cconj(xprev.a), g.a);
-                    g.b = cfma(s.b, cconj(xprev.b), g.b);
-                    c.a = cfma2(ac0, al0, s.a, zero2);
-                    c.b = cfma2(ac1, al1, s.b, zero2);
-                }
-            }
-        }
-    };
-    Batch q0, q1;
-    fetch(T - 1, q0);
-    for (int t0 = T - 1; t0 >= 0; t0 -= 2 * kUnrollBwd) {
-        fetch(t0 - kUnrollBwd, q1);
-        process(t0, q0);
-        fetch(t0 - 2 * kUnrollBwd, q0);
-        process(t0 - kUnrollBwd, q1);
-    }
-    gA_part[(size_t)b * P2 + pp] = c2_pack(g);
-    if (gx0) gx0[(size_t)b * P2 + pp] = c2_pack(c);
-}
-
 // =============================================================================================
 // Chunked, with decoupled look-back
 // =============================================================================================
@@ -307,6 +208,103 @@ template <> struct Raw1<uint32_t> {
         p[plane] = *reinterpret_cast<const uint32_t*>(&l);
     }
 };
+
+// Whole-sequence backward scan, ONE state per thread (8-byte accesses): the backward step carries
+// about twice the instructions of the forward one, and with two states per thread the SMs ran
+// short of warps to hide their latency.
+//   s_t = gx_t + c_t,  c_{t-1} = keep_t conj(Abar) s_t  (c_{T-1} = gxT);
+//   gAbar partial = sum_t keep_t s_t conj(x_{t-1}).  gBu may alias gx.
+// Two register batches of kUnroll1 steps alternate (the loads of one are issued before the other
+// is processed); pointers advance by a constant and a guard-free main loop handles full batches.
+constexpr int kUnroll1 = 8;
+template <typename XS>
+__global__ void __launch_bounds__(kSeqThreads)
+scan_bwd_seq1_kernel(int B, int T, int P, const float2* __restrict__ Abar, const float2* __restrict__ Alo,
+                     const uint8_t* __restrict__ done, const float2* __restrict__ x0, const XS* __restrict__ x,
+                     const float2* gx, const float2* __restrict__ gxT, XS* gBu, float2* __restrict__ gA_part,
+                     float2* __restrict__ gx0) {
+    const int idx = blockIdx.x * kSeqThreads + threadIdx.x;
+    if (idx >= B * P) return;
+    const int b = idx / P, p = idx - b * P;
+    const size_t plane = (size_t)B * T * P;
+    const float2 ac = cconj(Abar[p]);
+    const float2 acl = Alo ? cconj(Alo[p]) : make_float2(0.f, 0.f);
+    const float2 zero2 = make_float2(0.f, 0.f);
+    float2 c = gxT ? gxT[(size_t)b * P + p] : zero2;
+    float2 g = zero2;
+    const uint8_t* dn = done ? done + (size_t)b * T : nullptr;
+    const float2 xinit = x0 ? x0[(size_t)b * P + p] : zero2;
+    // pointers at step t = T-1; every step back moves them by -P
+    const float2* gp = gx + ((size_t)b * T + (T - 1)) * P + p;
+    const XS* xp = x + ((size_t)b * T + (T - 1)) * P + p - P;   // x_{t-1}
+    XS* sp = gBu + ((size_t)b * T + (T - 1)) * P + p;
+
+    struct Batch {
+        float2 v[kUnroll1];
+        Raw1<XS> xr[kUnroll1];
+        uint32_t flags;
+    };
+    // steps t0 .. t0-kUnroll1+1, all known to exist and t0-kUnroll1+1 >= 1 (so x_{t-1} exists)
+    auto fetch_full = [&](int t0, Batch& q) {
+        q.flags = 0u;
+#pragma unroll
+        for (int i = 0; i < kUnroll1; ++i) {
+            q.v[i] = __ldcs(gp - (ptrdiff_t)i * P);
+            q.xr[i].load(xp - (ptrdiff_t)i * P, plane);
+            if (dn && dn[t0 - i] != 0) q.flags |= 1u << i;
+        }
+        gp -= (ptrdiff_t)kUnroll1 * P;
+        xp -= (ptrdiff_t)kUnroll1 * P;
+    };
+    auto step = [&](float2 v, float2 xprev, bool flagged, XS* dst) {
+        const float2 s = cadd(v, c);
+        Raw1<XS>::store(dst, s, plane);
+        if (flagged) {
+            c = zero2;
+        } else {
+            g = cfma(s, cconj(xprev), g);
+            c = cfma2(ac, acl, s, zero2);
+        }
+    };
+    auto process_full = [&](const Batch& q) {
+#pragma unroll
+        for (int i = 0; i < kUnroll1; ++i) step(q.v[i], q.xr[i].get(), (q.flags >> i) & 1u, sp - (ptrdiff_t)i * P);
+        sp -= (ptrdiff_t)kUnroll1 * P;
+    };
+    // Full batches cover steps T-1 .. r where every step has t >= 1; the rest goes one by one.
+    int t = T - 1;
+    const int nfull = (T - 1) / kUnroll1;     // batches whose lowest step is >= 1
+    if (nfull > 0) {
+        Batch q0, q1;
+        fetch_full(t, q0);
+        int left = nfull - 1;
+        while (true) {
+            if (left > 0) fetch_full(t - kUnroll1, q1);
+            process_full(q0);
+            t -= kUnroll1;
+            if (left-- == 0) break;
+            if (left > 0) fetch_full(t - kUnroll1, q0);
+            process_full(q1);
+            t -= kUnroll1;
+            if (left-- == 0) break;
+        }
+    }
+    for (; t >= 0; --t) {
+        const float2 v = __ldcs(gp);
+        float2 xprev = xinit;
+        if (t > 0) {
+            Raw1<XS> r;
+            r.load(xp, plane);
+            xprev = r.get();
+        }
+        step(v, xprev, dn && dn[t] != 0, sp);
+        gp -= P;
+        xp -= P;
+        sp -= P;
+    }
+    gA_part[(size_t)b * P + p] = g;
+    if (gx0) gx0[(size_t)b * P + p] = c;
+}
 
 __device__ __forceinline__ void publish(const ChunkArgs& k, int item, float2 v, uint32_t state) {
     uint4 r;
@@ -687,7 +685,6 @@ int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
 int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done, const float2* x0,
                     const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
                     float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st) {
-    const int P2 = P / 2;
     const ScanPlan s = plan_scan(B, T, P, kBwdChunk);
     char* base = (char*)scratch;
     float* part = reinterpret_cast<float*>(base + s.off_part);
@@ -695,16 +692,14 @@ int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
     if (x_bf16 != s_bf16) return SSM_ERR_DTYPE;
     int rows = B;
     if (!s.chunked) {
-        const int blocks = (int)(((size_t)B * P2 + kSeqThreads - 1) / kSeqThreads);
         count_launch();
+        const int blocks1 = (int)(((size_t)B * P + kSeqThreads - 1) / kSeqThreads);
         if (x_bf16)
-            scan_bwd_seq_kernel<uint2, uint2><<<blocks, kSeqThreads, 0, st>>>(
-                B, T, P2, (const float4*)Abar, (const float4*)Alo, done, (const float4*)x0, (const uint2*)x, (const float4*)gx,
-                (const float4*)gxT, (uint2*)gBu, (float4*)part, (float4*)gx0);
+            scan_bwd_seq1_kernel<uint32_t><<<blocks1, kSeqThreads, 0, st>>>(
+                B, T, P, Abar, Alo, done, x0, (const uint32_t*)x, gx, gxT, (uint32_t*)gBu, (float2*)part, gx0);
         else
-            scan_bwd_seq_kernel<float4, float4><<<blocks, kSeqThreads, 0, st>>>(
-                B, T, P2, (const float4*)Abar, (const float4*)Alo, done, (const float4*)x0, (const float4*)x, (const float4*)gx,
-                (const float4*)gxT, (float4*)gBu, (float4*)part, (float4*)gx0);
+            scan_bwd_seq1_kernel<float2><<<blocks1, kSeqThreads, 0, st>>>(
+                B, T, P, Abar, Alo, done, x0, (const float2*)x, gx, gxT, (float2*)gBu, (float2*)part, gx0);
     } else {
         if (cudaMemsetAsync(scratch, 0, s.zero_bytes, st) != cudaSuccess) return SSM_ERR_CUDA;
         const ChunkArgs k = chunk_args(s, B, T, P, Abar, Alo, done, hdr, base);
