@@ -82,6 +82,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
         : "memory");
 }
+// Shared -> global tile store by the TMA unit (bulk async group of the issuing thread).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Waits until the TMA unit has read the shared-memory source of every store issued so far.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -235,7 +246,8 @@ struct TnParams {
 // halves of the same 128 output columns.
 template <int kEpi, bool kSplitW>
 __global__ void __launch_bounds__(kTnThreads, 1)
-gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, TnParams p) {
+gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                  const __grid_constant__ CUtensorMap tmOut, TnParams p) {
     extern __shared__ uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, kTnStages, kStagingBytes, kMaxDiag * 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -341,7 +353,11 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 tmem_ld32(t_row + (uint32_t)c, r);
                 if (kSplitW) tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
                 tmem_ld_wait();
-                // registers -> staging (16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7))
+                // registers -> staging (16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7): the
+                // 128-byte swizzle, so that the TMA unit can store the buffer as a 32 x 32 fp32 box)
+                if (kEpi == 0) {
+                    if (lane == 0) tma_store_wait_read();
+                }
                 __syncwarp();
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -358,15 +374,10 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 __syncwarp();
                 // staging -> global with full-line accesses
                 if (kEpi == 0) {
-                    // each instruction covers 4 rows x 128 bytes: lane -> (row i*4 + lane/8, chunk lane%8)
-                    float* out = reinterpret_cast<float*>(p.out);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int rr = i * 4 + (lane >> 3), ch = lane & 7;
-                        const float4 v = stg[rr * 8 + (ch ^ (rr & 7))];
-                        if (row0 + rr < p.M)
-                            *reinterpret_cast<float4*>(out + (size_t)(row0 + rr) * p.ldo + n_out0 + c + ch * 4) = v;
-                    }
+                    // one TMA store of the 32-row x 128-byte box; rows past M are clipped by the unit
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.M) tma_store_2d(&tmOut, smem_u32(stg), n_out0 + c, row0);
                 } else {
                     // each instruction covers 8 rows x 64 bytes of bf16: lane -> (row i*8 + lane/4, 8 columns)
                     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
@@ -413,6 +424,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             mbar_arrive(s.tmem_empty[acc]);
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
         }
+        if (kEpi == 0 && lane == 0) tma_store_wait_all();
     }
     epilogue_exit(s, warp, tmem_base, p.hdr);
 }
@@ -553,14 +565,14 @@ static PFN_cuTensorMapEncodeTiled encode_fn() {
 
 // Row-major bf16 matrix [rows, cols] (cols contiguous), boxes of box_cols x box_rows, 128-byte swizzle.
 static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_cols,
-                     uint32_t box_rows) {
+                     uint32_t box_rows, bool f32 = false) {
     PFN_cuTensorMapEncodeTiled fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
+    cuuint64_t strides[1] = {cols * (f32 ? 4u : 2u)};
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -592,9 +604,14 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     using namespace tc;
     const int out_cols = g.split_w ? BN / 2 : BN;
     const int n_tiles = g.N_out / out_cols;
-    CUtensorMap ma, mw;
+    CUtensorMap ma, mw, mo;
     if (!make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, BK, BM)) return SSM_ERR_CUDA;
     if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN)) return SSM_ERR_CUDA;
+    if (g.store_f32) {   // fp32 result, stored by the TMA unit in boxes of 32 rows x 32 columns
+        if (!make_map(&mo, g.out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, true)) return SSM_ERR_CUDA;
+    } else {
+        mo = ma;         // unused by the bf16 epilogue
+    }
     TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.out, g.diag, (const __nv_bfloat16*)g.skip,
                (const __nv_bfloat16*)g.add, g.hdr};
     const int m_tiles = (g.M + BM - 1) / BM;
@@ -604,14 +621,14 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     if (g.store_f32) {
         if (g.split_w) {
             ok = set_smem(gemm_tc_tn_kernel<0, true>, kTnSmemBytes);
-            gemm_tc_tn_kernel<0, true><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, p);
+            gemm_tc_tn_kernel<0, true><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, mo, p);
         } else {
             ok = set_smem(gemm_tc_tn_kernel<0, false>, kTnSmemBytes);
-            gemm_tc_tn_kernel<0, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, p);
+            gemm_tc_tn_kernel<0, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, mo, p);
         }
     } else {
         ok = set_smem(gemm_tc_tn_kernel<1, false>, kTnSmemBytes);
-        gemm_tc_tn_kernel<1, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, p);
+        gemm_tc_tn_kernel<1, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, mo, p);
     }
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
