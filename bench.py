@@ -46,6 +46,22 @@ STAGE_MODEL = {
 }
 
 
+# DRAM bytes per launch seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum, summaries under
+# profiles/) on c4_sweep_T1024_bf16, per timestep (B*T = 262144 rows).  They hold for H = 512,
+# P = 256, bf16 I/O, traffic growing in proportion to B*T; an entry is None once its kernel has
+# changed since the counters were taken.
+NCU_TRAFFIC_PER_TIMESTEP = {
+    "scan_fwd": 1016.9e6 / 262144,
+    "scan_bwd": 1557.3e6 / 262144,
+    "gemm_Bu": None,
+    "gemm_gx": None,
+    "gemm_y": 781.7e6 / 262144,
+    "gemm_du": 781.7e6 / 262144,
+    "gemm_gBbar": 811.8e6 / 262144,
+    "gemm_gC": 811.8e6 / 262144,
+}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -109,6 +125,10 @@ def oracle_sample_run(d, n_seq):
     done = None if d["done"] is None else d["done"][:n_seq]
     u, gy = d["u"][:n_seq], d["gy"][:n_seq]
     t0 = time.perf_counter()
+    if "params" in d:      # stacked model
+        _, cache = O.stack_fwd(d["params"], d["ln_weight"], d["ln_bias"], u, done, round_io=I.round_to_bf16)
+        O.stack_bwd(d["params"], d["ln_weight"], d["ln_bias"], cache, done, gy, round_io=I.round_to_bf16)
+        return time.perf_counter() - t0
     O.ssm_layer_fwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], u, done, None)
     O.ssm_layer_bwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], u, done, None, gy)
     return time.perf_counter() - t0
@@ -198,11 +218,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     w = I.WORKLOADS[args.workload]
-    if w.n_layers != 1:
-        raise SystemExit("bench.py times single-layer workloads")
     wr = I.small_variant(w, seed=w.seed + 1000 * rank)
     d = I.draw_layer(wr)
-    buf = harness.LayerBuffers(d, w.io_dtype)
+    stacked = w.n_layers > 1
+    buf = harness.StackBuffers(d, w.io_dtype) if stacked else harness.LayerBuffers(d, w.io_dtype)
     stream = torch.cuda.current_stream()
 
     def step():
@@ -237,10 +256,11 @@ def main():
     sb.ssm_check(buf.ws)
 
     # ---- end to end: pinned host inputs in, results out, every step ----
-    host_in = {k: getattr(buf, k).cpu().pin_memory() for k in ("u", "gy")}
+    in_names = ("u", "gout") if stacked else ("u", "gy")
+    host_in = {k: getattr(buf, k).cpu().pin_memory() for k in in_names}
     if buf.done is not None:
         host_in["done"] = buf.done.cpu().pin_memory()
-    out_names = ("y", "du", "dLambda", "dDelta", "dB", "dC", "dD")
+    out_names = ("out", "du") if stacked else ("y", "du", "dLambda", "dDelta", "dB", "dC", "dD")
     host_out = {k: torch.empty_like(getattr(buf, k), device="cpu").pin_memory() for k in out_names}
     h2d = sum(t.numel() * t.element_size() for t in host_in.values())
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
@@ -278,6 +298,8 @@ def main():
         n_launch, top_ms = stages[top]
         per_launch_s = top_ms * 1e-3 / n_launch
         alg = work(w.H, w.P, s_io) * w.timesteps
+        traffic = NCU_TRAFFIC_PER_TIMESTEP.get(top) if (w.H, w.P, w.io_dtype, stacked) == (512, 256, "bf16", False) else None
+        traffic = None if traffic is None else traffic * w.timesteps
         if bound == "hbm":
             achieved, peak, runit = alg / per_launch_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"
         else:
@@ -290,14 +312,15 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
-                       "p_done": w.p_done, "l2": "inputs larger than L2 (no flush)"
+                       "p_done": w.p_done, "n_layers": w.n_layers, "l2": "inputs larger than L2 (no flush)"
                        if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}"},
             "e2e": {"value": total_ts * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
             "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
-                         "frac": achieved / peak, "traffic": None, "peak_source": peak_kind,
+                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
+                         "algorithmic_per_launch": alg, "launches_per_step": n_launch / args.steps,
                          "ms_per_launch": per_launch_s * 1e3},
             "stage_ms_per_step": {k: round(v[1] / args.steps, 4) for k, v in stages.items()},
             "stage_share": stage_share,

@@ -1,0 +1,65 @@
+"""Host-side logic of the N > 1 path on CPU (gloo, world size 2): the batch is sharded over the
+ranks with no data-path collective, each rank's shard gives exactly the rows of the full
+result (sequences are independent), the parameter gradients add up across ranks, and the
+step time reported is the maximum over ranks."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from oracle import ssm_oracle as O
+from paper_2502_20168_b200 import inputs as I
+
+W = I.Workload("mp", B=5, T=12, H=8, P=8, p_done=0.2, seed=3)
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_main(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    d = I.draw_layer(W)
+    lo, hi = I.shard_batch(W.B, rank, world)
+    args = (d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"])
+    y, _, _ = O.ssm_layer_fwd(*args, d["u"][lo:hi], d["done"][lo:hi], None)
+    g = O.ssm_layer_bwd(*args, d["u"][lo:hi], d["done"][lo:hi], None, d["gy"][lo:hi])
+    dC = torch.from_numpy(np.stack([g["dC"].real, g["dC"].imag]))
+    dist.all_reduce(dC)                                    # what a data-parallel trainer would add
+    t = torch.tensor([1.0 + rank], dtype=torch.float64)    # this rank's step time
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    out.put((rank, lo, hi, y, dC.numpy(), float(t)))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_batch_sharding_over_two_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = [q.get(timeout=120) for _ in procs]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    d = I.draw_layer(W)
+    args = (d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"])
+    y, _, _ = O.ssm_layer_fwd(*args, d["u"], d["done"], None)
+    g = O.ssm_layer_bwd(*args, d["u"], d["done"], None, d["gy"])
+    covered = np.zeros(W.B, bool)
+    for rank, lo, hi, yr, dC, t in got:
+        assert np.allclose(yr, y[lo:hi], atol=1e-12)
+        assert not covered[lo:hi].any()
+        covered[lo:hi] = True
+        assert np.allclose(dC[0] + 1j * dC[1], g["dC"], atol=1e-10)
+        assert t == 2.0
+    assert covered.all()
