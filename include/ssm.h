@@ -29,7 +29,7 @@
  *  - Gradient convention for complex values under a real loss L:
  *    g_z = dL/dRe(z) + i dL/dIm(z).  Gradient outputs are overwritten, not accumulated.
  *  - Return value: SSM_OK (0) or a negative SSM_ERR_* code.  Nothing throws, aborts or
- *    traps.  Device-side waits (the scan's inter-chunk carry) are bounded; if one gives
+ *    traps.  Device-side waits (shared-memory barriers of the pipelines) are bounded; if one gives
  *    up it records SSM_ERR_TIMEOUT in the workspace header, which ssm_check reads back.
  *  - Workspaces: the *_workspace_bytes functions give the size for a shape; the caller
  *    passes a 256-byte aligned device buffer of at least that size.  A layer workspace
@@ -93,8 +93,9 @@ int ssm_discretize_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const floa
 
 /* ---- the scan: Sec. III-B Eq. "scan".."full_scan"; resets Sec. IV-A ---------------
  * x[b,t,p] = (done[b,t] ? 0 : Abar[p] x[b,t-1,p]) + Bu[b,t,p],  x[b,-1,:] = x0[b,:] or 0.
- * Long sequences are cut into chunks scanned concurrently; the carry between chunks
- * uses the operator's associativity (decoupled look-back).  done, x0, xT may be NULL.
+ * A sequence is scanned tile by tile; inside a tile groups of threads scan stretches of
+ * rows concurrently and are joined with the operator's associativity, so the result does
+ * not depend on scheduling.  done, x0, xT may be NULL.
  * x may alias Bu (in-place).  Uses shape->B, T, P. */
 size_t ssm_scan_workspace_bytes(const ssm_shape* shape);
 int ssm_scan_fwd(const ssm_shape* shape, const ssm_c64* Abar /*[P]*/,

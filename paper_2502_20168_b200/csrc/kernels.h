@@ -16,7 +16,7 @@ void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const flo
                           void* Cp, void* Cq, cudaStream_t st);
 
 // scan.cu
-// Scratch the scans need for a [B,T,P] problem: look-back records and the partial sums of gAbar.
+// Scratch the scans need for a [B,T,P] problem: a work counter and the partial sums of gAbar.
 size_t scan_scratch_bytes(int B, int T, int P);
 // Alo (may be NULL): low part of Abar, so that Abar + Alo carries the multiplier to ~48 bits.
 int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu, const uint8_t* done,
@@ -26,6 +26,17 @@ int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
 int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done, const float2* x0,
                     const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
                     float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st);
+
+// scan_stream.cu: the scans as TMA-fed streaming kernels (a CTA walks whole sequences; all
+// parallelism over time is inside the CTA).  `ticket`: one int of scratch.  The backward pass
+// leaves B rows of P partial gAbar sums in `part`.
+bool scan_stream_supported(int B, int T, int P);
+int launch_scan_fwd_stream(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu,
+                           const uint8_t* done, const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr,
+                           int* ticket, cudaStream_t st);
+int launch_scan_bwd_stream(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done,
+                           const float2* x0, const void* x, bool x_bf16, const float2* gx, const float2* gxT,
+                           void* gBu, float2* gx0, float2* part, WsHeader* hdr, int* ticket, cudaStream_t st);
 
 // reduce.cu
 // out[c] = sum_r in[r, c]; `tmp` must hold colsum_tmp_floats(R, C) floats.  Deterministic.

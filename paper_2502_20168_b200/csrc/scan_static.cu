@@ -54,8 +54,8 @@ SSM_API int ssm_scan_bwd_static(const ssm_shape* shape, const ssm_c64* Abar, con
     void* base = nullptr;
     if (int rc = static_scratch_for_current_device(&base)) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    // The array keeps whatever the previous call left; the header (status word, chunk
-    // ticket) is the part that has to start at zero.
+    // The array keeps whatever the previous call left; the header (status word) is the part
+    // that has to start at zero (the scan zeroes its own work counter).
     if (cudaMemsetAsync(base, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     int rc = launch_scan_bwd(shape->B, shape->T, shape->P, (const float2*)Abar, nullptr, done, (const float2*)x0,
                              (const float2*)x, false, (const float2*)gx, (const float2*)gxT, (float2*)gBu, false,

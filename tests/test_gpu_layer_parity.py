@@ -62,7 +62,7 @@ def test_every_step_flagged_and_no_flags(io):
 
 
 def test_long_sequence_small_batch_fp32():
-    # long enough that the sequence is cut into many chunks with carries in between
+    # long enough that a sequence is many tiles, with the state carried from tile to tile
     w = I.Workload("long", B=2, T=2500, H=16, P=24, io_dtype="f32", p_done=0.003, seed=77)
     run(w, with_x0=True, with_gxT=True)
 
@@ -70,7 +70,7 @@ def test_long_sequence_small_batch_fp32():
 def test_forward_backward_twice_is_bitwise_repeatable_and_workspace_reusable():
     import torch
     from paper_2502_20168_b200 import harness
-    # One thread per sequence (large B*P): every sum has a fixed order, results repeat bit for bit.
+    # Every sum has a fixed order: results repeat bit for bit.
     d = I.draw_layer(I.Workload("rep", B=160, T=24, H=64, P=256, io_dtype="f32", p_done=0.05, seed=9))
     buf = harness.LayerBuffers(d, "f32")
     buf.forward(); buf.backward()
@@ -80,8 +80,7 @@ def test_forward_backward_twice_is_bitwise_repeatable_and_workspace_reusable():
     second = buf.results()
     for k in ("y", "du", "dB", "dC", "dLambda", "dDelta", "dD"):
         assert np.array_equal(first[k], second[k]), k
-    # Chunked scan (few sequences): the carry into a chunk is assembled from whichever records its
-    # predecessors have published so far, so the rounding of that one value can differ between runs.
+    # Few sequences, narrow tiles: the order of every sum is still fixed by the shape alone.
     d = I.draw_layer(I.C1)
     buf = harness.LayerBuffers(d, "f32")
     buf.forward(); buf.backward()
@@ -90,4 +89,4 @@ def test_forward_backward_twice_is_bitwise_repeatable_and_workspace_reusable():
     torch.cuda.synchronize()
     second = buf.results()
     for k in ("y", "du", "dB", "dC", "dLambda", "dDelta", "dD"):
-        assert np.max(np.abs(first[k] - second[k]) / (1.0 + np.abs(first[k]))) < 1e-4, k
+        assert np.array_equal(first[k], second[k]), k

@@ -1,6 +1,7 @@
 """Stand-alone entry points (ssm_discretize, ssm_discretize_bwd, ssm_scan_fwd, ssm_scan_bwd)
-against the oracle, through the C ABI: both scan strategies (one thread per sequence; chunks
-with look-back), in place and out of place, error paths."""
+against the oracle, through the C ABI: both scan kernels (streaming tiles of several group
+widths; one thread per sequence for fewer than 16 states), in place and out of place, ragged
+last tiles, error paths."""
 import numpy as np
 import pytest
 
@@ -27,9 +28,10 @@ def _abar(rng, P):
     return np.exp(lam * dt).astype(np.complex64)
 
 
-# (B, T, P): small B with long T -> chunked; large B*P -> one thread per sequence
+# (B, T, P): P = 8 -> one thread per sequence; otherwise tiles of 16..128 states, the narrow ones
+# when B is small; T around multiples of the tile heights; P that is not a multiple of the width
 SCAN_SHAPES = [(1, 1, 8), (2, 63, 8), (3, 64, 24), (2, 65, 40), (1, 1000, 264), (4, 517, 128),
-               (2, 4100, 16), (800, 70, 256)]
+               (2, 4100, 16), (800, 70, 256), (40, 129, 136), (600, 33, 128), (5, 256, 64)]
 
 
 @pytest.mark.parametrize("B,T,P", SCAN_SHAPES)
