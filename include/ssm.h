@@ -157,6 +157,26 @@ int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* De
                   ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
                   ssm_c64* dx0, void* stream);
 
+/* ---- single-step mode: Sec. IV-A Eq. "wm", x_t, y_t = SSM(u_t, done_t, x_{t-1}) ------
+ * The form the world model is called in when a policy sits between two steps (imagination
+ * rollouts, Sec. IV-B; context warm-up followed by a rollout): one time step for B
+ * trajectories, the state handed from call to call by the caller.
+ *   x_next[b,p] = (done[b] ? 0 : Abar[p] x_prev[b,p]) + sum_h Bbar[p,h] u[b,h]
+ *   y[b,h]      = Re sum_p C[h,p] x_next[b,p] + D[h] u[b,h]
+ * ssm_step_prepare discretises the parameters and packs the projection operands into ws
+ * once (again after every parameter update); ssm_step then runs the step from that
+ * workspace and may be called any number of times.  shape->T is ignored (taken as 1);
+ * u, y are [B,H] in io_dtype; done is [B] or NULL; x_next may alias x_prev.  The state
+ * entering the first step is the xT of ssm_layer_fwd over the context, or zero. */
+size_t ssm_step_workspace_bytes(const ssm_shape* shape);
+int ssm_step_prepare(const ssm_shape* shape, const ssm_c64* Lambda /*[P]*/, const float* Delta /*[P]*/,
+                     const ssm_c64* Bc /*[P,H]*/, const ssm_c64* Cc /*[H,P]*/, void* ws,
+                     size_t ws_bytes, void* stream);
+int ssm_step(const ssm_shape* shape, const float* D /*[H]*/, const void* u /*[B,H] io*/,
+             const uint8_t* done /*[B] or NULL*/, const ssm_c64* x_prev /*[B,P]*/,
+             ssm_c64* x_next /*[B,P] out*/, void* y /*[B,H] io, out*/, void* ws, size_t ws_bytes,
+             void* stream);
+
 /* ---- stacked sequence model --------------------------------------------------------
  * n_layers layers of   v = SSM_l(u_l);  u_{l+1} = LayerNorm(u_l + GELU(v)) * ln_weight + ln_bias
  * (exact erf GELU, LayerNorm over the H features with eps 1e-5), the same done flags in every

@@ -27,6 +27,7 @@ EXPORTS = (
     "ssm_layer_workspace_bytes", "ssm_layer_fwd", "ssm_layer_bwd",
     "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static",
     "ssm_stack_workspace_bytes", "ssm_stack_fwd", "ssm_stack_bwd",
+    "ssm_step_workspace_bytes", "ssm_step_prepare", "ssm_step",
 )
 SSM_ERR_TOO_LARGE = -8
 SSM_STATIC_SCRATCH_BYTES = 8 << 20
@@ -88,6 +89,12 @@ def _load() -> ctypes.CDLL:
     lib.ssm_stack_bwd.restype = c_int
     lib.ssm_stack_bwd.argtypes = [S, c_int, POINTER(ssm_stack_params), P, P, P, P, c_size_t, P,
                                   POINTER(ssm_stack_grads), P]
+    lib.ssm_step_workspace_bytes.restype = c_size_t
+    lib.ssm_step_workspace_bytes.argtypes = [S]
+    lib.ssm_step_prepare.restype = c_int
+    lib.ssm_step_prepare.argtypes = [S] + [P] * 5 + [c_size_t, P]
+    lib.ssm_step.restype = c_int
+    lib.ssm_step.argtypes = [S] + [P] * 7 + [c_size_t, P]
     lib.ssm_launch_count.restype = ctypes.c_longlong
     lib.ssm_launch_count.argtypes = []
     lib.ssm_profile_begin.restype = c_int
@@ -195,6 +202,20 @@ def ssm_layer_bwd(shape, Lambda, Delta, Bc, Cc, D, u, done, x0, gy, gxT, ws, du,
                            _ptr(done), _ptr(x0), _ptr(gy), _ptr(gxT), _ptr(ws), _nbytes(ws), _ptr(du),
                            _ptr(dLambda), _ptr(dDelta), _ptr(dB), _ptr(dC), _ptr(dD), _ptr(dx0),
                            _stream(stream)), "ssm_layer_bwd")
+
+
+def ssm_step_workspace_bytes(shape) -> int:
+    return int(_lib.ssm_step_workspace_bytes(byref(shape)))
+
+
+def ssm_step_prepare(shape, Lambda, Delta, Bc, Cc, ws, stream=None) -> None:
+    _ok(_lib.ssm_step_prepare(byref(shape), _ptr(Lambda), _ptr(Delta), _ptr(Bc), _ptr(Cc), _ptr(ws), _nbytes(ws),
+                              _stream(stream)), "ssm_step_prepare")
+
+
+def ssm_step(shape, D, u, done, x_prev, x_next, y, ws, stream=None) -> None:
+    _ok(_lib.ssm_step(byref(shape), _ptr(D), _ptr(u), _ptr(done), _ptr(x_prev), _ptr(x_next), _ptr(y), _ptr(ws),
+                      _nbytes(ws), _stream(stream)), "ssm_step")
 
 
 def _struct_array(cls, dicts):

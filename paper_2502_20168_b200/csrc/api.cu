@@ -171,24 +171,27 @@ SSM_API size_t ssm_layer_workspace_bytes(const ssm_shape* shape) {
     return plan_layer(*shape).total;
 }
 
-// Launch sequence of one layer's forward pass.  `hdr` receives the status of bounded waits.
-static int layer_fwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
-                          const ssm_c64* Bc, const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
-                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr, cudaStream_t st) {
+// Discretised parameters and packed projection operands into the workspace.
+static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
+                          const ssm_c64* Bc, const ssm_c64* Cc, void* ws, cudaStream_t st) {
+    StageTimer tm("discretize_pack", st);
+    launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
+                      at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
+    if (p.tc)
+        launch_pack_operands_tc(s.H, s.P, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+                                at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
+    else
+        launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+                             at<void>(ws, p.W3), at<void>(ws, p.W2), at<void>(ws, p.W1), st);
+}
+
+// Launch sequence of one layer's forward pass from a prepared workspace.  `hdr` receives the
+// status of bounded waits.
+static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D, const void* u, const uint8_t* done,
+                         const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr, cudaStream_t st) {
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T, P2 = 2 * s.P;
     int rc = SSM_OK;
-    {
-        StageTimer tm("discretize_pack", st);
-        launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
-                          at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
-        if (p.tc)
-            launch_pack_operands_tc(s.H, s.P, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
-                                    at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
-        else
-            launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
-                                 at<void>(ws, p.W3), at<void>(ws, p.W2), at<void>(ws, p.W1), st);
-    }
     if (p.tc) {
         {   // Bu[m, 2p+c] = sum_h u[m,h] Bbar_c[p,h]     (weights as hi + lo bf16)
             StageTimer tm("gemm_Bu", st);
@@ -233,6 +236,12 @@ static int layer_fwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
     return SSM_OK;
 }
 
+static int layer_fwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
+                          const ssm_c64* Bc, const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
+                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr, cudaStream_t st) {
+    layer_prepare(s, p, Lambda, Delta, Bc, Cc, ws, st);
+    return layer_fwd_run(s, p, D, u, done, x0, y, xT, ws, hdr, st);
+}
 
 SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
                           const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
@@ -249,6 +258,46 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     WsHeader* hdr = at<WsHeader>(ws, p.hdr);
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     return layer_fwd_impl(s, p, Lambda, Delta, Bc, Cc, D, u, done, x0, y, xT, ws, hdr, st);
+}
+
+// Single-step mode: the layer's forward launch sequence for T = 1 from operands prepared once.
+static ssm_shape step_shape(const ssm_shape& s) {
+    ssm_shape t = s;
+    t.T = 1;
+    return t;
+}
+
+SSM_API size_t ssm_step_workspace_bytes(const ssm_shape* shape) {
+    if (check_shape(shape) != SSM_OK) return 0;
+    return plan_layer(step_shape(*shape)).total;
+}
+
+SSM_API int ssm_step_prepare(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
+                             const ssm_c64* Cc, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!Lambda || !Delta || !Bc || !Cc) return SSM_ERR_NULL;
+    if (misaligned(Lambda) || misaligned(Delta) || misaligned(Bc) || misaligned(Cc)) return SSM_ERR_ALIGN;
+    const ssm_shape s = step_shape(*shape);
+    const LayerPlan p = plan_layer(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    layer_prepare(s, p, Lambda, Delta, Bc, Cc, ws, st);
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_step(const ssm_shape* shape, const float* D, const void* u, const uint8_t* done,
+                     const ssm_c64* x_prev, ssm_c64* x_next, void* y, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!D || !u || !x_prev || !x_next || !y) return SSM_ERR_NULL;
+    if (misaligned(D) || misaligned(u) || misaligned(x_prev) || misaligned(x_next) || misaligned(y))
+        return SSM_ERR_ALIGN;
+    const ssm_shape s = step_shape(*shape);
+    const LayerPlan p = plan_layer(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    // each (trajectory, state) is read as x0 and written as xT by the same thread, so x_next may be x_prev
+    return layer_fwd_run(s, p, D, u, done, x_prev, y, x_next, ws, at<WsHeader>(ws, p.hdr), (cudaStream_t)stream);
 }
 
 // Launch sequence of one layer's backward pass.  du_add (io dtype, may be NULL) is added to du
