@@ -47,11 +47,11 @@ STAGE_MODEL = {
 
 # DRAM bytes per launch seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum, summaries under
 # profiles/) on c4_sweep_T1024_bf16, per timestep (B*T = 262144 rows).  They hold for H = 512,
-# P = 256, bf16 I/O, traffic growing in proportion to B*T; an entry is None once its kernel has
-# changed since the counters were taken.
+# P = 256, bf16 I/O at T = 1024 (the scans choose other tile shapes at other T); an entry is None
+# once its kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_TIMESTEP = {
-    "scan_fwd": 1016.9e6 / 262144,
-    "scan_bwd": 1557.3e6 / 262144,
+    "scan_fwd": 1021.7e6 / 262144,
+    "scan_bwd": 1579.9e6 / 262144,
     "gemm_Bu": None,
     "gemm_gx": None,
     "gemm_y": 781.7e6 / 262144,
@@ -298,7 +298,7 @@ def main():
         n_launch, top_ms = stages[top]
         per_launch_s = top_ms * 1e-3 / n_launch
         alg = work(w.H, w.P, s_io) * w.timesteps
-        traffic = NCU_TRAFFIC_PER_TIMESTEP.get(top) if (w.H, w.P, w.io_dtype, stacked) == (512, 256, "bf16", False) else None
+        traffic = NCU_TRAFFIC_PER_TIMESTEP.get(top) if (w.T, w.H, w.P, w.io_dtype, stacked) == (1024, 512, 256, "bf16", False) else None
         traffic = None if traffic is None else traffic * w.timesteps
         if bound == "hbm":
             achieved, peak, runit = alg / per_launch_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"

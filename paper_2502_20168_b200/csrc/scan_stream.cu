@@ -510,9 +510,14 @@ bool make_map3(CUtensorMap* map, const void* base, bool bf16, int B, int T, int 
     cuuint64_t strides[2] = {(cuuint64_t)2 * P * es, (cuuint64_t)T * 2 * P * es};
     cuuint32_t box[3] = {(cuuint32_t)2 * G, (cuuint32_t)R, 1};
     cuuint32_t estr[3] = {1, 1, 1};
+    // L2 fetch granularity no wider than a row of the box: wider would pull in neighbouring chains
+    const uint64_t row_bytes = 2 * (uint64_t)G * es;
+    const CUtensorMapL2promotion promo = row_bytes >= 256   ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+                                         : row_bytes >= 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
+                                                            : CU_TENSOR_MAP_L2_PROMOTION_L2_64B;
     return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_SWIZZLE_NONE, promo,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
