@@ -188,6 +188,39 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def time_step_mode(w, torch, sb, n_traj=4096, steps=50):
+    """Single-step mode (ssm_step) at the paper's imagination batch, 32 x 128 start states, with
+    the workload's H, P and I/O type: a rollout of `steps` calls, the state updated in place,
+    timed with CUDA events after a warm-up rollout.  Reported beside the headline, not part of it."""
+    io = torch.bfloat16 if w.io_dtype == "bf16" else torch.float32
+    d = I.draw_layer(I.small_variant(w, B=1, T=1, n_layers=1))
+    shape = sb.make_shape(n_traj, 1, w.H, w.P, w.io_dtype)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).cuda()
+    ws = sb.alloc_workspace(sb.ssm_step_workspace_bytes(shape))
+    sb.ssm_step_prepare(shape, dev(d["Lambda"], torch.complex64), dev(d["Delta"], torch.float32),
+                        dev(d["Bc"], torch.complex64), dev(d["Cc"], torch.complex64), ws)
+    D = dev(d["D"], torch.float32)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(w.seed)
+    u = torch.randn((steps, n_traj, w.H), device="cuda", generator=g).to(io)
+    x = torch.zeros((n_traj, w.P), dtype=torch.complex64, device="cuda")
+    y = torch.empty((n_traj, w.H), dtype=io, device="cuda")
+    stream = torch.cuda.current_stream()
+    for t in range(5):
+        sb.ssm_step(shape, D, u[t], None, x, x, y, ws, stream)
+    torch.cuda.synchronize()
+    n0 = sb.ssm_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(steps):
+        sb.ssm_step(shape, D, u[t], None, x, x, y, ws, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    sb.ssm_check(ws)
+    return {"trajectories": n_traj, "steps": steps, "us_per_step": e0.elapsed_time(e1) * 1e3 / steps,
+            "launches_per_step": (sb.ssm_launch_count() - n0) / steps}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -325,6 +358,8 @@ def main():
             "stage_ms_per_step": {k: round(v[1] / args.steps, 4) for k, v in stages.items()},
             "stage_share": stage_share,
         }
+        if world == 1 and not stacked:
+            line["step_mode"] = time_step_mode(w, torch, sb)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, max(1, 262144 // w.T)))))
         print(json.dumps(line))

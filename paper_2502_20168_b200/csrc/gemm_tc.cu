@@ -523,7 +523,7 @@ static int sm_count() {
 
 template <typename K>
 static bool set_smem(K kernel, size_t bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+    return set_max_dynamic_smem(reinterpret_cast<const void*>(kernel), bytes);
 }
 
 }  // namespace tc

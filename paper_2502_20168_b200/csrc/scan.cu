@@ -7,7 +7,8 @@
 //
 // The scans normally run as the TMA-fed streaming kernels of scan_stream.cu.  The kernels
 // here walk a whole sequence per thread with plain loads and stores; they serve the shapes
-// the streaming kernels do not take (fewer than 16 states) and need no tensor maps.
+// the streaming kernels do not take (fewer than 16 states) or are wasted on (fewer than 8
+// steps: single-step mode), and need no tensor maps.
 //
 // States are stored as fp32 pairs, or as bf16 pairs when they only feed bf16 tensor-core
 // operands (the arithmetic and the carried state stay fp32).
@@ -238,6 +239,33 @@ scan_bwd_seq1_kernel(int B, int T, int P, const float2* __restrict__ Abar, const
 }
 
 // =============================================================================================
+// One step (T = 1): x = keep Abar x0 + Bu, the recurrence of single-step mode
+// =============================================================================================
+// grid: ceil(B * P/2 / 256); thread -> (b, pair of states).  x is written in the layout the next
+// kernel wants and, if asked for, as the fp32 final state xT (which may be the array x0 came from:
+// a thread reads its entry before it writes it).
+template <typename XT>
+__global__ void __launch_bounds__(256)
+scan_fwd_step_kernel(int B, int P2, const float4* __restrict__ Abar, const float4* __restrict__ Alo,
+                     const float4* __restrict__ Bu, const uint8_t* __restrict__ done, const float4* x0, XT* x,
+                     float4* xT) {
+    const int idx = blockIdx.x * 256 + threadIdx.x;
+    if (idx >= B * P2) return;
+    const int b = idx / P2, pp = idx - b * P2;
+    const size_t plane = (size_t)B * P2;
+    C2 s = c2_from(Bu[idx]);
+    if (x0 && !(done && done[b] != 0)) {
+        const C2 a = c2_from(Abar[pp]);
+        const C2 al = Alo ? c2_from(Alo[pp]) : c2_zero();
+        const C2 prev = c2_from(x0[idx]);
+        s.a = cfma2(a.a, al.a, prev.a, s.a);
+        s.b = cfma2(a.b, al.b, prev.b, s.b);
+    }
+    StateIO<XT>::store(x + idx, s, plane);
+    if (xT) xT[idx] = c2_pack(s);
+}
+
+// =============================================================================================
 // Host side
 // =============================================================================================
 // Scratch layout: [counter of the streaming kernels (256 B)][gAbar partials: B rows of P float2]
@@ -266,6 +294,10 @@ ScanPlan plan_scan(int B, int P) {
 
 }  // namespace
 
+// Sequences of a few steps (single-step mode above all) are not worth a tile pipeline: one
+// thread per state walks them.
+static bool use_stream(int B, int T, int P) { return T >= 8 && scan_stream_supported(B, T, P); }
+
 size_t scan_scratch_bytes(int B, int T, int P) {
     (void)T;
     return align_up(plan_scan(B, P).total, 256);
@@ -274,7 +306,20 @@ size_t scan_scratch_bytes(int B, int T, int P) {
 int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu, const uint8_t* done,
                     const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr, void* scratch,
                     cudaStream_t st) {
-    if (scan_stream_supported(B, T, P))
+    if (T == 1) {
+        const int n = B * (P / 2);
+        count_launch();
+        if (x_bf16)
+            scan_fwd_step_kernel<uint2><<<(n + 255) / 256, 256, 0, st>>>(B, P / 2, (const float4*)Abar, (const float4*)Alo,
+                                                                         (const float4*)Bu, done, (const float4*)x0,
+                                                                         (uint2*)x, (float4*)xT);
+        else
+            scan_fwd_step_kernel<float4><<<(n + 255) / 256, 256, 0, st>>>(B, P / 2, (const float4*)Abar, (const float4*)Alo,
+                                                                          (const float4*)Bu, done, (const float4*)x0,
+                                                                          (float4*)x, (float4*)xT);
+        return SSM_OK;
+    }
+    if (use_stream(B, T, P))
         return launch_scan_fwd_stream(B, T, P, Abar, Alo, Bu, done, x0, x, x_bf16, xT, hdr,
                                       &reinterpret_cast<ScanCounters*>(scratch)->ticket, st);
     const int P2 = P / 2;
@@ -297,7 +342,7 @@ int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
     float* part = reinterpret_cast<float*>(base + s.off_part);
     float* tmp = reinterpret_cast<float*>(base + s.off_tmp);
     if (x_bf16 != s_bf16) return SSM_ERR_DTYPE;
-    if (scan_stream_supported(B, T, P)) {
+    if (use_stream(B, T, P)) {
         const int err = launch_scan_bwd_stream(B, T, P, Abar, Alo, done, x0, x, x_bf16, gx, gxT, gBu, gx0, (float2*)part,
                                                hdr, &reinterpret_cast<ScanCounters*>(scratch)->ticket, st);
         if (err != SSM_OK) return err;

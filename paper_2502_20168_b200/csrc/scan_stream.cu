@@ -567,7 +567,7 @@ Args make_args(int B, int T, int P, int rows, const float2* Abar, const float2* 
 
 template <typename K>
 bool set_smem(K kernel, size_t bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+    return set_max_dynamic_smem(reinterpret_cast<const void*>(kernel), bytes);
 }
 
 }  // namespace

@@ -28,10 +28,11 @@ def _abar(rng, P):
     return np.exp(lam * dt).astype(np.complex64)
 
 
-# (B, T, P): P = 8 -> one thread per sequence; otherwise tiles of 16..128 states, the narrow ones
+# (B, T, P): P = 8 or T < 8 -> one thread per sequence; otherwise tiles of 16..128 states, the narrow ones
 # when B is small; T around multiples of the tile heights; P that is not a multiple of the width
 SCAN_SHAPES = [(1, 1, 8), (2, 63, 8), (3, 64, 24), (2, 65, 40), (1, 1000, 264), (4, 517, 128),
-               (2, 4100, 16), (800, 70, 256), (40, 129, 136), (600, 33, 128), (5, 256, 64)]
+               (2, 4100, 16), (800, 70, 256), (40, 129, 136), (600, 33, 128), (5, 256, 64), (300, 1, 128),
+               (7, 7, 32), (6, 8, 32)]
 
 
 @pytest.mark.parametrize("B,T,P", SCAN_SHAPES)
