@@ -13,6 +13,10 @@
 // warps 2..5 drain accumulators (one TMEM lane quarter each).  Every mbarrier wait is bounded;
 // a wait that gives up raises a CTA-wide abort flag, the status word of the workspace header
 // is set, tensor memory is released and the kernel returns.
+#include <map>
+#include <mutex>
+#include <utility>
+
 #include "kernels.h"
 #include "tma.cuh"
 
@@ -63,6 +67,59 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 // Arrives on the mbarrier once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// ---- CTA pairs (cta_group::2): one MMA spans the tensor cores and tensor memory of two CTAs
+// of a cluster; each CTA holds its 128 rows of A and its half of the B rows in shared memory at
+// the same offsets.  Allocation and release of tensor memory are issued by one warp of each CTA.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// Asks L2 to fetch a contiguous range (a multiple of 16 bytes from a 16-byte aligned address).
+__device__ __forceinline__ void l2_prefetch_bulk(const void* ptr, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"(bytes) : "memory");
+}
+// Tile load whose completion is counted on a barrier of either CTA of the pair (cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrives on the barrier at this offset in both CTAs once every MMA issued so far has completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
 
 // 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (base lane + i).
@@ -116,11 +173,12 @@ struct Smem {
 };
 
 // Layout: [stages][epilogue staging][diag copy][barriers]; the NT kernel has no staging / diag.
-__device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging_bytes, int diag_bytes) {
+__device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging_bytes, int diag_bytes,
+                                           int stage_bytes = kStageBytes) {
     Smem s;
     uintptr_t base = (reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023;
     s.tiles = reinterpret_cast<uint8_t*>(base);
-    s.staging = s.tiles + (size_t)stages * kStageBytes;
+    s.staging = s.tiles + (size_t)stages * stage_bytes;
     s.diag = reinterpret_cast<float*>(s.staging + staging_bytes);
     uint8_t* bars = s.staging + staging_bytes + diag_bytes;
     for (int i = 0; i < kStages; ++i) {
@@ -184,7 +242,120 @@ struct TnParams {
     const __nv_bfloat16* skip;
     const __nv_bfloat16* add;
     WsHeader* hdr;
+    const char* a_base;   // A as bytes; rows are K * 2 bytes apart and contiguous
+    int a_row_bytes;
 };
+
+// One epilogue warp's share of a finished accumulator tile: rows m0 + 32 (warp % 4) .. + 31, one half
+// of the tile's output columns (from n_out0).  Waits for the tile's MMAs; false when aborting.
+template <int kEpi, bool kSplitW>
+__device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, const CUtensorMap* tmOut, int warp,
+                                              int lane, int m0, int n_out0, int acc, uint32_t acc_phase,
+                                              uint32_t tmem_base) {
+    constexpr int kOutCols = kSplitW ? BN / 2 : BN;
+    const int q = warp & 3;             // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp drains
+    const int row0 = m0 + q * 32;   // first of this warp's 32 rows
+    // skip[m, n] slabs are fetched kPre slabs ahead of their use (the first ones while the
+    // tile's MMAs are still running): lane -> (row i*8 + lane/4, 8 columns) per slab
+    constexpr int kSlabs = kOutCols / 32 / 2, kPre = kSlabs - 1 < 3 ? kSlabs - 1 : 3;
+    const int slab0 = half * kSlabs;   // this warp's slabs: slab0 .. slab0 + kSlabs - 1
+    uint4 skb[kPre + 1][4];
+    auto load_skip = [&](int slab, uint4 (&dst)[4]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int rr = i * 8 + (lane >> 2);
+            if (row0 + rr < p.M)
+                dst[i] = __ldg(reinterpret_cast<const uint4*>(
+                    p.skip + (size_t)(row0 + rr) * p.ldo + n_out0 + (slab0 + slab) * 32 + (lane & 3) * 8));
+        }
+    };
+    if (kEpi == 1) {
+#pragma unroll
+        for (int d = 0; d < kPre; ++d) load_skip(d, skb[d]);
+    }
+    if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
+    tc_fence_after();
+    const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+    float4* stg = reinterpret_cast<float4*>(s.staging) + (size_t)(warp - 2) * (32 * 8);
+#pragma unroll
+    for (int sl = 0; sl < kSlabs; ++sl) {
+        const int c = (slab0 + sl) * 32;
+        if (kEpi == 1 && sl + kPre < kSlabs) load_skip(sl + kPre, skb[(sl + kPre) % (kPre + 1)]);
+        // TMEM -> registers: lane = row, 32 consecutive columns
+        uint32_t r[32], r2[32];
+        tmem_ld32(t_row + (uint32_t)c, r);
+        if (kSplitW) tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
+        tmem_ld_wait();
+        // registers -> staging (16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7): the
+        // 128-byte swizzle, so that the TMA unit can store the buffer as a 32 x 32 fp32 box)
+        if (kEpi == 0) {
+            if (lane == 0) tma_store_wait_read();
+        }
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                   __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+            if (kSplitW) {
+                v.x += __uint_as_float(r2[4 * j]);
+                v.y += __uint_as_float(r2[4 * j + 1]);
+                v.z += __uint_as_float(r2[4 * j + 2]);
+                v.w += __uint_as_float(r2[4 * j + 3]);
+            }
+            stg[lane * 8 + (j ^ (lane & 7))] = v;
+        }
+        __syncwarp();
+        // staging -> global with full-line accesses
+        if (kEpi == 0) {
+            // one TMA store of the 32-row x 128-byte box; rows past M are clipped by the unit
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0 && row0 < p.M) tma_store_2d(tmOut, smem_u32(stg), n_out0 + c, row0);
+        } else {
+            // each instruction covers 8 rows x 64 bytes of bf16: lane -> (row i*8 + lane/4, 8 columns)
+            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+            const int cq = lane & 3;
+            const float4 d0 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8);
+            const float4 d1 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8 + 4);
+            const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int rr = i * 8 + (lane >> 2);
+                const float4 a0 = stg[rr * 8 + ((2 * cq) ^ (rr & 7))];
+                const float4 a1 = stg[rr * 8 + ((2 * cq + 1) ^ (rr & 7))];
+                if (row0 + rr < p.M) {
+                    const size_t off = (size_t)(row0 + rr) * p.ldo + n_out0 + c + cq * 8;
+                    const uint4 sv = skb[sl % (kPre + 1)][i];
+                    const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
+                    float o[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 sf = __bfloat1622float2(s2[j]);
+                        o[2 * j] = fmaf(dd[2 * j], sf.x, o[2 * j]);
+                        o[2 * j + 1] = fmaf(dd[2 * j + 1], sf.y, o[2 * j + 1]);
+                    }
+                    if (p.add) {
+                        const uint4 av = *reinterpret_cast<const uint4*>(p.add + off);
+                        const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&av);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 af = __bfloat1622float2(a2[j]);
+                            o[2 * j] += af.x;
+                            o[2 * j + 1] += af.y;
+                        }
+                    }
+                    uint4 ov;
+                    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(o[2 * j], o[2 * j + 1]);
+                    *reinterpret_cast<uint4*>(out + off) = ov;
+                }
+            }
+        }
+    }
+    return true;
+}
 
 // kEpi 0: store fp32;  kEpi 1: out = bf16(acc + diag[n] * skip[m, n] (+ add[m, n])).
 // kSplitW: columns [0,128) and [128,256) of the accumulator tile are the hi and lo weight
@@ -266,105 +437,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
             const int m0 = (tile / p.n_tiles) * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
-            const int row0 = m0 + q * 32;   // first of this warp's 32 rows
-            // skip[m, n] slabs are fetched kPre slabs ahead of their use (the first ones while the
-            // tile's MMAs are still running): lane -> (row i*8 + lane/4, 8 columns) per slab
-            constexpr int kSlabs = kOutCols / 32 / 2, kPre = kSlabs - 1 < 3 ? kSlabs - 1 : 3;
-            const int slab0 = half * kSlabs;   // this warp's slabs: slab0 .. slab0 + kSlabs - 1
-            uint4 skb[kPre + 1][4];
-            auto load_skip = [&](int slab, uint4 (&dst)[4]) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int rr = i * 8 + (lane >> 2);
-                    if (row0 + rr < p.M)
-                        dst[i] = __ldg(reinterpret_cast<const uint4*>(
-                            p.skip + (size_t)(row0 + rr) * p.ldo + n_out0 + (slab0 + slab) * 32 + (lane & 3) * 8));
-                }
-            };
-            if (kEpi == 1) {
-#pragma unroll
-                for (int d = 0; d < kPre; ++d) load_skip(d, skb[d]);
-            }
-            if (!(ok = mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag))) break;
-            tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-            float4* stg = reinterpret_cast<float4*>(s.staging) + (size_t)(warp - 2) * (32 * 8);
-#pragma unroll
-            for (int sl = 0; sl < kSlabs; ++sl) {
-                const int c = (slab0 + sl) * 32;
-                if (kEpi == 1 && sl + kPre < kSlabs) load_skip(sl + kPre, skb[(sl + kPre) % (kPre + 1)]);
-                // TMEM -> registers: lane = row, 32 consecutive columns
-                uint32_t r[32], r2[32];
-                tmem_ld32(t_row + (uint32_t)c, r);
-                if (kSplitW) tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
-                tmem_ld_wait();
-                // registers -> staging (16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7): the
-                // 128-byte swizzle, so that the TMA unit can store the buffer as a 32 x 32 fp32 box)
-                if (kEpi == 0) {
-                    if (lane == 0) tma_store_wait_read();
-                }
-                __syncwarp();
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                           __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-                    if (kSplitW) {
-                        v.x += __uint_as_float(r2[4 * j]);
-                        v.y += __uint_as_float(r2[4 * j + 1]);
-                        v.z += __uint_as_float(r2[4 * j + 2]);
-                        v.w += __uint_as_float(r2[4 * j + 3]);
-                    }
-                    stg[lane * 8 + (j ^ (lane & 7))] = v;
-                }
-                __syncwarp();
-                // staging -> global with full-line accesses
-                if (kEpi == 0) {
-                    // one TMA store of the 32-row x 128-byte box; rows past M are clipped by the unit
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && row0 < p.M) tma_store_2d(&tmOut, smem_u32(stg), n_out0 + c, row0);
-                } else {
-                    // each instruction covers 8 rows x 64 bytes of bf16: lane -> (row i*8 + lane/4, 8 columns)
-                    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-                    const int cq = lane & 3;
-                    const float4 d0 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8);
-                    const float4 d1 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8 + 4);
-                    const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int rr = i * 8 + (lane >> 2);
-                        const float4 a0 = stg[rr * 8 + ((2 * cq) ^ (rr & 7))];
-                        const float4 a1 = stg[rr * 8 + ((2 * cq + 1) ^ (rr & 7))];
-                        if (row0 + rr < p.M) {
-                            const size_t off = (size_t)(row0 + rr) * p.ldo + n_out0 + c + cq * 8;
-                            const uint4 sv = skb[sl % (kPre + 1)][i];
-                            const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
-                            float o[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float2 sf = __bfloat1622float2(s2[j]);
-                                o[2 * j] = fmaf(dd[2 * j], sf.x, o[2 * j]);
-                                o[2 * j + 1] = fmaf(dd[2 * j + 1], sf.y, o[2 * j + 1]);
-                            }
-                            if (p.add) {
-                                const uint4 av = *reinterpret_cast<const uint4*>(p.add + off);
-                                const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&av);
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const float2 af = __bfloat1622float2(a2[j]);
-                                    o[2 * j] += af.x;
-                                    o[2 * j + 1] += af.y;
-                                }
-                            }
-                            uint4 ov;
-                            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(o[2 * j], o[2 * j + 1]);
-                            *reinterpret_cast<uint4*>(out + off) = ov;
-                        }
-                    }
-                }
-            }
+            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, warp, lane, m0, n_out0, acc, acc_phase, tmem_base))) break;
             tc_fence_before();
             mbar_arrive(s.tmem_empty[acc]);
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
@@ -372,6 +445,145 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (kEpi == 0 && lane == 0) tma_store_wait_all();
     }
     epilogue_exit(s, warp, tmem_base, p.hdr);
+}
+
+// ---------------------------------------------------------------------------------------------
+// TN kernel on CTA pairs
+// ---------------------------------------------------------------------------------------------
+// Same product, same epilogue, but a cluster of two CTAs works on a 256 x 256 accumulator tile:
+// CTA r holds rows m0 + 128 r .. of A and rows n0 + 128 r .. of the W tile, so every CTA brings
+// in 32 KB per k-block instead of 48 KB for the same number of tensor-core cycles (operand
+// delivery into the SM, not the tensor pipe, bounds the single-CTA kernel).  The leader (CTA 0)
+// issues the MMAs; its `full` barriers count the bytes of both CTAs' loads; its commits arrive
+// on the `empty` / `tmem_full` barriers of both CTAs; both CTAs' epilogue warps arrive on the
+// leader's `tmem_empty` barriers.
+constexpr int kPairStages = 4;
+constexpr int kPairStageBytes = kABytes + kBBytes / 2;
+constexpr size_t kPairSmemBytes = (size_t)kPairStages * kPairStageBytes + kStagingBytes + kMaxDiag * 4 + 1024 + 256;
+
+template <int kEpi, bool kSplitW>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTnThreads, 1)
+gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
+                       const __grid_constant__ CUtensorMap tmOut, TnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, kPairStages, kStagingBytes, kMaxDiag * 4, kPairStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    if (kEpi == 1)
+        for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
+    // barriers and tensor memory (both CTAs), then the whole pair meets
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(s.full[i], 1);
+            mbar_init(s.empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s.tmem_full[i], 1);
+            mbar_init(s.tmem_empty[i], 2 * 32 * kTnEpiWarps);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == 1) tmem_alloc_pair(s.tmem_slot, kTmemCols);
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *s.tmem_slot_ptr;
+
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int m_pairs = (p.M + 2 * BM - 1) / (2 * BM);
+    const int total = m_pairs * p.n_tiles;
+    constexpr int kOutCols = kSplitW ? BN / 2 : BN;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmWh);
+            uint32_t leader_full[kPairStages];
+            for (int i = 0; i < kPairStages; ++i) leader_full[i] = map_to_cta(s.full[i], 0);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            // The 128 rows of A a tile needs are one contiguous range: have L2 fetch the next tile's
+            // range in one piece, so that DRAM sees long bursts instead of 128-byte row pieces.
+            auto prefetch_a = [&](int tile) {
+                if (tile >= total) return;
+                const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM;
+                const int rows = min(BM, p.M - m0);
+                if (rows > 0) l2_prefetch_bulk(p.a_base + (size_t)m0 * p.a_row_bytes, (uint32_t)rows * p.a_row_bytes);
+            };
+            prefetch_a(pair);
+            for (int tile = pair; tile < total && ok; tile += npairs) {
+                const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM;
+                const int n0 = (tile % p.n_tiles) * BN + (int)rank * (BN / 2);
+                prefetch_a(tile + npairs);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag))) break;
+                    if (rank == 0) mbar_expect_tx(s.full[stage], 2 * kPairStageBytes);
+                    const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                    tma_load_2d_pair(a_dst, &tmA, leader_full[stage], kb * BK, m0);
+                    tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full[stage], kb * BK, n0);
+                    if (++stage == kPairStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = instr_desc(2 * BM, BN, 0, 0);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total && ok; tile += npairs) {
+                if (!(ok = mbar_wait(s.tmem_empty[acc], acc_phase ^ 1u, s.abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                    const uint64_t adesc = smem_desc_kmajor(a_addr);
+                    const uint64_t bdesc = smem_desc_kmajor(a_addr + kABytes);
+#pragma unroll
+                    for (int k = 0; k < BK / UK; ++k)
+                        umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                       (uint32_t)((kb | k) != 0));
+                    umma_commit_pair(s.empty[stage]);
+                    if (++stage == kPairStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit_pair(s.tmem_full[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1u;
+            }
+        }
+    } else {
+        const uint32_t leader_empty[2] = {map_to_cta(s.tmem_empty[0], 0), map_to_cta(s.tmem_empty[1], 0)};
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = pair; tile < total && ok; tile += npairs) {
+            const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
+            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, warp, lane, m0, n_out0, acc, acc_phase, tmem_base))) break;
+            tc_fence_before();
+            mbar_arrive_cluster(leader_empty[acc]);
+            if ((acc ^= 1) == 0) acc_phase ^= 1u;
+        }
+        if (kEpi == 0 && lane == 0) tma_store_wait_all();
+    }
+    // nobody leaves (or frees tensor memory) while the other CTA may still signal or compute
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync_all();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+    if (threadIdx.x == 0 && *s.abort_flag && p.hdr) p.hdr->status = SSM_ERR_TIMEOUT;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -521,6 +733,36 @@ static int sm_count() {
     return n;
 }
 
+// How many clusters of two CTAs of `kernel` the current device runs at the same time (cached per
+// kernel and device).
+static int resident_pairs(const void* kernel, size_t smem_bytes) {
+    static std::mutex mu;
+    static std::map<std::pair<const void*, int>, int> cache;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find({kernel, dev});
+    if (it != cache.end()) return it->second;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)sm_count(), 1, 1);
+    cfg.blockDim = dim3(kTnThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    cache[{kernel, dev}] = n;
+    return n;
+}
+
 template <typename K>
 static bool set_smem(K kernel, size_t bytes) {
     return set_max_dynamic_smem(reinterpret_cast<const void*>(kernel), bytes);
@@ -546,8 +788,32 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
         mo = ma;         // unused by the bf16 epilogue
     }
     TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.out, g.diag, (const __nv_bfloat16*)g.skip,
-               (const __nv_bfloat16*)g.add, g.hdr};
+               (const __nv_bfloat16*)g.add, g.hdr, (const char*)g.A, g.K * 2};
     const int m_tiles = (g.M + BM - 1) / BM;
+    const int pair_tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * n_tiles;
+    // CTA pairs pay off where the main loop is the bottleneck (fp32 results, stored by TMA); with the
+    // bf16 epilogue, whose skip loads and stores go through the load/store units, the single-CTA
+    // kernel measured faster (0.193 vs 0.208 ms at M = 262144, N = K = 512).
+    if (g.store_f32 && pair_tiles >= sm_count() / 2) {   // enough 256-row tiles to give every pair one
+        CUtensorMap mwh;
+        if (!make_map(&mwh, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN / 2)) return SSM_ERR_CUDA;
+        count_launch();
+        bool okp = true;
+        // The kernel is persistent: its grid is the number of CTA pairs the device can hold at once
+        // (not every SM has a partner that a cluster may use).
+#define SSM_LAUNCH_PAIR(EPI, SPLIT)                                                                        \
+    do {                                                                                                   \
+        auto kern = gemm_tc_tn_pair_kernel<EPI, SPLIT>;                                                    \
+        okp = set_smem(kern, kPairSmemBytes);                                                              \
+        const int pairs = okp ? resident_pairs(reinterpret_cast<const void*>(kern), kPairSmemBytes) : 0;   \
+        okp = okp && pairs > 0;                                                                            \
+        if (okp) kern<<<2 * min(pairs, pair_tiles), kTnThreads, kPairSmemBytes, st>>>(ma, mwh, mo, p);     \
+    } while (0)
+        if (g.split_w) SSM_LAUNCH_PAIR(0, true);
+        else SSM_LAUNCH_PAIR(0, false);
+#undef SSM_LAUNCH_PAIR
+        return okp ? SSM_OK : SSM_ERR_CUDA;
+    }
     const int grid = min(sm_count(), m_tiles * n_tiles);
     count_launch();
     bool ok;
