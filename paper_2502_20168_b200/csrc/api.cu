@@ -195,8 +195,7 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D,
     if (p.tc) {
         {   // Bu[m, 2p+c] = sum_h u[m,h] Bbar_c[p,h]     (weights as hi + lo bf16)
             StageTimer tm("gemm_Bu", st);
-            GemmTcTN g{u, at<void>(ws, p.W0), BT, P2, s.H, true, true, at<void>(ws, p.f32buf),
-                       nullptr, nullptr, nullptr, hdr};
+            GemmTcTN g{u, at<void>(ws, p.W0), BT, P2, s.H, true, true, at<void>(ws, p.f32buf), nullptr, nullptr, hdr};
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
         }
         {
@@ -208,7 +207,7 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D,
         }
         {   // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
             StageTimer tm("gemm_y", st);
-            GemmTcTN g{at<void>(ws, p.xs), at<void>(ws, p.W2), BT, s.H, P2, false, false, y, D, u, nullptr, hdr};
+            GemmTcTN g{at<void>(ws, p.xs), at<void>(ws, p.W2), BT, s.H, P2, false, false, y, D, u, hdr};
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
         }
     } else {
@@ -316,8 +315,7 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
     if (p.tc) {
         {   // gx[m, 2p+c] = sum_h gy[m,h] conj(C)_c[h,p]   (weights as hi + lo bf16)
             StageTimer tm("gemm_gx", st);
-            GemmTcTN g{gy, at<void>(ws, p.W1), BT, P2, s.H, true, true, at<void>(ws, p.f32buf),
-                       nullptr, nullptr, nullptr, hdr};
+            GemmTcTN g{gy, at<void>(ws, p.W1), BT, P2, s.H, true, true, at<void>(ws, p.f32buf), nullptr, nullptr, hdr};
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
         }
         {
@@ -330,7 +328,8 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
         }
         {   // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]
             StageTimer tm("gemm_du", st);
-            GemmTcTN g{at<void>(ws, p.gs), at<void>(ws, p.W3), BT, s.H, P2, false, false, du, D, gy, du_add, hdr};
+            if (du_add) return SSM_ERR_SHAPE;   // the residual addend exists only on the CUDA-core path (stacks)
+            GemmTcTN g{at<void>(ws, p.gs), at<void>(ws, p.W3), BT, s.H, P2, false, false, du, D, gy, hdr};
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
         }
         {   // gBbar[p,h] = sum_m s[m,p] u[m,h]

@@ -39,8 +39,13 @@ constexpr int kTnThreads = 64 + 32 * kTnEpiWarps;
 constexpr int kTmemCols = 512;  // two accumulator buffers of BN columns
 constexpr int kStagingBytes = kTnEpiWarps * 32 * 32 * 4;  // per epilogue warp: 32 rows x 32 fp32 columns
 constexpr int kMaxDiag = 4096;                  // widest output whose diagonal fits the shared copy
-constexpr size_t kTnSmemBytes = (size_t)kTnStages * kStageBytes + kStagingBytes + kMaxDiag * 4 +
-                                1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kSkipBytes = kTnEpiWarps * 2 * 32 * 32 * 2;   // bf16 epilogue: two 32 x 32 bf16 skip tiles per warp
+__host__ __device__ constexpr int tn_skip_bytes(int epi) { return epi == 1 ? kSkipBytes : 0; }
+__host__ __device__ constexpr int tn_diag_bytes(int epi) { return epi == 1 ? kMaxDiag * 4 : 0; }
+constexpr size_t tn_smem_bytes(int epi) {
+    return (size_t)kTnStages * kStageBytes + kStagingBytes + tn_skip_bytes(epi) + tn_diag_bytes(epi) +
+           1024 /*alignment slack*/ + 256 /*barriers*/;
+}
 constexpr size_t kNtSmemBytes = (size_t)kStages * kStageBytes + 1024 + 256;
 
 // ---------------------------------------------------------------------------------------------
@@ -166,21 +171,25 @@ struct Smem {
     uint8_t* tiles;       // 1024-byte aligned
     uint8_t* staging;     // epilogue transpose buffers
     float* diag;          // copy of the epilogue's diagonal
+    uint8_t* skipbuf;     // bf16 epilogue: per epilogue warp two 32 x 32 bf16 tiles of the skip operand
     uint32_t full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    uint32_t skip_full[2 * kTnEpiWarps];
     uint32_t tmem_slot;   // where tcgen05.alloc writes the base address
     volatile int* abort_flag;
     volatile uint32_t* tmem_slot_ptr;
 };
 
-// Layout: [stages][epilogue staging][diag copy][barriers]; the NT kernel has no staging / diag.
+// Layout: [stages][epilogue staging][skip tiles][diag copy][barriers]; the NT kernel has none of the
+// epilogue buffers.
 __device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging_bytes, int diag_bytes,
-                                           int stage_bytes = kStageBytes) {
+                                           int stage_bytes = kStageBytes, int skip_bytes = 0) {
     Smem s;
     uintptr_t base = (reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023;
     s.tiles = reinterpret_cast<uint8_t*>(base);
     s.staging = s.tiles + (size_t)stages * stage_bytes;
-    s.diag = reinterpret_cast<float*>(s.staging + staging_bytes);
-    uint8_t* bars = s.staging + staging_bytes + diag_bytes;
+    s.skipbuf = s.staging + staging_bytes;
+    s.diag = reinterpret_cast<float*>(s.skipbuf + skip_bytes);
+    uint8_t* bars = s.skipbuf + skip_bytes + diag_bytes;
     for (int i = 0; i < kStages; ++i) {
         s.full[i] = smem_u32(bars + 8 * i);
         s.empty[i] = smem_u32(bars + 8 * (kStages + i));
@@ -192,6 +201,7 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging
     s.tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(bars + 8 * (2 * kStages + 4));
     s.tmem_slot = smem_u32(bars + 8 * (2 * kStages + 4));
     s.abort_flag = reinterpret_cast<volatile int*>(bars + 8 * (2 * kStages + 4) + 4);
+    for (int i = 0; i < 2 * kTnEpiWarps; ++i) s.skip_full[i] = smem_u32(bars + 8 * (2 * kStages + 5 + i));
     return s;
 }
 
@@ -206,6 +216,7 @@ __device__ __forceinline__ uint32_t prologue(const Smem& s, int warp, int lane, 
             mbar_init(s.tmem_full[i], 1);
             mbar_init(s.tmem_empty[i], epilogue_threads);
         }
+        for (int i = 0; i < 2 * kTnEpiWarps; ++i) mbar_init(s.skip_full[i], 1);
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -236,136 +247,134 @@ struct TnParams {
     int M;            // rows of A / out
     int n_tiles;      // accumulator tiles along N (each BN columns of W rows)
     int k_blocks;     // K / BK
-    int ldo;          // leading dimension of out (and skip/add)
-    void* out;        // fp32 (kEpi == 0) or bf16 (kEpi == 1)
+    int ldo;          // leading dimension of out (and skip): the number of output columns
     const float* diag;
-    const __nv_bfloat16* skip;
-    const __nv_bfloat16* add;
     WsHeader* hdr;
     const char* a_base;   // A as bytes; rows are K * 2 bytes apart and contiguous
     int a_row_bytes;
 };
 
 // One epilogue warp's share of a finished accumulator tile: rows m0 + 32 (warp % 4) .. + 31, one half
-// of the tile's output columns (from n_out0).  Waits for the tile's MMAs; false when aborting.
+// of the tile's output columns (from n_out0), in slabs of 32 columns; a lane holds one row of a slab.
+// Waits for the tile's MMAs; false when aborting.
+//  kEpi 0: fp32 results.  The slab goes through a 128-byte-swizzled staging buffer and leaves as
+//          one TMA store of a 32 x 32 box (rows past M are clipped by the unit).
+//  kEpi 1: out = bf16(acc + diag[n] * skip[m, n]).  The skip slab arrives by TMA (two buffers per
+//          warp, fetched two slabs ahead, the first ones while the tile's MMAs still run) and the
+//          bf16 slab leaves by TMA, both as 32 x 32 boxes with the 64-byte swizzle, so a lane reads
+//          and writes its own 64-byte row without bank conflicts and nothing passes through the
+//          load/store path to global memory.  `skip_phase`: the warp's barrier parities (bit b).
 template <int kEpi, bool kSplitW>
-__device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, const CUtensorMap* tmOut, int warp,
-                                              int lane, int m0, int n_out0, int acc, uint32_t acc_phase,
-                                              uint32_t tmem_base) {
+__device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, const CUtensorMap* tmOut,
+                                              const CUtensorMap* tmSkip, int warp, int lane, int m0, int n_out0,
+                                              int acc, uint32_t acc_phase, uint32_t tmem_base, uint32_t& skip_phase) {
     constexpr int kOutCols = kSplitW ? BN / 2 : BN;
     const int q = warp & 3;             // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp drains
-    const int row0 = m0 + q * 32;   // first of this warp's 32 rows
-    // skip[m, n] slabs are fetched kPre slabs ahead of their use (the first ones while the
-    // tile's MMAs are still running): lane -> (row i*8 + lane/4, 8 columns) per slab
-    constexpr int kSlabs = kOutCols / 32 / 2, kPre = kSlabs - 1 < 3 ? kSlabs - 1 : 3;
-    const int slab0 = half * kSlabs;   // this warp's slabs: slab0 .. slab0 + kSlabs - 1
-    uint4 skb[kPre + 1][4];
-    auto load_skip = [&](int slab, uint4 (&dst)[4]) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int rr = i * 8 + (lane >> 2);
-            if (row0 + rr < p.M)
-                dst[i] = __ldg(reinterpret_cast<const uint4*>(
-                    p.skip + (size_t)(row0 + rr) * p.ldo + n_out0 + (slab0 + slab) * 32 + (lane & 3) * 8));
-        }
-    };
-    if (kEpi == 1) {
-#pragma unroll
-        for (int d = 0; d < kPre; ++d) load_skip(d, skb[d]);
-    }
-    if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
-    tc_fence_after();
+    const int row0 = m0 + q * 32;       // first of this warp's 32 rows
+    constexpr int kSlabs = kOutCols / 32 / 2;
+    const int slab0 = half * kSlabs;    // this warp's slabs: slab0 .. slab0 + kSlabs - 1
     const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-    float4* stg = reinterpret_cast<float4*>(s.staging) + (size_t)(warp - 2) * (32 * 8);
+    uint8_t* stg_bytes = s.staging + (size_t)(warp - 2) * 4096;
+
+    if (kEpi == 0) {
+        if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
+        tc_fence_after();
+        float4* stg = reinterpret_cast<float4*>(stg_bytes);
 #pragma unroll
-    for (int sl = 0; sl < kSlabs; ++sl) {
-        const int c = (slab0 + sl) * 32;
-        if (kEpi == 1 && sl + kPre < kSlabs) load_skip(sl + kPre, skb[(sl + kPre) % (kPre + 1)]);
-        // TMEM -> registers: lane = row, 32 consecutive columns
-        uint32_t r[32], r2[32];
-        tmem_ld32(t_row + (uint32_t)c, r);
-        if (kSplitW) tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
-        tmem_ld_wait();
-        // registers -> staging (16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7): the
-        // 128-byte swizzle, so that the TMA unit can store the buffer as a 32 x 32 fp32 box)
-        if (kEpi == 0) {
-            if (lane == 0) tma_store_wait_read();
-        }
-        __syncwarp();
+        for (int sl = 0; sl < kSlabs; ++sl) {
+            const int c = (slab0 + sl) * 32;
+            uint32_t r[32], r2[32];
+            tmem_ld32(t_row + (uint32_t)c, r);
+            if (kSplitW) tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
+            tmem_ld_wait();
+            if (lane == 0) tma_store_wait_read();   // the previous slab has left the staging buffer
+            __syncwarp();
+            // 16-byte chunk j of row `lane` sits at chunk j ^ (lane & 7): the 128-byte swizzle
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                   __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-            if (kSplitW) {
-                v.x += __uint_as_float(r2[4 * j]);
-                v.y += __uint_as_float(r2[4 * j + 1]);
-                v.z += __uint_as_float(r2[4 * j + 2]);
-                v.w += __uint_as_float(r2[4 * j + 3]);
+            for (int j = 0; j < 8; ++j) {
+                float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                       __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                if (kSplitW) {
+                    v.x += __uint_as_float(r2[4 * j]);
+                    v.y += __uint_as_float(r2[4 * j + 1]);
+                    v.z += __uint_as_float(r2[4 * j + 2]);
+                    v.w += __uint_as_float(r2[4 * j + 3]);
+                }
+                stg[lane * 8 + (j ^ (lane & 7))] = v;
             }
-            stg[lane * 8 + (j ^ (lane & 7))] = v;
-        }
-        __syncwarp();
-        // staging -> global with full-line accesses
-        if (kEpi == 0) {
-            // one TMA store of the 32-row x 128-byte box; rows past M are clipped by the unit
             fence_async_smem();
             __syncwarp();
             if (lane == 0 && row0 < p.M) tma_store_2d(tmOut, smem_u32(stg), n_out0 + c, row0);
-        } else {
-            // each instruction covers 8 rows x 64 bytes of bf16: lane -> (row i*8 + lane/4, 8 columns)
-            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-            const int cq = lane & 3;
-            const float4 d0 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8);
-            const float4 d1 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + cq * 8 + 4);
+        }
+        return true;
+    }
+
+    // ---- kEpi == 1
+    const int w = warp - 2;
+    uint8_t* skb = s.skipbuf + (size_t)w * 4096;   // two 2 KB skip tiles
+    const uint32_t sbar[2] = {s.skip_full[2 * w], s.skip_full[2 * w + 1]};
+    const int swz = (lane >> 1) & 3;               // 64-byte swizzle: chunk c of row `lane` sits at chunk c ^ swz
+    auto fetch_skip = [&](int sl) {
+        const int b = sl & 1;
+        mbar_expect_tx(sbar[b], 2048);
+        tma_load_2d(smem_u32(skb + b * 2048), tmSkip, sbar[b], n_out0 + (slab0 + sl) * 32, row0);
+    };
+    if (lane == 0) {
+        fetch_skip(0);
+        if (kSlabs > 1) fetch_skip(1);
+    }
+    if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
+    tc_fence_after();
+#pragma unroll
+    for (int sl = 0; sl < kSlabs; ++sl) {
+        const int c = (slab0 + sl) * 32, b = sl & 1;
+        uint32_t r[32];
+        tmem_ld32(t_row + (uint32_t)c, r);
+        if (!mbar_wait(sbar[b], (skip_phase >> b) & 1u, s.abort_flag)) return false;
+        skip_phase ^= 1u << b;
+        uint4 sk[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sk[j] = *reinterpret_cast<const uint4*>(skb + b * 2048 + lane * 64 + ((j ^ swz) << 4));
+        tmem_ld_wait();
+        __syncwarp();   // every lane has its skip row: the buffer can take the slab after next
+        if (lane == 0 && sl + 2 < kSlabs) fetch_skip(sl + 2);
+        uint4 o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float4 d0 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + 8 * j);
+            const float4 d1 = *reinterpret_cast<const float4*>(s.diag + n_out0 + c + 8 * j + 4);
             const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+            const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sk[j]);
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o[j]);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int rr = i * 8 + (lane >> 2);
-                const float4 a0 = stg[rr * 8 + ((2 * cq) ^ (rr & 7))];
-                const float4 a1 = stg[rr * 8 + ((2 * cq + 1) ^ (rr & 7))];
-                if (row0 + rr < p.M) {
-                    const size_t off = (size_t)(row0 + rr) * p.ldo + n_out0 + c + cq * 8;
-                    const uint4 sv = skb[sl % (kPre + 1)][i];
-                    const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sv);
-                    float o[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 sf = __bfloat1622float2(s2[j]);
-                        o[2 * j] = fmaf(dd[2 * j], sf.x, o[2 * j]);
-                        o[2 * j + 1] = fmaf(dd[2 * j + 1], sf.y, o[2 * j + 1]);
-                    }
-                    if (p.add) {
-                        const uint4 av = *reinterpret_cast<const uint4*>(p.add + off);
-                        const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&av);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float2 af = __bfloat1622float2(a2[j]);
-                            o[2 * j] += af.x;
-                            o[2 * j + 1] += af.y;
-                        }
-                    }
-                    uint4 ov;
-                    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(o[2 * j], o[2 * j + 1]);
-                    *reinterpret_cast<uint4*>(out + off) = ov;
-                }
+            for (int e = 0; e < 4; ++e) {
+                const float2 sf = __bfloat1622float2(s2[e]);
+                o2[e] = __floats2bfloat162_rn(fmaf(dd[2 * e], sf.x, __uint_as_float(r[8 * j + 2 * e])),
+                                              fmaf(dd[2 * e + 1], sf.y, __uint_as_float(r[8 * j + 2 * e + 1])));
             }
         }
+        uint8_t* ob = stg_bytes + b * 2048;
+        if (lane == 0) tma_store_wait_read_n<1>();   // the store from this buffer two slabs ago has read it
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(ob + lane * 64 + ((j ^ swz) << 4)) = o[j];
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < p.M) tma_store_2d(tmOut, smem_u32(ob), n_out0 + c, row0);
     }
     return true;
 }
 
-// kEpi 0: store fp32;  kEpi 1: out = bf16(acc + diag[n] * skip[m, n] (+ add[m, n])).
+// kEpi 0: store fp32;  kEpi 1: out = bf16(acc + diag[n] * skip[m, n]).
 // kSplitW: columns [0,128) and [128,256) of the accumulator tile are the hi and lo weight
 // halves of the same 128 output columns.
 template <int kEpi, bool kSplitW>
 __global__ void __launch_bounds__(kTnThreads, 1)
 gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                  const __grid_constant__ CUtensorMap tmOut, TnParams p) {
+                  const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmSkip, TnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, kTnStages, kStagingBytes, kMaxDiag * 4);
+    const Smem s = carve_smem(smem_raw, kTnStages, kStagingBytes, tn_diag_bytes(kEpi), kStageBytes, tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (kEpi == 1)
         for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
@@ -430,19 +439,19 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
         }
     } else {
-        const int q = warp & 3;          // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp drains
         int acc = 0;
-        uint32_t acc_phase = 0;
+        uint32_t acc_phase = 0, skip_phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
             const int m0 = (tile / p.n_tiles) * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
-            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, warp, lane, m0, n_out0, acc, acc_phase, tmem_base))) break;
+            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
+                                                    skip_phase)))
+                break;
             tc_fence_before();
             mbar_arrive(s.tmem_empty[acc]);
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
         }
-        if (kEpi == 0 && lane == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_all();
     }
     epilogue_exit(s, warp, tmem_base, p.hdr);
 }
@@ -459,14 +468,18 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 // leader's `tmem_empty` barriers.
 constexpr int kPairStages = 4;
 constexpr int kPairStageBytes = kABytes + kBBytes / 2;
-constexpr size_t kPairSmemBytes = (size_t)kPairStages * kPairStageBytes + kStagingBytes + kMaxDiag * 4 + 1024 + 256;
+constexpr size_t pair_smem_bytes(int epi) {
+    return (size_t)kPairStages * kPairStageBytes + kStagingBytes + tn_skip_bytes(epi) + tn_diag_bytes(epi) + 1024 + 256;
+}
 
 template <int kEpi, bool kSplitW>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTnThreads, 1)
 gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
-                       const __grid_constant__ CUtensorMap tmOut, TnParams p) {
+                       const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmSkip,
+                       TnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, kPairStages, kStagingBytes, kMaxDiag * 4, kPairStageBytes);
+    const Smem s = carve_smem(smem_raw, kPairStages, kStagingBytes, tn_diag_bytes(kEpi), kPairStageBytes,
+                              tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     if (kEpi == 1)
@@ -481,6 +494,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             mbar_init(s.tmem_full[i], 1);
             mbar_init(s.tmem_empty[i], 2 * 32 * kTnEpiWarps);
         }
+        for (int i = 0; i < 2 * kTnEpiWarps; ++i) mbar_init(s.skip_full[i], 1);
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -566,16 +580,18 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     } else {
         const uint32_t leader_empty[2] = {map_to_cta(s.tmem_empty[0], 0), map_to_cta(s.tmem_empty[1], 0)};
         int acc = 0;
-        uint32_t acc_phase = 0;
+        uint32_t acc_phase = 0, skip_phase = 0;
         bool ok = true;
         for (int tile = pair; tile < total && ok; tile += npairs) {
             const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
-            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, warp, lane, m0, n_out0, acc, acc_phase, tmem_base))) break;
+            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
+                                                    skip_phase)))
+                break;
             tc_fence_before();
             mbar_arrive_cluster(leader_empty[acc]);
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
         }
-        if (kEpi == 0 && lane == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_all();
     }
     // nobody leaves (or frees tensor memory) while the other CTA may still signal or compute
     tc_fence_before();
@@ -710,7 +726,7 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 // ---------------------------------------------------------------------------------------------
 // Row-major bf16 matrix [rows, cols] (cols contiguous), boxes of box_cols x box_rows, 128-byte swizzle.
 static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_cols,
-                     uint32_t box_rows, bool f32 = false) {
+                     uint32_t box_rows, bool f32 = false, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     PFN_cuTensorMapEncodeTiled fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
@@ -718,7 +734,7 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -779,56 +795,54 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     using namespace tc;
     const int out_cols = g.split_w ? BN / 2 : BN;
     const int n_tiles = g.N_out / out_cols;
-    CUtensorMap ma, mw, mo;
+    const int epi = g.store_f32 ? 0 : 1;
+    if (epi == 1 && (g.split_w || !g.diag || !g.skip)) return SSM_ERR_SHAPE;
+    CUtensorMap ma, mw, mo, ms;
     if (!make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, BK, BM)) return SSM_ERR_CUDA;
-    if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN)) return SSM_ERR_CUDA;
     if (g.store_f32) {   // fp32 result, stored by the TMA unit in boxes of 32 rows x 32 columns
         if (!make_map(&mo, g.out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, true)) return SSM_ERR_CUDA;
-    } else {
-        mo = ma;         // unused by the bf16 epilogue
+        ms = mo;         // unused
+    } else {             // bf16 result and skip operand: 32 x 32 boxes, 64-byte rows
+        if (!make_map(&mo, g.out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B)) return SSM_ERR_CUDA;
+        if (!make_map(&ms, g.skip, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B)) return SSM_ERR_CUDA;
     }
-    TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.out, g.diag, (const __nv_bfloat16*)g.skip,
-               (const __nv_bfloat16*)g.add, g.hdr, (const char*)g.A, g.K * 2};
+    TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.diag, g.hdr, (const char*)g.A, g.K * 2};
     const int m_tiles = (g.M + BM - 1) / BM;
     const int pair_tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * n_tiles;
-    // CTA pairs pay off where the main loop is the bottleneck (fp32 results, stored by TMA); with the
-    // bf16 epilogue, whose skip loads and stores go through the load/store units, the single-CTA
-    // kernel measured faster (0.193 vs 0.208 ms at M = 262144, N = K = 512).
-    if (g.store_f32 && pair_tiles >= sm_count() / 2) {   // enough 256-row tiles to give every pair one
-        CUtensorMap mwh;
-        if (!make_map(&mwh, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN / 2)) return SSM_ERR_CUDA;
+    bool ok = true;
+    if (pair_tiles >= sm_count() / 2) {   // enough 256-row tiles to give every CTA pair one
+        if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN / 2)) return SSM_ERR_CUDA;
         count_launch();
-        bool okp = true;
         // The kernel is persistent: its grid is the number of CTA pairs the device can hold at once
         // (not every SM has a partner that a cluster may use).
 #define SSM_LAUNCH_PAIR(EPI, SPLIT)                                                                        \
     do {                                                                                                   \
         auto kern = gemm_tc_tn_pair_kernel<EPI, SPLIT>;                                                    \
-        okp = set_smem(kern, kPairSmemBytes);                                                              \
-        const int pairs = okp ? resident_pairs(reinterpret_cast<const void*>(kern), kPairSmemBytes) : 0;   \
-        okp = okp && pairs > 0;                                                                            \
-        if (okp) kern<<<2 * min(pairs, pair_tiles), kTnThreads, kPairSmemBytes, st>>>(ma, mwh, mo, p);     \
+        constexpr size_t smem = pair_smem_bytes(EPI);                                                      \
+        ok = set_smem(kern, smem);                                                                         \
+        const int pairs = ok ? resident_pairs(reinterpret_cast<const void*>(kern), smem) : 0;              \
+        ok = ok && pairs > 0;                                                                              \
+        if (ok) kern<<<2 * min(pairs, pair_tiles), kTnThreads, smem, st>>>(ma, mw, mo, ms, p);             \
     } while (0)
-        if (g.split_w) SSM_LAUNCH_PAIR(0, true);
+        if (epi == 1) SSM_LAUNCH_PAIR(1, false);
+        else if (g.split_w) SSM_LAUNCH_PAIR(0, true);
         else SSM_LAUNCH_PAIR(0, false);
 #undef SSM_LAUNCH_PAIR
-        return okp ? SSM_OK : SSM_ERR_CUDA;
+        return ok ? SSM_OK : SSM_ERR_CUDA;
     }
+    if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN)) return SSM_ERR_CUDA;
     const int grid = min(sm_count(), m_tiles * n_tiles);
     count_launch();
-    bool ok;
-    if (g.store_f32) {
-        if (g.split_w) {
-            ok = set_smem(gemm_tc_tn_kernel<0, true>, kTnSmemBytes);
-            gemm_tc_tn_kernel<0, true><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, mo, p);
-        } else {
-            ok = set_smem(gemm_tc_tn_kernel<0, false>, kTnSmemBytes);
-            gemm_tc_tn_kernel<0, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, mo, p);
-        }
-    } else {
-        ok = set_smem(gemm_tc_tn_kernel<1, false>, kTnSmemBytes);
-        gemm_tc_tn_kernel<1, false><<<grid, kTnThreads, kTnSmemBytes, st>>>(ma, mw, mo, p);
-    }
+#define SSM_LAUNCH_TN(EPI, SPLIT)                                                                          \
+    do {                                                                                                   \
+        auto kern = gemm_tc_tn_kernel<EPI, SPLIT>;                                                         \
+        ok = set_smem(kern, tn_smem_bytes(EPI));                                                           \
+        if (ok) kern<<<grid, kTnThreads, tn_smem_bytes(EPI), st>>>(ma, mw, mo, ms, p);                     \
+    } while (0)
+    if (epi == 1) SSM_LAUNCH_TN(1, false);
+    else if (g.split_w) SSM_LAUNCH_TN(0, true);
+    else SSM_LAUNCH_TN(0, false);
+#undef SSM_LAUNCH_TN
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
 

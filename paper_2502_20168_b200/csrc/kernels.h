@@ -85,7 +85,7 @@ struct GemmTcTN {
     bool split_w;
     bool store_f32;                      // true: out fp32 [M, N_out]; false: out bf16 with the epilogue below
     void* out;
-    const float* diag; const void* skip; const void* add;   // out = acc + diag[n] * skip[m, n] (+ add[m, n])
+    const float* diag; const void* skip;   // bf16 result: out = acc + diag[n] * skip[m, n]
     WsHeader* hdr;
 };
 bool tc_tn_supported(int M, int N_out, int K, bool split_w);
