@@ -52,12 +52,12 @@ STAGE_MODEL = {
 NCU_TRAFFIC_PER_TIMESTEP = {
     "scan_fwd": 1021.7e6 / 262144,
     "scan_bwd": 1579.9e6 / 262144,
-    "gemm_Bu": None,
-    "gemm_gx": None,
-    "gemm_y": 781.7e6 / 262144,
-    "gemm_du": 781.7e6 / 262144,
-    "gemm_gBbar": 811.8e6 / 262144,
-    "gemm_gC": 811.8e6 / 262144,
+    "gemm_Bu": 763.6e6 / 262144,
+    "gemm_gx": 763.6e6 / 262144,
+    "gemm_y": 793.0e6 / 262144,
+    "gemm_du": 793.0e6 / 262144,
+    "gemm_gBbar": 813.4e6 / 262144,
+    "gemm_gC": 813.4e6 / 262144,
 }
 
 
