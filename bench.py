@@ -298,23 +298,74 @@ def main():
     h2d = sum(t.numel() * t.element_size() for t in host_in.values())
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
 
-    def e2e_step():
-        for k, t in host_in.items():
-            getattr(buf, k).copy_(t, non_blocking=True)
-        step()
-        for k, t in host_out.items():
-            t.copy_(getattr(buf, k), non_blocking=True)
-
     e2e_steps = max(1, min(args.steps, 10))
-    e2e_step()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
+    if stacked:
+        def e2e_step():
+            for k, t in host_in.items():
+                getattr(buf, k).copy_(t, non_blocking=True)
+            step()
+            for k, t in host_out.items():
+                t.copy_(getattr(buf, k), non_blocking=True)
+
         e2e_step()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e_mode = "copies and compute in sequence on one stream"
+    else:
+        # Every step still moves all of its inputs in and all of its results out; the copies of
+        # neighbouring steps overlap the compute through two sets of input / output buffers and three
+        # streams (in, compute, out), as a training loop that streams batches would do.
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        dev_in = [{k: torch.empty_like(getattr(buf, k)) for k in host_in} for _ in range(2)]
+        dev_out = [{k: torch.empty_like(getattr(buf, k)) for k in host_out} for _ in range(2)]
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        in_done, comp_done, out_done = {}, {}, {}
+
+        def pipeline(n):
+            first, last = ev(), ev()
+            first.record(stream)
+            s_in.wait_event(first)
+            for i in range(n):
+                j = i % 2
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(comp_done[i - 2])      # step i-2 has consumed this input set
+                    for k, t in host_in.items():
+                        dev_in[j][k].copy_(t, non_blocking=True)
+                    in_done[i] = ev()
+                    in_done[i].record(s_in)
+                stream.wait_event(in_done[i])
+                if i >= 2:
+                    stream.wait_event(out_done[i - 2])         # step i-2's results have left this output set
+                for k, t in dev_in[j].items():
+                    setattr(buf, k, t)
+                for k, t in dev_out[j].items():
+                    setattr(buf, k, t)
+                step()
+                comp_done[i] = ev()
+                comp_done[i].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(comp_done[i])
+                    for k, t in host_out.items():
+                        t.copy_(dev_out[j][k], non_blocking=True)
+                    out_done[i] = ev()
+                    out_done[i].record(s_out)
+            stream.wait_event(out_done[n - 1])
+            last.record(stream)
+            return first, last
+
+        pipeline(2)
+        barrier()
+        e0, e1 = pipeline(e2e_steps)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e_mode = "double-buffered: H2D, compute and D2H of neighbouring steps overlap on three streams"
 
     times = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
     if world > 1:
@@ -348,7 +399,7 @@ def main():
                        "p_done": w.p_done, "n_layers": w.n_layers, "l2": "inputs larger than L2 (no flush)"
                        if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}"},
             "e2e": {"value": total_ts * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "mode": e2e_mode},
             "gpu_launches": int(launches),
             "clocks": clocks,
             "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
