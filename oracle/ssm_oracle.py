@@ -217,6 +217,35 @@ def gelu_grad(v):
     return 0.5 * (1.0 + _erf(v / np.sqrt(2.0))) + v * np.exp(-0.5 * v * v) / np.sqrt(2.0 * np.pi)
 
 
+# --------------------------------------------------------------------------
+# Half-GLU gate of the S5 sequence layer (Appendix "S5 Sequence Layer")
+# --------------------------------------------------------------------------
+def half_glu_fwd(W, v):
+    """x1 = GELU(v);  out = v * sigmoid(W^T x1), row by row (v: [..., H], W: [H, H]).
+
+    Appendix "S5 Sequence Layer": the gate's argument is the linear layer W applied to the
+    GELU of the gate's input, (W^T x1)_j = sum_i W[i, j] x1_i; the input itself is what gets
+    gated.  No bias (the appendix names only the weights W)."""
+    v = np.asarray(v, F64)
+    W = np.asarray(W, F64)
+    z = gelu(v) @ W
+    return v / (1.0 + np.exp(-z))
+
+
+def half_glu_bwd(W, v, gout):
+    """Gradients of L = sum(gout * out) for out = half_glu_fwd(W, v): (gv, dW)."""
+    v = np.asarray(v, F64)
+    W = np.asarray(W, F64)
+    gout = np.asarray(gout, F64)
+    x1 = gelu(v)
+    s = 1.0 / (1.0 + np.exp(-(x1 @ W)))
+    gz = gout * v * s * (1.0 - s)
+    gv = gout * s + (gz @ W.T) * gelu_grad(v)
+    H = v.shape[-1]
+    dW = x1.reshape(-1, H).T @ gz.reshape(-1, H)
+    return gv, dW
+
+
 def layernorm_fwd(z, weight, bias):
     mu = z.mean(axis=-1, keepdims=True)
     var = ((z - mu) ** 2).mean(axis=-1, keepdims=True)
