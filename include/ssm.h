@@ -177,6 +177,21 @@ int ssm_step(const ssm_shape* shape, const float* D /*[H]*/, const void* u /*[B,
              ssm_c64* x_next /*[B,P] out*/, void* y /*[B,H] io, out*/, void* ws, size_t ws_bytes,
              void* stream);
 
+/* ---- half-GLU gate of the S5 sequence layer: Appendix "S5 Sequence Layer" -----------
+ * The gate the paper's block applies to the SSM output v:
+ *   x1 = GELU(v);   out[m,j] = v[m,j] * sigmoid( sum_i W[i,j] x1[m,i] )      (exact erf GELU, no bias)
+ * over the B*T rows m of [B,T,H] tensors in io_dtype; W is [H,H] fp32, row i = input feature.
+ * ssm_glu_fwd leaves GELU(v) and the gate's argument in ws; ssm_glu_bwd needs that workspace
+ * and returns, for L = sum(gout * out), gv[B,T,H] (io_dtype) and dW[H,H] (overwritten).
+ * A block of the paper is ssm_layer_fwd followed by ssm_glu_fwd on its y (and the reverse order
+ * backward, the gate's gv being the layer's gy).  Uses shape->B, T, H. */
+size_t ssm_glu_workspace_bytes(const ssm_shape* shape);
+int ssm_glu_fwd(const ssm_shape* shape, const float* W /*[H,H]*/, const void* v /*[B,T,H] io*/,
+                void* out /*[B,T,H] io*/, void* ws, size_t ws_bytes, void* stream);
+int ssm_glu_bwd(const ssm_shape* shape, const float* W, const void* v, const void* gout /*[B,T,H] io*/,
+                void* ws, size_t ws_bytes, void* gv /*[B,T,H] io, out*/, float* dW /*[H,H] out*/,
+                void* stream);
+
 /* ---- stacked sequence model --------------------------------------------------------
  * n_layers layers of   v = SSM_l(u_l);  u_{l+1} = LayerNorm(u_l + GELU(v)) * ln_weight + ln_bias
  * (exact erf GELU, LayerNorm over the H features with eps 1e-5), the same done flags in every

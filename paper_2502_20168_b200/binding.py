@@ -28,6 +28,7 @@ EXPORTS = (
     "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static",
     "ssm_stack_workspace_bytes", "ssm_stack_fwd", "ssm_stack_bwd",
     "ssm_step_workspace_bytes", "ssm_step_prepare", "ssm_step",
+    "ssm_glu_workspace_bytes", "ssm_glu_fwd", "ssm_glu_bwd",
 )
 SSM_ERR_TOO_LARGE = -8
 SSM_STATIC_SCRATCH_BYTES = 8 << 20
@@ -95,6 +96,12 @@ def _load() -> ctypes.CDLL:
     lib.ssm_step_prepare.argtypes = [S] + [P] * 5 + [c_size_t, P]
     lib.ssm_step.restype = c_int
     lib.ssm_step.argtypes = [S] + [P] * 7 + [c_size_t, P]
+    lib.ssm_glu_workspace_bytes.restype = c_size_t
+    lib.ssm_glu_workspace_bytes.argtypes = [S]
+    lib.ssm_glu_fwd.restype = c_int
+    lib.ssm_glu_fwd.argtypes = [S] + [P] * 4 + [c_size_t, P]
+    lib.ssm_glu_bwd.restype = c_int
+    lib.ssm_glu_bwd.argtypes = [S] + [P] * 4 + [c_size_t] + [P] * 3
     lib.ssm_launch_count.restype = ctypes.c_longlong
     lib.ssm_launch_count.argtypes = []
     lib.ssm_profile_begin.restype = c_int
@@ -216,6 +223,20 @@ def ssm_step_prepare(shape, Lambda, Delta, Bc, Cc, ws, stream=None) -> None:
 def ssm_step(shape, D, u, done, x_prev, x_next, y, ws, stream=None) -> None:
     _ok(_lib.ssm_step(byref(shape), _ptr(D), _ptr(u), _ptr(done), _ptr(x_prev), _ptr(x_next), _ptr(y), _ptr(ws),
                       _nbytes(ws), _stream(stream)), "ssm_step")
+
+
+def ssm_glu_workspace_bytes(shape) -> int:
+    return int(_lib.ssm_glu_workspace_bytes(byref(shape)))
+
+
+def ssm_glu_fwd(shape, W, v, out, ws, stream=None) -> None:
+    _ok(_lib.ssm_glu_fwd(byref(shape), _ptr(W), _ptr(v), _ptr(out), _ptr(ws), _nbytes(ws), _stream(stream)),
+        "ssm_glu_fwd")
+
+
+def ssm_glu_bwd(shape, W, v, gout, ws, gv, dW, stream=None) -> None:
+    _ok(_lib.ssm_glu_bwd(byref(shape), _ptr(W), _ptr(v), _ptr(gout), _ptr(ws), _nbytes(ws), _ptr(gv), _ptr(dW),
+                         _stream(stream)), "ssm_glu_bwd")
 
 
 def _struct_array(cls, dicts):

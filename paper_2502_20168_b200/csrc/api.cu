@@ -299,6 +299,137 @@ SSM_API int ssm_step(const ssm_shape* shape, const float* D, const void* u, cons
     return layer_fwd_run(s, p, D, u, done, x_prev, y, x_next, ws, at<WsHeader>(ws, p.hdr), (cudaStream_t)stream);
 }
 
+// ---- half-GLU gate -----------------------------------------------------------------------
+namespace {
+
+struct GluPlan {
+    bool tc;
+    int splits;
+    size_t hdr, Wt, Wn, x1, z, gz, gx1, part, total;
+};
+
+GluPlan plan_glu(const ssm_shape& s) {
+    GluPlan p{};
+    size_t off = 0;
+    const size_t M = (size_t)s.B * s.T, HH = (size_t)s.H * s.H;
+    p.tc = s.io_dtype == SSM_BF16 && tc_tn_supported((int)M, s.H, s.H, true) && tc_nt_supported(s.H, s.H);
+    p.splits = p.tc ? tc_nt_splits((int)M, s.H, s.H) : gemm_nt_splits((int)M);
+    p.hdr = take(off, sizeof(WsHeader));
+    p.Wt = take(off, p.tc ? 2 * HH * 2 : HH * 4);   // tc: hi/lo stacked bf16 [2H, H]; else W^T fp32
+    p.Wn = take(off, p.tc ? 2 * HH * 2 : 0);
+    p.x1 = take(off, M * s.H * 4);                  // GELU(v): fp32, or two bf16 planes
+    p.z = take(off, M * s.H * 4);                   // the gate's argument
+    p.gz = take(off, M * s.H * 4);                  // fp32, or two bf16 planes
+    p.gx1 = take(off, M * s.H * 4);
+    p.part = take(off, (size_t)2 * p.splits * HH * 4);
+    p.total = off;
+    return p;
+}
+
+}  // namespace
+
+SSM_API size_t ssm_glu_workspace_bytes(const ssm_shape* shape) {
+    if (check_shape(shape) != SSM_OK) return 0;
+    return plan_glu(*shape).total;
+}
+
+SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, void* out, void* ws, size_t ws_bytes,
+                        void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!W || !v || !out) return SSM_ERR_NULL;
+    if (misaligned(W) || misaligned(v) || misaligned(out)) return SSM_ERR_ALIGN;
+    const ssm_shape& s = *shape;
+    const GluPlan p = plan_glu(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf16 = s.io_dtype == SSM_BF16;
+    const int M = s.B * s.T;
+    const size_t n = (size_t)M * s.H;
+    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
+    {
+        StageTimer tm("glu_pack_gelu", st);
+        launch_glu_pack(s.H, W, p.tc ? at<void>(ws, p.Wt) : nullptr, p.tc ? at<void>(ws, p.Wn) : nullptr,
+                        p.tc ? nullptr : at<float>(ws, p.Wt), st);
+        launch_glu_gelu(bf16, p.tc, n, v, at<void>(ws, p.x1), st);
+    }
+    {   // z[m, j] = sum_i x1[m, i] W[i, j]
+        StageTimer tm("glu_gemm_z", st);
+        if (p.tc) {
+            // x1 = hi + lo: one product per plane (the second one lands in the buffer g_x1 uses later);
+            // the gate's argument needs both, a single bf16 rounding of x1 there costs 2e-2 on dW
+            GemmTcTN g{at<void>(ws, p.x1), at<void>(ws, p.Wt), M, s.H, s.H, true, true, at<void>(ws, p.z), nullptr, nullptr, hdr};
+            if (int rc = launch_gemm_tc_tn(g, st)) return rc;
+            g.A = at<void>(ws, p.x1 + n * 2);
+            g.out = at<void>(ws, p.gx1);
+            if (int rc = launch_gemm_tc_tn(g, st)) return rc;
+        } else {
+            GemmTN g{at<void>(ws, p.x1), false, s.H, at<void>(ws, p.Wt), false, s.H, M, s.H, s.H, Epi::StoreF32,
+                     at<void>(ws, p.z), false, nullptr, nullptr, nullptr};
+            launch_gemm_tn(g, st);
+        }
+    }
+    {
+        StageTimer tm("glu_out", st);
+        launch_glu_out(bf16, n, v, at<float>(ws, p.z), p.tc ? at<float>(ws, p.gx1) : nullptr, out, st);
+    }
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
+SSM_API int ssm_glu_bwd(const ssm_shape* shape, const float* W, const void* v, const void* gout, void* ws,
+                        size_t ws_bytes, void* gv, float* dW, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!W || !v || !gout || !gv || !dW) return SSM_ERR_NULL;
+    if (misaligned(W) || misaligned(v) || misaligned(gout) || misaligned(gv) || misaligned(dW)) return SSM_ERR_ALIGN;
+    const ssm_shape& s = *shape;
+    const GluPlan p = plan_glu(s);
+    if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf16 = s.io_dtype == SSM_BF16;
+    const int M = s.B * s.T;
+    const size_t n = (size_t)M * s.H, HH = (size_t)s.H * s.H;
+    WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    {
+        StageTimer tm("glu_gz", st);
+        launch_glu_gz(bf16, p.tc, n, v, gout, at<float>(ws, p.z), at<void>(ws, p.gz), st);
+    }
+    {   // g_x1[m, i] = sum_j gz[m, j] W[i, j]
+        StageTimer tm("glu_gemm_gx1", st);
+        if (p.tc) {
+            GemmTcTN g{at<void>(ws, p.gz), at<void>(ws, p.Wn), M, s.H, s.H, true, true, at<void>(ws, p.gx1), nullptr, nullptr, hdr};
+            if (int rc = launch_gemm_tc_tn(g, st)) return rc;
+        } else {
+            GemmTN g{at<void>(ws, p.gz), false, s.H, W, false, s.H, M, s.H, s.H, Epi::StoreF32,
+                     at<void>(ws, p.gx1), false, nullptr, nullptr, nullptr};
+            launch_gemm_tn(g, st);
+        }
+    }
+    {   // dW[i, j] = sum_m x1[m, i] gz[m, j]
+        StageTimer tm("glu_gemm_dW", st);
+        if (p.tc) {
+            // (x1_hi + x1_lo)^T (gz_hi + gz_lo) as two products, one per plane of x1
+            GemmTcNT g{at<void>(ws, p.x1), s.H, at<void>(ws, p.gz), at<void>(ws, p.gz + n * 2), s.H, M, p.splits,
+                       at<float>(ws, p.part), hdr};
+            if (int rc = launch_gemm_tc_nt(g, st)) return rc;
+            g.A = at<void>(ws, p.x1 + n * 2);
+            g.part = at<float>(ws, p.part) + (size_t)p.splits * HH;
+            if (int rc = launch_gemm_tc_nt(g, st)) return rc;
+            launch_glu_reduce(at<float>(ws, p.part), 2 * p.splits, HH, dW, st);
+        } else {
+            GemmNT g{at<void>(ws, p.x1), false, s.H, at<void>(ws, p.gz), false, s.H, M, p.splits, at<float>(ws, p.part)};
+            launch_gemm_nt(g, st);
+            launch_glu_reduce(at<float>(ws, p.part), p.splits, HH, dW, st);
+        }
+    }
+    {
+        StageTimer tm("glu_gv", st);
+        launch_glu_gv(bf16, n, v, gout, at<float>(ws, p.z), at<float>(ws, p.gx1), gv, st);
+    }
+    SSM_RETURN_IF_CUDA_ERROR();
+    return SSM_OK;
+}
+
 // Launch sequence of one layer's backward pass.  du_add (io dtype, may be NULL) is added to du
 // before it is rounded (the residual branch of a stacked model).
 static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,

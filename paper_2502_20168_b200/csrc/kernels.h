@@ -109,6 +109,21 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st);
 
+// glu.cu: what surrounds the GEMMs of the half-GLU gate out = v * sigmoid(GELU(v) W).
+// Wt_split / Wn_split (tensor-core path, may be NULL): hi/lo stacked bf16 operands [2H, H] for
+// z = x1 W and g_x1 = gz W^T;  Wt_f32 (CUDA-core path, may be NULL): W transposed.
+void launch_glu_pack(int H, const float* W, void* Wt_split, void* Wn_split, float* Wt_f32, cudaStream_t st);
+// x1 = GELU(v); planes: two bf16 planes (hi, lo) n elements apart, else fp32
+void launch_glu_gelu(bool io_bf16, bool planes, size_t n, const void* v, void* x1, cudaStream_t st);
+// out = v * sigmoid(z); if z2 is given, z += z2 first (stored back)
+void launch_glu_out(bool io_bf16, size_t n, const void* v, float* z, const float* z2, void* out, cudaStream_t st);
+// gz = gout * v * s (1 - s), s = sigmoid(z); planes: two bf16 planes (hi, lo) n elements apart, else fp32
+void launch_glu_gz(bool io_bf16, bool planes, size_t n, const void* v, const void* gout, const float* z, void* gz,
+                   cudaStream_t st);
+void launch_glu_gv(bool io_bf16, size_t n, const void* v, const void* gout, const float* z, const float* gx1, void* gv,
+                   cudaStream_t st);
+void launch_glu_reduce(const float* part, int splits, size_t n, float* out, cudaStream_t st);
+
 // stack.cu: out = LayerNorm(u + GELU(v)) * w + b per row of H features, and its backward
 // (gzr = round(LN'(g)), gv = round(gz * GELU'(v)), dw, db).  tmp: stack_tmp_floats(M, H) floats.
 size_t stack_tmp_floats(int M, int H);

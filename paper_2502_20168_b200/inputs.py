@@ -125,6 +125,17 @@ def draw_layer(w: Workload, *, with_x0: bool = False, with_gxT: bool = False) ->
     return out
 
 
+def draw_glu(w: Workload) -> dict:
+    """Inputs of the half-GLU gate at a workload's B, T, H: weights W ~ N(0, 1/H) (fp32), the gate's
+    input v ~ N(0, 1) (it stands in for the SSM output) and the output gradient gout ~ N(0, 1),
+    both in the workload's I/O precision.  Its own stream of numbers (seed + 7919)."""
+    rng = np.random.default_rng(w.seed + 7919)
+    W = rng.normal(0.0, 1.0 / math.sqrt(w.H), size=(w.H, w.H)).astype(np.float32)
+    v = cast_io(rng.normal(size=(w.B, w.T, w.H)), w.io_dtype)
+    gout = cast_io(rng.normal(size=(w.B, w.T, w.H)), w.io_dtype)
+    return {"W": W, "v": v, "gout": gout}
+
+
 def small_variant(w: Workload, **changes) -> Workload:
     """Same distributions, other sizes (used by edge-case tests)."""
     return replace(w, **changes)
