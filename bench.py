@@ -221,6 +221,41 @@ def time_step_mode(w, torch, sb, n_traj=4096, steps=50):
             "launches_per_step": (sb.ssm_launch_count() - n0) / steps}
 
 
+def time_half_glu(w, torch, sb, steps=10):
+    """The half-GLU gate (ssm_glu_fwd + ssm_glu_bwd) on the workload's [B, T, H] activations,
+    device-resident, per-stage CUDA events.  Reported beside the headline, not part of it."""
+    io = torch.bfloat16 if w.io_dtype == "bf16" else torch.float32
+    shape = sb.make_shape(w.B, w.T, w.H, w.P, w.io_dtype)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(w.seed + 1)
+    W = (torch.randn((w.H, w.H), device="cuda", generator=g) / w.H ** 0.5).contiguous()
+    v = torch.randn((w.B, w.T, w.H), device="cuda", generator=g).to(io)
+    gout = torch.randn((w.B, w.T, w.H), device="cuda", generator=g).to(io)
+    out, gv, dW = torch.empty_like(v), torch.empty_like(v), torch.empty_like(W)
+    ws = sb.alloc_workspace(sb.ssm_glu_workspace_bytes(shape))
+    stream = torch.cuda.current_stream()
+
+    def step():
+        sb.ssm_glu_fwd(shape, W, v, out, ws, stream)
+        sb.ssm_glu_bwd(shape, W, v, gout, ws, gv, dW, stream)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    sb.ssm_profile_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    stages = sb.ssm_profile_end()
+    sb.ssm_check(ws)
+    ms = e0.elapsed_time(e1) / steps
+    return {"ms_per_step": ms, "timesteps_per_sec": w.timesteps / (ms * 1e-3),
+            "stage_ms_per_step": {k: round(v_[1] / steps, 4) for k, v_ in stages.items()}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -411,6 +446,9 @@ def main():
         }
         if world == 1 and not stacked:
             line["step_mode"] = time_step_mode(w, torch, sb)
+            del buf
+            torch.cuda.empty_cache()
+            line["half_glu"] = time_half_glu(w, torch, sb)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, max(1, 262144 // w.T)))))
         print(json.dumps(line))

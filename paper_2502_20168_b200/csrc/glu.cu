@@ -17,7 +17,7 @@ __device__ __forceinline__ float sigmoid_f(float z) { return 1.f / (1.f + expf(-
 constexpr int kThreads = 256;
 inline int blocks_for(size_t n) {
     const size_t b = (n + kThreads - 1) / kThreads;
-    return (int)(b < 148 * 16 ? b : 148 * 16);
+    return (int)(b < 148 * 32 ? b : 148 * 32);
 }
 
 // Weight operands.  tc: hi/lo bf16 halves stacked as the TN kernel wants them (rows
@@ -43,20 +43,68 @@ __global__ void glu_pack_kernel(int H, const float* __restrict__ W, __nv_bfloat1
     }
 }
 
-// x1 = GELU(v): fp32, or two bf16 planes hi / lo n elements apart (hi alone feeds the gate's GEMM,
-// hi + lo the weight-gradient sum over all rows, where a single bf16 rounding is not enough)
+// The elementwise passes work on groups of 8 consecutive elements (H is a multiple of 8): 16- or
+// 32-byte accesses per array and thread.
+struct F8 {
+    float x[8];
+};
+template <typename T> __device__ __forceinline__ F8 load8(const T* p);
+template <> __device__ __forceinline__ F8 load8<float>(const float* p) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p)), b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    return F8{{a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w}};
+}
+template <> __device__ __forceinline__ F8 load8<__nv_bfloat16>(const __nv_bfloat16* p) {
+    const uint4 r = __ldcs(reinterpret_cast<const uint4*>(p));
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&r);
+    F8 o;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h[i]);
+        o.x[2 * i] = f.x;
+        o.x[2 * i + 1] = f.y;
+    }
+    return o;
+}
+template <typename T> __device__ __forceinline__ void store8(T* p, const F8& v);
+template <> __device__ __forceinline__ void store8<float>(float* p, const F8& v) {
+    reinterpret_cast<float4*>(p)[0] = make_float4(v.x[0], v.x[1], v.x[2], v.x[3]);
+    reinterpret_cast<float4*>(p)[1] = make_float4(v.x[4], v.x[5], v.x[6], v.x[7]);
+}
+template <> __device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16* p, const F8& v) {
+    uint4 r;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(v.x[2 * i], v.x[2 * i + 1]);
+    *reinterpret_cast<uint4*>(p) = r;
+}
+// hi = bf16(v), lo = bf16(v - hi) into two planes `plane` elements apart
+__device__ __forceinline__ void store8_planes(__nv_bfloat16* p, size_t plane, const F8& v) {
+    F8 hi_f, lo;
+    uint4 r;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        h[i] = __floats2bfloat162_rn(v.x[2 * i], v.x[2 * i + 1]);
+        const float2 f = __bfloat1622float2(h[i]);
+        hi_f.x[2 * i] = f.x;
+        hi_f.x[2 * i + 1] = f.y;
+    }
+    *reinterpret_cast<uint4*>(p) = r;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) lo.x[i] = v.x[i] - hi_f.x[i];
+    store8<__nv_bfloat16>(p + plane, lo);
+}
+
+// x1 = GELU(v): fp32, or two bf16 planes hi / lo n elements apart (hi alone would do for a product
+// that tolerates one bf16 rounding; the gate's argument and the weight gradient do not)
 template <typename IO, bool kPlanes>
 __global__ void glu_gelu_kernel(size_t n, const IO* __restrict__ v, void* __restrict__ x1) {
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        const float g = gelu_f(to_f32<IO>(v[e]));
-        if (kPlanes) {
-            __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(x1);
-            const __nv_bfloat16 hi = __float2bfloat16_rn(g);
-            p[e] = hi;
-            p[n + e] = __float2bfloat16_rn(g - __bfloat162float(hi));
-        } else {
-            reinterpret_cast<float*>(x1)[e] = g;
-        }
+    for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; e < n; e += (size_t)gridDim.x * blockDim.x * 8) {
+        F8 a = load8<IO>(v + e);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a.x[i] = gelu_f(a.x[i]);
+        if (kPlanes) store8_planes(reinterpret_cast<__nv_bfloat16*>(x1) + e, n, a);
+        else store8<float>(reinterpret_cast<float*>(x1) + e, a);
     }
 }
 
@@ -64,13 +112,19 @@ __global__ void glu_gelu_kernel(size_t n, const IO* __restrict__ v, void* __rest
 template <typename IO>
 __global__ void glu_out_kernel(size_t n, const IO* __restrict__ v, float* __restrict__ z, const float* __restrict__ z2,
                                IO* __restrict__ out) {
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        float zz = z[e];
+    for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; e < n; e += (size_t)gridDim.x * blockDim.x * 8) {
+        const F8 a = load8<IO>(v + e);
+        F8 zz = load8<float>(z + e);
         if (z2) {
-            zz += z2[e];
-            z[e] = zz;
+            const F8 z2v = load8<float>(z2 + e);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) zz.x[i] += z2v.x[i];
+            store8<float>(z + e, zz);
         }
-        out[e] = from_f32<IO>(to_f32<IO>(v[e]) * sigmoid_f(zz));
+        F8 o;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o.x[i] = a.x[i] * sigmoid_f(zz.x[i]);
+        store8<IO>(out + e, o);
     }
 }
 
@@ -78,26 +132,28 @@ __global__ void glu_out_kernel(size_t n, const IO* __restrict__ v, float* __rest
 template <typename IO, bool kPlanes>
 __global__ void glu_gz_kernel(size_t n, const IO* __restrict__ v, const IO* __restrict__ gout,
                               const float* __restrict__ z, void* __restrict__ gz, size_t plane) {
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        const float s = sigmoid_f(z[e]);
-        const float g = to_f32<IO>(gout[e]) * to_f32<IO>(v[e]) * s * (1.f - s);
-        if (kPlanes) {
-            __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(gz);
-            const __nv_bfloat16 hi = __float2bfloat16_rn(g);
-            p[e] = hi;
-            p[plane + e] = __float2bfloat16_rn(g - __bfloat162float(hi));
-        } else {
-            reinterpret_cast<float*>(gz)[e] = g;
+    for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; e < n; e += (size_t)gridDim.x * blockDim.x * 8) {
+        const F8 a = load8<IO>(v + e), g = load8<IO>(gout + e), zz = load8<float>(z + e);
+        F8 o;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float s = sigmoid_f(zz.x[i]);
+            o.x[i] = g.x[i] * a.x[i] * s * (1.f - s);
         }
+        if (kPlanes) store8_planes(reinterpret_cast<__nv_bfloat16*>(gz) + e, plane, o);
+        else store8<float>(reinterpret_cast<float*>(gz) + e, o);
     }
 }
 
 template <typename IO>
 __global__ void glu_gv_kernel(size_t n, const IO* __restrict__ v, const IO* __restrict__ gout,
                               const float* __restrict__ z, const float* __restrict__ gx1, IO* __restrict__ gv) {
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        const float vv = to_f32<IO>(v[e]);
-        gv[e] = from_f32<IO>(to_f32<IO>(gout[e]) * sigmoid_f(z[e]) + gx1[e] * gelu_grad_f(vv));
+    for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; e < n; e += (size_t)gridDim.x * blockDim.x * 8) {
+        const F8 a = load8<IO>(v + e), g = load8<IO>(gout + e), zz = load8<float>(z + e), x = load8<float>(gx1 + e);
+        F8 o;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o.x[i] = g.x[i] * sigmoid_f(zz.x[i]) + x.x[i] * gelu_grad_f(a.x[i]);
+        store8<IO>(gv + e, o);
     }
 }
 
@@ -119,7 +175,7 @@ void launch_glu_pack(int H, const float* W, void* Wt_split, void* Wn_split, floa
 
 void launch_glu_gelu(bool io_bf16, bool planes, size_t n, const void* v, void* x1, cudaStream_t st) {
     count_launch();
-    const int b = blocks_for(n);
+    const int b = blocks_for(n / 8);
     if (io_bf16 && planes)
         glu_gelu_kernel<__nv_bfloat16, true><<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, x1);
     else if (io_bf16)
@@ -130,7 +186,7 @@ void launch_glu_gelu(bool io_bf16, bool planes, size_t n, const void* v, void* x
 
 void launch_glu_out(bool io_bf16, size_t n, const void* v, float* z, const float* z2, void* out, cudaStream_t st) {
     count_launch();
-    const int b = blocks_for(n);
+    const int b = blocks_for(n / 8);
     if (io_bf16) glu_out_kernel<<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, z, z2, (__nv_bfloat16*)out);
     else glu_out_kernel<<<b, kThreads, 0, st>>>(n, (const float*)v, z, z2, (float*)out);
 }
@@ -138,7 +194,7 @@ void launch_glu_out(bool io_bf16, size_t n, const void* v, float* z, const float
 void launch_glu_gz(bool io_bf16, bool planes, size_t n, const void* v, const void* gout, const float* z, void* gz,
                    cudaStream_t st) {
     count_launch();
-    const int b = blocks_for(n);
+    const int b = blocks_for(n / 8);
     if (io_bf16 && planes)
         glu_gz_kernel<__nv_bfloat16, true><<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, (const __nv_bfloat16*)gout, z, gz, n);
     else if (io_bf16)
@@ -150,7 +206,7 @@ void launch_glu_gz(bool io_bf16, bool planes, size_t n, const void* v, const voi
 void launch_glu_gv(bool io_bf16, size_t n, const void* v, const void* gout, const float* z, const float* gx1, void* gv,
                    cudaStream_t st) {
     count_launch();
-    const int b = blocks_for(n);
+    const int b = blocks_for(n / 8);
     if (io_bf16)
         glu_gv_kernel<<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, (const __nv_bfloat16*)gout, z, gx1, (__nv_bfloat16*)gv);
     else
