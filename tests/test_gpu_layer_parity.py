@@ -90,3 +90,28 @@ def test_forward_backward_twice_is_bitwise_repeatable_and_workspace_reusable():
     second = buf.results()
     for k in ("y", "du", "dB", "dC", "dLambda", "dDelta", "dD"):
         assert np.array_equal(first[k], second[k]), k
+
+
+def test_layer_step_replays_from_a_cuda_graph():
+    """After a warm-up call, forward + backward issue only stream work (kernels, memsets), so a
+    step can be captured once and replayed: the replay gives the results of the eager run."""
+    import torch
+    from paper_2502_20168_b200 import harness
+    for w in (I.C1, I.Workload("paper_batch", B=32, T=128, H=512, P=256, io_dtype="bf16", p_done=0.01, seed=9)):
+        d = I.draw_layer(w)
+        buf = harness.LayerBuffers(d, w.io_dtype)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            buf.forward(s); buf.backward(s)
+        torch.cuda.synchronize()
+        eager = buf.results()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            buf.forward(s); buf.backward(s)
+        for k in ("y", "du", "dLambda", "dB", "dC"):
+            getattr(buf, k).zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        sb_res = buf.results()
+        for k in ("y", "du", "dLambda", "dDelta", "dB", "dC", "dD"):
+            assert np.array_equal(eager[k], sb_res[k]), k
