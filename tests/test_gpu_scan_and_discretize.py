@@ -32,7 +32,9 @@ def _abar(rng, P):
 # when B is small; T around multiples of the tile heights; P that is not a multiple of the width
 SCAN_SHAPES = [(1, 1, 8), (2, 63, 8), (3, 64, 24), (2, 65, 40), (1, 1000, 264), (4, 517, 128),
                (2, 4100, 16), (800, 70, 256), (40, 129, 136), (600, 33, 128), (5, 256, 64), (300, 1, 128),
-               (7, 7, 32), (6, 8, 32)]
+               (7, 7, 32), (6, 8, 32),
+               # few sequences, long: narrow chains, many tiles per chain (ragged ends, P off the width)
+               (2, 5000, 128), (3, 1100, 64), (16, 1200, 256), (9, 2100, 136), (1, 1024, 64), (4, 1025, 192)]
 
 
 @pytest.mark.parametrize("B,T,P", SCAN_SHAPES)
