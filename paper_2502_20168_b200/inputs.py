@@ -49,7 +49,11 @@ C3 = Workload("c3_long_bf16", B=16, T=1024, H=512, P=256, io_dtype="bf16", p_don
 C4_TS = (64, 256, 1024, 4096, 16384)
 C4 = tuple(Workload(f"c4_sweep_T{t}_bf16", B=262144 // t, T=t, H=512, P=256,
                     io_dtype="bf16", seed=4) for t in C4_TS)
-WORKLOADS = {w.name: w for w in (C0, C1, C2, C3) + C4}
+# The paper's own training batch (32 sequences of 128 steps, hyper-parameter tables of the appendix):
+# state task (deterministic state 512, SSM state 256) and vision task (1024 / 512).
+PAPER_STATE = Workload("paper_state_batch_bf16", B=32, T=128, H=512, P=256, io_dtype="bf16", p_done=0.01, seed=5)
+PAPER_VISION = Workload("paper_vision_batch_bf16", B=32, T=128, H=1024, P=512, io_dtype="bf16", p_done=0.01, seed=6)
+WORKLOADS = {w.name: w for w in (C0, C1, C2, C3) + C4 + (PAPER_STATE, PAPER_VISION)}
 
 
 def round_to_bf16(a: np.ndarray) -> np.ndarray:

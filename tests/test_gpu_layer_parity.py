@@ -33,6 +33,12 @@ def test_c3_long_horizon_bf16():
     run(I.C3)
 
 
+def test_paper_training_batches_bf16():
+    # 32 x 128 batches at the sizes of the paper's state task (512 / 256) and vision task (1024 / 512)
+    run(I.PAPER_STATE)
+    run(I.PAPER_VISION)
+
+
 @pytest.mark.parametrize("io", ["f32", "bf16"])
 @pytest.mark.parametrize("B,T,H,P", [(3, 1, 8, 8), (2, 7, 24, 8), (5, 33, 40, 24), (2, 130, 72, 56),
                                      (1, 300, 64, 128), (9, 64, 128, 64)])
