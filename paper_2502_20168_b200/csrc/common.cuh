@@ -30,11 +30,10 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 
 // ---- workspace header -------------------------------------------------------------------
 // First 256 bytes of every workspace.  `status` is written by kernels whose bounded waits
-// give up; `ticket` hands out chunk ids in launch order.
+// give up.
 struct WsHeader {
     int status;
-    int ticket;
-    int pad[62];
+    int pad[63];
 };
 static_assert(sizeof(WsHeader) == 256, "header is one 256-byte line group");
 

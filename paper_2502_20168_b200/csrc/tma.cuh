@@ -1,5 +1,5 @@
 // Shared-memory barriers and bulk tensor copies (TMA) used by the tensor-core projections and
-// the chunked scans: PTX wrappers, bounded waits, and the host-side tensor-map encoder lookup.
+// the streaming scans: PTX wrappers, bounded waits, and the host-side tensor-map encoder lookup.
 #pragma once
 
 #include <cuda.h>
