@@ -217,8 +217,29 @@ def time_step_mode(w, torch, sb, n_traj=4096, steps=50):
     e1.record(stream)
     torch.cuda.synchronize()
     sb.ssm_check(ws)
-    return {"trajectories": n_traj, "steps": steps, "us_per_step": e0.elapsed_time(e1) * 1e3 / steps,
-            "launches_per_step": (sb.ssm_launch_count() - n0) / steps}
+    eager_us = e0.elapsed_time(e1) * 1e3 / steps
+    launches = (sb.ssm_launch_count() - n0) / steps
+    # the same rollout captured once in a CUDA graph and replayed: no host work per step
+    horizon = 15
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for t in range(horizon):
+            sb.ssm_step(shape, D, u[t], None, x, x, y, ws, side)
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 10
+    g0.record()
+    for _ in range(reps):
+        graph.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    sb.ssm_check(ws)
+    return {"trajectories": n_traj, "steps": steps, "us_per_step": eager_us, "launches_per_step": launches,
+            "graph_horizon": horizon, "graph_us_per_step": g0.elapsed_time(g1) * 1e3 / (reps * horizon)}
 
 
 def time_half_glu(w, torch, sb, steps=10):

@@ -312,10 +312,11 @@ GluPlan plan_glu(const ssm_shape& s) {
     GluPlan p{};
     size_t off = 0;
     const size_t M = (size_t)s.B * s.T, HH = (size_t)s.H * s.H;
-    p.tc = s.io_dtype == SSM_BF16 && tc_tn_supported((int)M, s.H, s.H, true) && tc_nt_supported(s.H, s.H);
+    p.tc = s.io_dtype == SSM_BF16 && tc_tn_supported((int)M, s.H, 2 * s.H, true) &&
+           tc_tn_supported((int)M, s.H, s.H, true) && tc_nt_supported(s.H, s.H);
     p.splits = p.tc ? tc_nt_splits((int)M, s.H, s.H) : gemm_nt_splits((int)M);
     p.hdr = take(off, sizeof(WsHeader));
-    p.Wt = take(off, p.tc ? 2 * HH * 2 : HH * 4);   // tc: hi/lo stacked bf16 [2H, H]; else W^T fp32
+    p.Wt = take(off, p.tc ? 4 * HH * 2 : HH * 4);   // tc: hi/lo stacked bf16 [2H, 2H]; else W^T fp32
     p.Wn = take(off, p.tc ? 2 * HH * 2 : 0);
     p.x1 = take(off, M * s.H * 4);                  // GELU(v): fp32, or two bf16 planes
     p.z = take(off, M * s.H * 4);                   // the gate's argument
@@ -351,17 +352,13 @@ SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, v
         StageTimer tm("glu_pack_gelu", st);
         launch_glu_pack(s.H, W, p.tc ? at<void>(ws, p.Wt) : nullptr, p.tc ? at<void>(ws, p.Wn) : nullptr,
                         p.tc ? nullptr : at<float>(ws, p.Wt), st);
-        launch_glu_gelu(bf16, p.tc, n, v, at<void>(ws, p.x1), st);
+        launch_glu_gelu(bf16, p.tc, n, s.H, v, at<void>(ws, p.x1), st);
     }
     {   // z[m, j] = sum_i x1[m, i] W[i, j]
         StageTimer tm("glu_gemm_z", st);
         if (p.tc) {
-            // x1 = hi + lo: one product per plane (the second one lands in the buffer g_x1 uses later);
-            // the gate's argument needs both, a single bf16 rounding of x1 there costs 2e-2 on dW
-            GemmTcTN g{at<void>(ws, p.x1), at<void>(ws, p.Wt), M, s.H, s.H, true, true, at<void>(ws, p.z), nullptr, nullptr, hdr};
-            if (int rc = launch_gemm_tc_tn(g, st)) return rc;
-            g.A = at<void>(ws, p.x1 + n * 2);
-            g.out = at<void>(ws, p.gx1);
+            // both planes of x1 along K: a single bf16 rounding of x1 here costs 2e-2 on dW
+            GemmTcTN g{at<void>(ws, p.x1), at<void>(ws, p.Wt), M, s.H, 2 * s.H, true, true, at<void>(ws, p.z), nullptr, nullptr, hdr};
             if (int rc = launch_gemm_tc_tn(g, st)) return rc;
         } else {
             GemmTN g{at<void>(ws, p.x1), false, s.H, at<void>(ws, p.Wt), false, s.H, M, s.H, s.H, Epi::StoreF32,
@@ -371,7 +368,7 @@ SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, v
     }
     {
         StageTimer tm("glu_out", st);
-        launch_glu_out(bf16, n, v, at<float>(ws, p.z), p.tc ? at<float>(ws, p.gx1) : nullptr, out, st);
+        launch_glu_out(bf16, n, v, at<float>(ws, p.z), out, st);
     }
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;
@@ -410,9 +407,9 @@ SSM_API int ssm_glu_bwd(const ssm_shape* shape, const float* W, const void* v, c
         if (p.tc) {
             // (x1_hi + x1_lo)^T (gz_hi + gz_lo) as two products, one per plane of x1
             GemmTcNT g{at<void>(ws, p.x1), s.H, at<void>(ws, p.gz), at<void>(ws, p.gz + n * 2), s.H, M, p.splits,
-                       at<float>(ws, p.part), hdr};
+                       at<float>(ws, p.part), hdr, 2 * s.H};
             if (int rc = launch_gemm_tc_nt(g, st)) return rc;
-            g.A = at<void>(ws, p.x1 + n * 2);
+            g.A = at<void>(ws, p.x1 + (size_t)s.H * 2);   // the low halves: columns [H, 2H) of x1
             g.part = at<float>(ws, p.part) + (size_t)p.splits * HH;
             if (int rc = launch_gemm_tc_nt(g, st)) return rc;
             launch_glu_reduce(at<float>(ws, p.part), 2 * p.splits, HH, dW, st);

@@ -726,11 +726,12 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 // ---------------------------------------------------------------------------------------------
 // Row-major bf16 matrix [rows, cols] (cols contiguous), boxes of box_cols x box_rows, 128-byte swizzle.
 static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_cols,
-                     uint32_t box_rows, bool f32 = false, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
+                     uint32_t box_rows, bool f32 = false, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B,
+                     uint64_t pitch_elems = 0) {
     PFN_cuTensorMapEncodeTiled fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * (f32 ? 4u : 2u)};
+    cuuint64_t strides[1] = {(pitch_elems ? pitch_elems : cols) * (f32 ? 4u : 2u)};   // rows may be wider than the view
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -861,7 +862,8 @@ int tc_nt_splits(int K, int I, int J) {
 int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
     using namespace tc;
     CUtensorMap ma, mbh, mbl;
-    if (!make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.I, 64, BK)) return SSM_ERR_CUDA;
+    if (!make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.I, 64, BK, false, CU_TENSOR_MAP_SWIZZLE_128B, (uint64_t)g.lda))
+        return SSM_ERR_CUDA;
     if (!make_map(&mbh, g.Bm_hi, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
     if (!make_map(&mbl, g.Bm_lo, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
     const int blocks = (g.K + BK - 1) / BK;

@@ -22,21 +22,26 @@ inline int blocks_for(size_t n) {
 
 // Weight operands.  tc: hi/lo bf16 halves stacked as the TN kernel wants them (rows
 // (n/128)*256 + n%128 hold the high halves of output column n, 128 rows further the low halves).
-//   Wt*: output column j, reduction index i (for z = x1 W);  Wn*: output column i, reduction j
-//   (for g_x1 = gz W^T).  Both are H x H reads of W[i, j].
-__global__ void glu_pack_kernel(int H, const float* __restrict__ W, __nv_bfloat16* __restrict__ Wt_split,
+//   Wt2: for z = [x1_hi | x1_lo] W (the two planes of x1 side by side along K): output column j,
+//        reduction index k < H -> W[k, j] (hi, lo rows), k >= H -> W[k - H, j] (hi rows only;
+//        the product of two low halves is dropped);  [2H rows, 2H columns].
+//   Wn:  for g_x1 = gz W^T: output column i, reduction index j;  [2H rows, H columns].
+__global__ void glu_pack_kernel(int H, const float* __restrict__ W, __nv_bfloat16* __restrict__ Wt2,
                                 __nv_bfloat16* __restrict__ Wn_split, float* __restrict__ Wt_f32) {
     const size_t n = (size_t)H * H;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
         const int i = (int)(e / H), j = (int)(e % H);
         const float w = W[e];
         if (Wt_f32) Wt_f32[(size_t)j * H + i] = w;
-        if (Wt_split) {
+        if (Wt2) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(w);
             const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
             const size_t rt = (size_t)(j / 128) * 256 + (j % 128), rn = (size_t)(i / 128) * 256 + (i % 128);
-            Wt_split[rt * H + i] = hi;
-            Wt_split[(rt + 128) * H + i] = lo;
+            const size_t K2 = 2 * (size_t)H;
+            Wt2[rt * K2 + i] = hi;
+            Wt2[rt * K2 + H + i] = hi;
+            Wt2[(rt + 128) * K2 + i] = lo;
+            Wt2[(rt + 128) * K2 + H + i] = __float2bfloat16_rn(0.f);
             Wn_split[rn * H + j] = hi;
             Wn_split[(rn + 128) * H + j] = lo;
         }
@@ -95,32 +100,28 @@ __device__ __forceinline__ void store8_planes(__nv_bfloat16* p, size_t plane, co
     store8<__nv_bfloat16>(p + plane, lo);
 }
 
-// x1 = GELU(v): fp32, or two bf16 planes hi / lo n elements apart (hi alone would do for a product
-// that tolerates one bf16 rounding; the gate's argument and the weight gradient do not)
+// x1 = GELU(v): fp32 [M, H], or bf16 [M, 2H] with the high halves in columns [0, H) and the low
+// halves (bf16(x1 - hi)) in [H, 2H): one operand for the gate's GEMM with both planes along K, two
+// column blocks for the weight-gradient products.  A single bf16 rounding of x1 is not enough there.
 template <typename IO, bool kPlanes>
-__global__ void glu_gelu_kernel(size_t n, const IO* __restrict__ v, void* __restrict__ x1) {
+__global__ void glu_gelu_kernel(size_t n, int H, const IO* __restrict__ v, void* __restrict__ x1) {
     for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; e < n; e += (size_t)gridDim.x * blockDim.x * 8) {
         F8 a = load8<IO>(v + e);
 #pragma unroll
         for (int i = 0; i < 8; ++i) a.x[i] = gelu_f(a.x[i]);
-        if (kPlanes) store8_planes(reinterpret_cast<__nv_bfloat16*>(x1) + e, n, a);
-        else store8<float>(reinterpret_cast<float*>(x1) + e, a);
+        if (kPlanes) {
+            const size_t m = e / H, h = e % H;   // a group of 8 stays inside one row (H % 8 == 0)
+            store8_planes(reinterpret_cast<__nv_bfloat16*>(x1) + m * 2 * H + h, (size_t)H, a);
+        } else {
+            store8<float>(reinterpret_cast<float*>(x1) + e, a);
+        }
     }
 }
 
-// out = v * sigmoid(z); with z2 (the product with the low half of x1) z becomes z + z2 first
 template <typename IO>
-__global__ void glu_out_kernel(size_t n, const IO* __restrict__ v, float* __restrict__ z, const float* __restrict__ z2,
-                               IO* __restrict__ out) {
+__global__ void glu_out_kernel(size_t n, const IO* __restrict__ v, const float* __restrict__ z, IO* __restrict__ out) {
     for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; e < n; e += (size_t)gridDim.x * blockDim.x * 8) {
-        const F8 a = load8<IO>(v + e);
-        F8 zz = load8<float>(z + e);
-        if (z2) {
-            const F8 z2v = load8<float>(z2 + e);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) zz.x[i] += z2v.x[i];
-            store8<float>(z + e, zz);
-        }
+        const F8 a = load8<IO>(v + e), zz = load8<float>(z + e);
         F8 o;
 #pragma unroll
         for (int i = 0; i < 8; ++i) o.x[i] = a.x[i] * sigmoid_f(zz.x[i]);
@@ -167,28 +168,28 @@ __global__ void glu_reduce_kernel(const float* __restrict__ part, int splits, si
 
 }  // namespace
 
-void launch_glu_pack(int H, const float* W, void* Wt_split, void* Wn_split, float* Wt_f32, cudaStream_t st) {
+void launch_glu_pack(int H, const float* W, void* Wt2, void* Wn_split, float* Wt_f32, cudaStream_t st) {
     count_launch();
-    glu_pack_kernel<<<blocks_for((size_t)H * H), kThreads, 0, st>>>(H, W, (__nv_bfloat16*)Wt_split,
+    glu_pack_kernel<<<blocks_for((size_t)H * H), kThreads, 0, st>>>(H, W, (__nv_bfloat16*)Wt2,
                                                                     (__nv_bfloat16*)Wn_split, Wt_f32);
 }
 
-void launch_glu_gelu(bool io_bf16, bool planes, size_t n, const void* v, void* x1, cudaStream_t st) {
+void launch_glu_gelu(bool io_bf16, bool planes, size_t n, int H, const void* v, void* x1, cudaStream_t st) {
     count_launch();
     const int b = blocks_for(n / 8);
     if (io_bf16 && planes)
-        glu_gelu_kernel<__nv_bfloat16, true><<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, x1);
+        glu_gelu_kernel<__nv_bfloat16, true><<<b, kThreads, 0, st>>>(n, H, (const __nv_bfloat16*)v, x1);
     else if (io_bf16)
-        glu_gelu_kernel<__nv_bfloat16, false><<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, x1);
+        glu_gelu_kernel<__nv_bfloat16, false><<<b, kThreads, 0, st>>>(n, H, (const __nv_bfloat16*)v, x1);
     else
-        glu_gelu_kernel<float, false><<<b, kThreads, 0, st>>>(n, (const float*)v, x1);
+        glu_gelu_kernel<float, false><<<b, kThreads, 0, st>>>(n, H, (const float*)v, x1);
 }
 
-void launch_glu_out(bool io_bf16, size_t n, const void* v, float* z, const float* z2, void* out, cudaStream_t st) {
+void launch_glu_out(bool io_bf16, size_t n, const void* v, const float* z, void* out, cudaStream_t st) {
     count_launch();
     const int b = blocks_for(n / 8);
-    if (io_bf16) glu_out_kernel<<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, z, z2, (__nv_bfloat16*)out);
-    else glu_out_kernel<<<b, kThreads, 0, st>>>(n, (const float*)v, z, z2, (float*)out);
+    if (io_bf16) glu_out_kernel<<<b, kThreads, 0, st>>>(n, (const __nv_bfloat16*)v, z, (__nv_bfloat16*)out);
+    else glu_out_kernel<<<b, kThreads, 0, st>>>(n, (const float*)v, z, (float*)out);
 }
 
 void launch_glu_gz(bool io_bf16, bool planes, size_t n, const void* v, const void* gout, const float* z, void* gz,

@@ -99,6 +99,7 @@ struct GemmTcNT {
     int K; int splits;
     float* part;
     WsHeader* hdr;
+    int lda = 0;   // elements between rows of A when A is a column block of a wider matrix (0: I)
 };
 bool tc_nt_supported(int I, int J);
 int tc_nt_splits(int K, int I, int J);
@@ -110,13 +111,12 @@ void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc,
                              void* Cp, void* Bq, cudaStream_t st);
 
 // glu.cu: what surrounds the GEMMs of the half-GLU gate out = v * sigmoid(GELU(v) W).
-// Wt_split / Wn_split (tensor-core path, may be NULL): hi/lo stacked bf16 operands [2H, H] for
-// z = x1 W and g_x1 = gz W^T;  Wt_f32 (CUDA-core path, may be NULL): W transposed.
-void launch_glu_pack(int H, const float* W, void* Wt_split, void* Wn_split, float* Wt_f32, cudaStream_t st);
-// x1 = GELU(v); planes: two bf16 planes (hi, lo) n elements apart, else fp32
-void launch_glu_gelu(bool io_bf16, bool planes, size_t n, const void* v, void* x1, cudaStream_t st);
-// out = v * sigmoid(z); if z2 is given, z += z2 first (stored back)
-void launch_glu_out(bool io_bf16, size_t n, const void* v, float* z, const float* z2, void* out, cudaStream_t st);
+// Tensor-core path (may be NULL): Wt2 [2H, 2H], the hi/lo stacked operand of z = [x1_hi | x1_lo] W, and
+// Wn_split [2H, H], that of g_x1 = gz W^T;  Wt_f32 (CUDA-core path, may be NULL): W transposed.
+void launch_glu_pack(int H, const float* W, void* Wt2, void* Wn_split, float* Wt_f32, cudaStream_t st);
+// x1 = GELU(v); planes: bf16 [M, 2H], high halves in columns [0, H), low halves in [H, 2H); else fp32 [M, H]
+void launch_glu_gelu(bool io_bf16, bool planes, size_t n, int H, const void* v, void* x1, cudaStream_t st);
+void launch_glu_out(bool io_bf16, size_t n, const void* v, const float* z, void* out, cudaStream_t st);
 // gz = gout * v * s (1 - s), s = sigmoid(z); planes: two bf16 planes (hi, lo) n elements apart, else fp32
 void launch_glu_gz(bool io_bf16, bool planes, size_t n, const void* v, const void* gout, const float* z, void* gz,
                    cudaStream_t st);
