@@ -347,6 +347,7 @@ SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, v
     const int M = s.B * s.T;
     const size_t n = (size_t)M * s.H;
     WsHeader* hdr = at<WsHeader>(ws, p.hdr);
+    const bool fused_gate = p.tc && tc_tn_gate_supported(M, s.H, 2 * s.H);
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
     {
         StageTimer tm("glu_pack_gelu", st);
@@ -359,6 +360,10 @@ SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, v
         if (p.tc) {
             // both planes of x1 along K: a single bf16 rounding of x1 here costs 2e-2 on dW
             GemmTcTN g{at<void>(ws, p.x1), at<void>(ws, p.Wt), M, s.H, 2 * s.H, true, true, at<void>(ws, p.z), nullptr, nullptr, hdr};
+            if (fused_gate) {   // out = v * sigmoid(z) leaves from the same epilogue
+                g.skip = v;
+                g.gate_out = out;
+            }
             if (int rc = launch_gemm_tc_tn(g, st)) return rc;
         } else {
             GemmTN g{at<void>(ws, p.x1), false, s.H, at<void>(ws, p.Wt), false, s.H, M, s.H, s.H, Epi::StoreF32,
@@ -366,7 +371,7 @@ SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, v
             launch_gemm_tn(g, st);
         }
     }
-    {
+    if (!fused_gate) {
         StageTimer tm("glu_out", st);
         launch_glu_out(bf16, n, v, at<float>(ws, p.z), out, st);
     }

@@ -39,11 +39,14 @@ constexpr int kTnThreads = 64 + 32 * kTnEpiWarps;
 constexpr int kTmemCols = 512;  // two accumulator buffers of BN columns
 constexpr int kStagingBytes = kTnEpiWarps * 32 * 32 * 4;  // per epilogue warp: 32 rows x 32 fp32 columns
 constexpr int kMaxDiag = 4096;                  // widest output whose diagonal fits the shared copy
-constexpr int kSkipBytes = kTnEpiWarps * 2 * 32 * 32 * 2;   // bf16 epilogue: two 32 x 32 bf16 skip tiles per warp
-__host__ __device__ constexpr int tn_skip_bytes(int epi) { return epi == 1 ? kSkipBytes : 0; }
+constexpr int kSkipBytes = kTnEpiWarps * 2 * 32 * 32 * 2;   // two 32 x 32 bf16 skip tiles per epilogue warp
+// Epilogues of the TN kernels: 0 = fp32 result; 1 = bf16(acc + diag * skip); 2 = fp32 result AND
+// a gated bf16 result skip * sigmoid(acc) (needs a staging buffer for each).
+__host__ __device__ constexpr int tn_skip_bytes(int epi) { return epi == 0 ? 0 : kSkipBytes; }
 __host__ __device__ constexpr int tn_diag_bytes(int epi) { return epi == 1 ? kMaxDiag * 4 : 0; }
+__host__ __device__ constexpr int tn_staging_bytes(int epi) { return epi == 2 ? kStagingBytes + kStagingBytes / 2 : kStagingBytes; }
 constexpr size_t tn_smem_bytes(int epi) {
-    return (size_t)kTnStages * kStageBytes + kStagingBytes + tn_skip_bytes(epi) + tn_diag_bytes(epi) +
+    return (size_t)kTnStages * kStageBytes + tn_staging_bytes(epi) + tn_skip_bytes(epi) + tn_diag_bytes(epi) +
            1024 /*alignment slack*/ + 256 /*barriers*/;
 }
 constexpr size_t kNtSmemBytes = (size_t)kStages * kStageBytes + 1024 + 256;
@@ -266,8 +269,9 @@ struct TnParams {
 //          load/store path to global memory.  `skip_phase`: the warp's barrier parities (bit b).
 template <int kEpi, bool kSplitW>
 __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, const CUtensorMap* tmOut,
-                                              const CUtensorMap* tmSkip, int warp, int lane, int m0, int n_out0,
-                                              int acc, uint32_t acc_phase, uint32_t tmem_base, uint32_t& skip_phase) {
+                                              const CUtensorMap* tmSkip, const CUtensorMap* tmGate, int warp, int lane,
+                                              int m0, int n_out0, int acc, uint32_t acc_phase, uint32_t tmem_base,
+                                              uint32_t& skip_phase) {
     constexpr int kOutCols = kSplitW ? BN / 2 : BN;
     const int q = warp & 3;             // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp drains
@@ -275,7 +279,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
     constexpr int kSlabs = kOutCols / 32 / 2;
     const int slab0 = half * kSlabs;    // this warp's slabs: slab0 .. slab0 + kSlabs - 1
     const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-    uint8_t* stg_bytes = s.staging + (size_t)(warp - 2) * 4096;
+    uint8_t* stg_bytes = s.staging + (size_t)(warp - 2) * (tn_staging_bytes(kEpi) / kTnEpiWarps);
 
     if (kEpi == 0) {
         if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
@@ -310,7 +314,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         return true;
     }
 
-    // ---- kEpi == 1
+    // ---- kEpi == 1, 2: the skip operand arrives by TMA
     const int w = warp - 2;
     uint8_t* skb = s.skipbuf + (size_t)w * 4096;   // two 2 KB skip tiles
     const uint32_t sbar[2] = {s.skip_full[2 * w], s.skip_full[2 * w + 1]};
@@ -326,6 +330,52 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
     }
     if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
     tc_fence_after();
+    if (kEpi == 2) {
+        // z = acc (hi + lo columns) goes out in fp32, skip * sigmoid(z) in bf16; one staging buffer each
+        float4* stg = reinterpret_cast<float4*>(stg_bytes);
+        uint8_t* ob = stg_bytes + 4096;
+#pragma unroll
+        for (int sl = 0; sl < kSlabs; ++sl) {
+            const int c = (slab0 + sl) * 32, b = sl & 1;
+            uint32_t r[32], r2[32];
+            tmem_ld32(t_row + (uint32_t)c, r);
+            tmem_ld32(t_row + (uint32_t)(BN / 2 + c), r2);
+            if (!mbar_wait(sbar[b], (skip_phase >> b) & 1u, s.abort_flag)) return false;
+            skip_phase ^= 1u << b;
+            uint4 sk[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sk[j] = *reinterpret_cast<const uint4*>(skb + b * 2048 + lane * 64 + ((j ^ swz) << 4));
+            tmem_ld_wait();
+            __syncwarp();
+            if (lane == 0 && sl + 2 < kSlabs) fetch_skip(sl + 2);
+            if (lane == 0) tma_store_wait_read();   // the previous slab has left both staging buffers
+            __syncwarp();
+            uint4 o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sk[j]);
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o[j]);
+                float z[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) z[e] = __uint_as_float(r[8 * j + e]) + __uint_as_float(r2[8 * j + e]);
+                stg[lane * 8 + ((2 * j) ^ (lane & 7))] = make_float4(z[0], z[1], z[2], z[3]);
+                stg[lane * 8 + ((2 * j + 1) ^ (lane & 7))] = make_float4(z[4], z[5], z[6], z[7]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 sf = __bfloat1622float2(s2[e]);
+                    o2[e] = __floats2bfloat162_rn(sf.x / (1.f + __expf(-z[2 * e])), sf.y / (1.f + __expf(-z[2 * e + 1])));
+                }
+                *reinterpret_cast<uint4*>(ob + lane * 64 + ((j ^ swz) << 4)) = o[j];
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0 && row0 < p.M) {
+                tma_store_2d(tmOut, smem_u32(stg), n_out0 + c, row0);
+                tma_store_2d(tmGate, smem_u32(ob), n_out0 + c, row0);
+            }
+        }
+        return true;
+    }
 #pragma unroll
     for (int sl = 0; sl < kSlabs; ++sl) {
         const int c = (slab0 + sl) * 32, b = sl & 1;
@@ -372,9 +422,10 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
 template <int kEpi, bool kSplitW>
 __global__ void __launch_bounds__(kTnThreads, 1)
 gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                  const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmSkip, TnParams p) {
+                  const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmSkip,
+                  const __grid_constant__ CUtensorMap tmGate, TnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, kTnStages, kStagingBytes, tn_diag_bytes(kEpi), kStageBytes, tn_skip_bytes(kEpi));
+    const Smem s = carve_smem(smem_raw, kTnStages, tn_staging_bytes(kEpi), tn_diag_bytes(kEpi), kStageBytes, tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (kEpi == 1)
         for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
@@ -444,7 +495,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
             const int m0 = (tile / p.n_tiles) * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
-            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
+            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, &tmGate, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
                                                     skip_phase)))
                 break;
             tc_fence_before();
@@ -469,16 +520,17 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 constexpr int kPairStages = 4;
 constexpr int kPairStageBytes = kABytes + kBBytes / 2;
 constexpr size_t pair_smem_bytes(int epi) {
-    return (size_t)kPairStages * kPairStageBytes + kStagingBytes + tn_skip_bytes(epi) + tn_diag_bytes(epi) + 1024 + 256;
+    return (size_t)kPairStages * kPairStageBytes + tn_staging_bytes(epi) + tn_skip_bytes(epi) + tn_diag_bytes(epi) + 1024 +
+           256;
 }
 
 template <int kEpi, bool kSplitW>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTnThreads, 1)
 gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
                        const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmSkip,
-                       TnParams p) {
+                       const __grid_constant__ CUtensorMap tmGate, TnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, kPairStages, kStagingBytes, tn_diag_bytes(kEpi), kPairStageBytes,
+    const Smem s = carve_smem(smem_raw, kPairStages, tn_staging_bytes(kEpi), tn_diag_bytes(kEpi), kPairStageBytes,
                               tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -584,7 +636,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         bool ok = true;
         for (int tile = pair; tile < total && ok; tile += npairs) {
             const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
-            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
+            if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, &tmGate, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
                                                     skip_phase)))
                 break;
             tc_fence_before();
@@ -792,24 +844,35 @@ bool tc_tn_supported(int M, int N_out, int K, bool split_w) {
     return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % out_cols) == 0 && N_out <= tc::kMaxDiag;
 }
 
+static int pair_tiles_of(int M, int n_tiles) { return ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * n_tiles; }
+
+bool tc_tn_gate_supported(int M, int N_out, int K) {
+    return tc_tn_supported(M, N_out, K, true) && pair_tiles_of(M, N_out / (tc::BN / 2)) >= tc::sm_count() / 2;
+}
+
 int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     using namespace tc;
     const int out_cols = g.split_w ? BN / 2 : BN;
     const int n_tiles = g.N_out / out_cols;
-    const int epi = g.store_f32 ? 0 : 1;
+    const int epi = g.gate_out ? 2 : (g.store_f32 ? 0 : 1);
     if (epi == 1 && (g.split_w || !g.diag || !g.skip)) return SSM_ERR_SHAPE;
-    CUtensorMap ma, mw, mo, ms;
+    if (epi == 2 && (!g.split_w || !g.store_f32 || !g.skip || !tc_tn_gate_supported(g.M, g.N_out, g.K))) return SSM_ERR_SHAPE;
+    CUtensorMap ma, mw, mo, ms, mg;
     if (!make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, BK, BM)) return SSM_ERR_CUDA;
     if (g.store_f32) {   // fp32 result, stored by the TMA unit in boxes of 32 rows x 32 columns
         if (!make_map(&mo, g.out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, true)) return SSM_ERR_CUDA;
-        ms = mo;         // unused
-    } else {             // bf16 result and skip operand: 32 x 32 boxes, 64-byte rows
+    } else {             // bf16 result: 32 x 32 boxes, 64-byte rows
         if (!make_map(&mo, g.out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B)) return SSM_ERR_CUDA;
-        if (!make_map(&ms, g.skip, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B)) return SSM_ERR_CUDA;
     }
+    ms = mo;             // unused unless there is a skip operand
+    mg = mo;             // unused unless there is a gated result
+    if (epi != 0 && !make_map(&ms, g.skip, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B))
+        return SSM_ERR_CUDA;
+    if (epi == 2 && !make_map(&mg, g.gate_out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B))
+        return SSM_ERR_CUDA;
     TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.diag, g.hdr, (const char*)g.A, g.K * 2};
     const int m_tiles = (g.M + BM - 1) / BM;
-    const int pair_tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * n_tiles;
+    const int pair_tiles = pair_tiles_of(g.M, n_tiles);
     bool ok = true;
     if (pair_tiles >= sm_count() / 2) {   // enough 256-row tiles to give every CTA pair one
         if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN / 2)) return SSM_ERR_CUDA;
@@ -823,9 +886,10 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
         ok = set_smem(kern, smem);                                                                         \
         const int pairs = ok ? resident_pairs(reinterpret_cast<const void*>(kern), smem) : 0;              \
         ok = ok && pairs > 0;                                                                              \
-        if (ok) kern<<<2 * min(pairs, pair_tiles), kTnThreads, smem, st>>>(ma, mw, mo, ms, p);             \
+        if (ok) kern<<<2 * min(pairs, pair_tiles), kTnThreads, smem, st>>>(ma, mw, mo, ms, mg, p);         \
     } while (0)
-        if (epi == 1) SSM_LAUNCH_PAIR(1, false);
+        if (epi == 2) SSM_LAUNCH_PAIR(2, true);
+        else if (epi == 1) SSM_LAUNCH_PAIR(1, false);
         else if (g.split_w) SSM_LAUNCH_PAIR(0, true);
         else SSM_LAUNCH_PAIR(0, false);
 #undef SSM_LAUNCH_PAIR
@@ -838,7 +902,7 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     do {                                                                                                   \
         auto kern = gemm_tc_tn_kernel<EPI, SPLIT>;                                                         \
         ok = set_smem(kern, tn_smem_bytes(EPI));                                                           \
-        if (ok) kern<<<grid, kTnThreads, tn_smem_bytes(EPI), st>>>(ma, mw, mo, ms, p);                     \
+        if (ok) kern<<<grid, kTnThreads, tn_smem_bytes(EPI), st>>>(ma, mw, mo, ms, mg, p);                 \
     } while (0)
     if (epi == 1) SSM_LAUNCH_TN(1, false);
     else if (g.split_w) SSM_LAUNCH_TN(0, true);

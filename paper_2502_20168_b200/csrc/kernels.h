@@ -87,8 +87,12 @@ struct GemmTcTN {
     void* out;
     const float* diag; const void* skip;   // bf16 result: out = acc + diag[n] * skip[m, n]
     WsHeader* hdr;
+    // Gate (with store_f32, split_w and skip): besides the fp32 result also gate_out[m, n] =
+    // bf16(skip[m, n] * sigmoid(acc)).  Only where tc_tn_gate_supported says so.
+    void* gate_out = nullptr;
 };
 bool tc_tn_supported(int M, int N_out, int K, bool split_w);
+bool tc_tn_gate_supported(int M, int N_out, int K);
 int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st);
 
 struct GemmTcNT {
