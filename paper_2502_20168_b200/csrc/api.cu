@@ -192,7 +192,19 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D,
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T, P2 = 2 * s.P;
     int rc = SSM_OK;
-    if (p.tc) {
+    if (p.tc && tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P)) {
+        {   // projection and scan in one kernel: x = scan(u Bbar^T), Bu stays on chip
+            StageTimer tm("gemm_Bu_scan_fwd", st);
+            GemmScanFwd g{u, at<void>(ws, p.W0), s.B, s.T, s.H, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+                          at<void>(ws, p.xs), (float2*)xT, hdr};
+            if ((rc = launch_gemm_scan_fwd(g, st))) return rc;
+        }
+        {   // y[m,h] = sum_k x[m,k] Cp[h,k] + D[h] u[m,h]
+            StageTimer tm("gemm_y", st);
+            GemmTcTN g{at<void>(ws, p.xs), at<void>(ws, p.W2), BT, s.H, P2, false, false, y, D, u, hdr};
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+    } else if (p.tc) {
         {   // Bu[m, 2p+c] = sum_h u[m,h] Bbar_c[p,h]     (weights as hi + lo bf16)
             StageTimer tm("gemm_Bu", st);
             GemmTcTN g{u, at<void>(ws, p.W0), BT, P2, s.H, true, true, at<void>(ws, p.f32buf), nullptr, nullptr, hdr};

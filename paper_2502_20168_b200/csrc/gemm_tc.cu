@@ -655,6 +655,282 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------
+// Input projection and forward scan in one kernel (CTA pairs)
+// ---------------------------------------------------------------------------------------------
+// x_t = keep_t Abar x_{t-1} + Bbar u_t without Bu ever reaching HBM: the accumulator tile of the
+// projection (128 consecutive steps of one sequence x 64 states, weights hi + lo) is scanned by
+// the epilogue and leaves as the two bf16 planes of x.  To make that possible a CTA walks the
+// tiles of one (sequence, 64 states) chain in time order and keeps the state between tiles; the
+// two CTAs of a pair take different sequences (the rows of an MMA need not be neighbours) and the
+// same weight tile.  Epilogue per tile, 256 threads: (1) accumulators (hi + lo) into a
+// 128 x 128 fp32 tile in shared memory, 128-byte swizzled; (2) thread (state, quarter of the
+// rows) reads its 32 rows into registers and folds them - the first quarter from the carried
+// state, the others from zero - and the quarters are joined as in the streaming scan kernels;
+// (3) it folds again and writes the hi and lo bf16 halves of its results straight to global
+// memory (a warp writes 128 contiguous bytes per row and plane), so the shared-memory tile is free
+// for the next drain as soon as everybody has read it.  T must be a multiple of 128.
+struct FsParams {
+    int B, T, P;
+    int n_tiles;      // 2P / 128
+    int k_blocks;     // H / 64
+    int tblocks;      // T / 128
+    int nchains;      // n_tiles * ceil(B / 2)
+    const float2* Abar;
+    const uint8_t* done;
+    const float2* x0;
+    float2* xT;
+    uint32_t* x_hi;   // plane of high halves, one 32-bit word (re, im as bf16) per state: [B*T, P]
+    size_t plane;     // words from the hi plane to the lo plane
+    WsHeader* hdr;
+    const char* a_base;
+    int a_row_bytes;
+};
+
+constexpr int kFsTileBytes = BM * 128 * 4;   // 128 rows x 128 fp32
+constexpr size_t kFsSmemBytes = (size_t)kPairStages * kPairStageBytes + kFsTileBytes + 1024 + 256;
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kTnEpiWarps) : "memory"); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTnThreads, 1)
+gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh, FsParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ float2 agg_e[32 * kTnEpiWarps], agg_m[32 * kTnEpiWarps], carry_s[64];
+    __shared__ uint32_t masks[4];
+    const Smem s = carve_smem(smem_raw, kPairStages, kFsTileBytes, 0, kPairStageBytes, 0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(s.full[i], 1);
+            mbar_init(s.empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s.tmem_full[i], 1);
+            mbar_init(s.tmem_empty[i], 2 * 32 * kTnEpiWarps);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x < 4) masks[threadIdx.x] = 0u;
+    __syncwarp();
+    if (warp == 1) tmem_alloc_pair(s.tmem_slot, kTmemCols);
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *s.tmem_slot_ptr;
+
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int M = p.B * p.T;
+    // chain -> (64 states, this CTA's sequence); tile tb of a chain -> first row
+    auto seq_of = [&](int chain) { return 2 * (chain / p.n_tiles) + (int)rank; };
+    auto row_of = [&](int chain, int tb) {
+        const int b = seq_of(chain);
+        return b < p.B ? b * p.T + tb * BM : M;   // no sequence (odd B): rows past the end read as zero
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmWh);
+            uint32_t leader_full[kPairStages];
+            for (int i = 0; i < kPairStages; ++i) leader_full[i] = map_to_cta(s.full[i], 0);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
+                const int n0 = (chain % p.n_tiles) * BN + (int)rank * (BN / 2);
+                for (int tb = 0; tb < p.tblocks && ok; ++tb) {
+                    const int m0 = row_of(chain, tb);
+                    {   // L2 prefetch of the next tile's rows of A (contiguous)
+                        int nc = chain, nt = tb + 1;
+                        if (nt == p.tblocks) {
+                            nt = 0;
+                            nc += npairs;
+                        }
+                        if (nc < p.nchains) {
+                            const int nm = row_of(nc, nt);
+                            if (nm < M) l2_prefetch_bulk(p.a_base + (size_t)nm * p.a_row_bytes, (uint32_t)BM * p.a_row_bytes);
+                        }
+                    }
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!(ok = mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag))) break;
+                        if (rank == 0) mbar_expect_tx(s.full[stage], 2 * kPairStageBytes);
+                        const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        tma_load_2d_pair(a_dst, &tmA, leader_full[stage], kb * BK, m0);
+                        tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full[stage], kb * BK, n0);
+                        if (++stage == kPairStages) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = instr_desc(2 * BM, BN, 0, 0);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
+                for (int tb = 0; tb < p.tblocks && ok; ++tb) {
+                    if (!(ok = mbar_wait(s.tmem_empty[acc], acc_phase ^ 1u, s.abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                        tc_fence_after();
+                        const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        const uint64_t adesc = smem_desc_kmajor(a_addr);
+                        const uint64_t bdesc = smem_desc_kmajor(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < BK / UK; ++k)
+                            umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                           (uint32_t)((kb | k) != 0));
+                        umma_commit_pair(s.empty[stage]);
+                        if (++stage == kPairStages) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                    if (!ok) break;
+                    umma_commit_pair(s.tmem_full[acc]);
+                    if ((acc ^= 1) == 0) acc_phase ^= 1u;
+                }
+            }
+        }
+    } else {
+        const uint32_t leader_empty[2] = {map_to_cta(s.tmem_empty[0], 0), map_to_cta(s.tmem_empty[1], 0)};
+        const int te = threadIdx.x - 64;            // 0..255
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        const int st = te & 63, sl = te >> 6;       // scan role: state of the tile, quarter of its rows
+        const int prow = q * 32 + lane;             // drain role: row of the tile
+        float4* T4 = reinterpret_cast<float4*>(s.staging);
+        const float2* T2 = reinterpret_cast<const float2*>(s.staging);
+        const float2 zero2 = make_float2(0.f, 0.f);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
+            const int n_tile = chain % p.n_tiles, b = seq_of(chain);
+            const bool has_seq = b < p.B;
+            const int pg = n_tile * 64 + st;        // state
+            const float2 a = p.Abar[pg];
+            float2 aR;
+            {   // Abar^32 in double
+                double re = a.x, im = a.y;
+#pragma unroll
+                for (int i = 0; i < 5; ++i) {
+                    const double r2 = re * re - im * im, i2 = 2.0 * re * im;
+                    re = r2;
+                    im = i2;
+                }
+                aR = make_float2((float)re, (float)im);
+            }
+            if (sl == 0) carry_s[st] = (p.x0 && has_seq) ? p.x0[(size_t)b * p.P + pg] : zero2;
+            for (int tb = 0; tb < p.tblocks; ++tb) {
+                const int m0 = row_of(chain, tb);
+                if (p.done && te < BM) {
+                    const bool f = has_seq && p.done[(size_t)m0 + te] != 0;
+                    const uint32_t mk = __ballot_sync(0xffffffffu, f);
+                    if (lane == 0) masks[te >> 5] = mk;
+                }
+                (void)mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag);
+                epi_sync();   // flags visible, tile free (everybody has read the previous one); also:
+                              // the 256 threads leave together or not at all
+                if (*s.abort_flag) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7)
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll
+                for (int sb = 0; sb < 2; ++sb) {
+                    const int grp = half * 2 + sb;   // 32 columns = one 128-byte group of the row
+                    uint32_t r[32], r2[32];
+                    tmem_ld32(t_row + (uint32_t)(grp * 32), r);
+                    tmem_ld32(t_row + (uint32_t)(BN / 2 + grp * 32), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        T4[prow * 32 + grp * 8 + (j ^ (prow & 7))] =
+                            make_float4(__uint_as_float(r[4 * j]) + __uint_as_float(r2[4 * j]),
+                                        __uint_as_float(r[4 * j + 1]) + __uint_as_float(r2[4 * j + 1]),
+                                        __uint_as_float(r[4 * j + 2]) + __uint_as_float(r2[4 * j + 2]),
+                                        __uint_as_float(r[4 * j + 3]) + __uint_as_float(r2[4 * j + 3]));
+                }
+                tc_fence_before();
+                mbar_arrive_cluster(leader_empty[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1u;
+                epi_sync();
+                // (2) scan: this thread's state over its 32 rows
+                const uint32_t mask = masks[sl];
+                const int r0 = sl * 32;
+                float2 v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    v[i] = T2[(r0 + i) * 64 + ((st >> 4) * 8 + (((st & 15) >> 1) ^ (i & 7))) * 2 + (st & 1)];
+                float2 e = zero2, m = aR;
+                if (sl == 0) {
+                    float2 x = carry_s[st];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if ((mask >> i) & 1u) x = zero2;
+                        v[i] = x = cfma(a, x, v[i]);
+                    }
+                    e = x;
+                    m = zero2;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if ((mask >> i) & 1u) e = zero2;
+                        e = cfma(a, e, v[i]);
+                    }
+                    if (mask != 0u) m = zero2;
+                }
+                agg_e[te] = e;
+                agg_m[te] = m;
+                epi_sync();   // pairs visible; every thread has its rows in registers
+                float2 x = e;
+                if (sl > 0) {
+                    x = agg_e[st];   // the first quarter left its final state
+                    for (int qq = 1; qq < sl; ++qq) x = cfma(agg_m[qq * 64 + st], x, agg_e[qq * 64 + st]);
+                }
+                // (3) fold again; results to global memory as hi / lo bf16 halves
+                uint32_t* out = p.x_hi + ((size_t)m0 + r0) * p.P + pg;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float2 xv = v[i];
+                    if (sl > 0) {
+                        if ((mask >> i) & 1u) x = zero2;
+                        xv = x = cfma(a, x, v[i]);
+                    }
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(xv.x, xv.y);
+                    const float2 hf = __bfloat1622float2(h);
+                    const __nv_bfloat162 l = __floats2bfloat162_rn(xv.x - hf.x, xv.y - hf.y);
+                    if (has_seq) {
+                        out[(size_t)i * p.P] = *reinterpret_cast<const uint32_t*>(&h);
+                        out[p.plane + (size_t)i * p.P] = *reinterpret_cast<const uint32_t*>(&l);
+                    }
+                }
+                if (sl == 3) {
+                    carry_s[st] = x;
+                    if (tb == p.tblocks - 1 && p.xT && has_seq) p.xT[(size_t)b * p.P + pg] = x;
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync_all();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+    if (threadIdx.x == 0 && *s.abort_flag && p.hdr) p.hdr->status = SSM_ERR_TIMEOUT;
+}
+
+// ---------------------------------------------------------------------------------------------
 // NT kernel (weight gradients): one 128 x 256 output tile and one slice of the rows per CTA
 // ---------------------------------------------------------------------------------------------
 struct NtParams {
@@ -909,6 +1185,28 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     else SSM_LAUNCH_TN(0, false);
 #undef SSM_LAUNCH_TN
     return ok ? SSM_OK : SSM_ERR_CUDA;
+}
+
+bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) {
+    if (T % tc::BM != 0 || H % tc::BK != 0 || P % 64 != 0) return false;
+    return (2 * P / 128) * ((B + 1) / 2) >= tc::sm_count() / 2;   // a chain for every CTA pair
+}
+
+int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
+    using namespace tc;
+    if (!tc_gemm_scan_fwd_supported(g.B, g.T, g.H, g.P)) return SSM_ERR_SHAPE;
+    const int M = g.B * g.T, P2 = 2 * g.P;
+    CUtensorMap ma, mw;
+    if (!make_map(&ma, g.u, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
+    if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
+    FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T / BM, (P2 / 128) * ((g.B + 1) / 2),
+               g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr, (const char*)g.u, g.H * 2};
+    count_launch();
+    if (!set_smem(gemm_scan_fwd_kernel, kFsSmemBytes)) return SSM_ERR_CUDA;
+    const int pairs = resident_pairs(reinterpret_cast<const void*>(gemm_scan_fwd_kernel), kFsSmemBytes);
+    if (pairs <= 0) return SSM_ERR_CUDA;
+    gemm_scan_fwd_kernel<<<2 * min(pairs, p.nchains), kTnThreads, kFsSmemBytes, st>>>(ma, mw, p);
+    return SSM_OK;
 }
 
 bool tc_nt_supported(int I, int J) { return (I % tc::BM) == 0 && (J % (tc::BN / 2)) == 0; }

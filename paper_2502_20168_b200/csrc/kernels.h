@@ -95,6 +95,23 @@ bool tc_tn_supported(int M, int N_out, int K, bool split_w);
 bool tc_tn_gate_supported(int M, int N_out, int K);
 int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st);
 
+// Input projection and forward scan fused (gemm_tc.cu): x = scan(u Bbar^T) written as the two bf16
+// planes of x; Bu never reaches memory.  T must be a multiple of 128 and there must be enough
+// (sequence, 64 states) chains for every pair of CTAs (tc_gemm_scan_fwd_supported).
+struct GemmScanFwd {
+    const void* u;          // bf16 [B*T, H]
+    const void* Wsplit;     // hi/lo stacked Bbar operand [4P, H] (as for GemmTcTN with split_w)
+    int B, T, H, P;
+    const float2* Abar;     // [P]
+    const uint8_t* done;    // [B*T] or NULL
+    const float2* x0;       // [B, P] or NULL
+    void* x_planes;         // out: bf16 hi plane [B*T, 2P], then the lo plane
+    float2* xT;             // out [B, P] or NULL
+    WsHeader* hdr;
+};
+bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P);
+int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st);
+
 struct GemmTcNT {
     // part[s, i, j] = sum_{m in slice s} A[m, i] * (Bm_hi[m, j] + Bm_lo[m, j]);  A bf16 [K, I],
     // Bm_hi / Bm_lo bf16 [K, J]: the two planes of a state tensor
