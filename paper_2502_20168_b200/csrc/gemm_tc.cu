@@ -689,12 +689,17 @@ struct FsParams {
 constexpr int kFsTileBytes = BM * 128 * 4;   // 128 rows x 128 fp32
 constexpr size_t kFsSmemBytes = (size_t)kPairStages * kPairStageBytes + kFsTileBytes + 1024 + 256;
 
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kTnEpiWarps) : "memory"); }
+constexpr int kFsEpiWarps = 8;               // two per TMEM lane quarter (16 measured slower: 0.34 against 0.31 ms)
+constexpr int kFsEpiThreads = 32 * kFsEpiWarps;
+constexpr int kFsThreads = 64 + kFsEpiThreads;
+constexpr int kFsRows = BM * 64 / kFsEpiThreads;   // rows per scanning thread: 64 states x (128 / kFsRows) groups
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTnThreads, 1)
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kFsEpiThreads) : "memory"); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFsThreads, 1)
 gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh, FsParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float2 agg_e[32 * kTnEpiWarps], agg_m[32 * kTnEpiWarps], carry_s[64];
+    __shared__ float2 agg_e[kFsEpiThreads], agg_m[kFsEpiThreads], carry_s[64];
     __shared__ uint32_t masks[4];
     const Smem s = carve_smem(smem_raw, kPairStages, kFsTileBytes, 0, kPairStageBytes, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -706,7 +711,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(s.tmem_full[i], 1);
-            mbar_init(s.tmem_empty[i], 2 * 32 * kTnEpiWarps);
+            mbar_init(s.tmem_empty[i], 2 * kFsEpiThreads);
         }
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -802,9 +807,10 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else {
         const uint32_t leader_empty[2] = {map_to_cta(s.tmem_empty[0], 0), map_to_cta(s.tmem_empty[1], 0)};
-        const int te = threadIdx.x - 64;            // 0..255
-        const int q = warp & 3, half = (warp - 2) >> 2;
-        const int st = te & 63, sl = te >> 6;       // scan role: state of the tile, quarter of its rows
+        constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
+        const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
+        const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
+        const int st = te & 63, sl = te >> 6;       // scan role: state of the tile, group of its rows
         const int prow = q * 32 + lane;             // drain role: row of the tile
         float4* T4 = reinterpret_cast<float4*>(s.staging);
         const float2* T2 = reinterpret_cast<const float2*>(s.staging);
@@ -818,10 +824,10 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const int pg = n_tile * 64 + st;        // state
             const float2 a = p.Abar[pg];
             float2 aR;
-            {   // Abar^32 in double
+            {   // Abar^R in double
                 double re = a.x, im = a.y;
 #pragma unroll
-                for (int i = 0; i < 5; ++i) {
+                for (int n = 1; n < R; n *= 2) {
                     const double r2 = re * re - im * im, i2 = 2.0 * re * im;
                     re = r2;
                     im = i2;
@@ -847,8 +853,8 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7)
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll
-                for (int sb = 0; sb < 2; ++sb) {
-                    const int grp = half * 2 + sb;   // 32 columns = one 128-byte group of the row
+                for (int g = grp; g < 4; g += kFsEpiWarps / 4) {   // 32 columns = one 128-byte group of the row
+                    const int grp = g;
                     uint32_t r[32], r2[32];
                     tmem_ld32(t_row + (uint32_t)(grp * 32), r);
                     tmem_ld32(t_row + (uint32_t)(BN / 2 + grp * 32), r2);
@@ -865,18 +871,19 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 mbar_arrive_cluster(leader_empty[acc]);
                 if ((acc ^= 1) == 0) acc_phase ^= 1u;
                 epi_sync();
-                // (2) scan: this thread's state over its 32 rows
-                const uint32_t mask = masks[sl];
-                const int r0 = sl * 32;
-                float2 v[32];
+                // (2) scan: this thread's state over its R rows
+                const int r0 = sl * R;
+                // (the flag tests stay in the loops even without flags: a variant compiled without them ran 10 % slower)
+                const uint32_t mask = (masks[r0 >> 5] >> (r0 & 31)) & ((R == 32) ? 0xffffffffu : ((1u << R) - 1u));
+                float2 v[R];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    v[i] = T2[(r0 + i) * 64 + ((st >> 4) * 8 + (((st & 15) >> 1) ^ (i & 7))) * 2 + (st & 1)];
+                for (int i = 0; i < R; ++i)
+                    v[i] = T2[(r0 + i) * 64 + ((st >> 4) * 8 + (((st & 15) >> 1) ^ ((r0 + i) & 7))) * 2 + (st & 1)];
                 float2 e = zero2, m = aR;
                 if (sl == 0) {
                     float2 x = carry_s[st];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = 0; i < R; ++i) {
                         if ((mask >> i) & 1u) x = zero2;
                         v[i] = x = cfma(a, x, v[i]);
                     }
@@ -884,7 +891,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     m = zero2;
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = 0; i < R; ++i) {
                         if ((mask >> i) & 1u) e = zero2;
                         e = cfma(a, e, v[i]);
                     }
@@ -901,7 +908,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 // (3) fold again; results to global memory as hi / lo bf16 halves
                 uint32_t* out = p.x_hi + ((size_t)m0 + r0) * p.P + pg;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
+                for (int i = 0; i < R; ++i) {
                     float2 xv = v[i];
                     if (sl > 0) {
                         if ((mask >> i) & 1u) x = zero2;
@@ -915,9 +922,10 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         out[p.plane + (size_t)i * p.P] = *reinterpret_cast<const uint32_t*>(&l);
                     }
                 }
-                if (sl == 3) {
-                    carry_s[st] = x;
-                    if (tb == p.tblocks - 1 && p.xT && has_seq) p.xT[(size_t)b * p.P + pg] = x;
+                if (sl == nsl - 1) {
+                    // (not after the chain's last tile: by then the first quarter may already have set up the next chain)
+                    if (tb < p.tblocks - 1) carry_s[st] = x;
+                    else if (p.xT && has_seq) p.xT[(size_t)b * p.P + pg] = x;
                 }
             }
         }
@@ -1080,7 +1088,7 @@ static int sm_count() {
 
 // How many clusters of two CTAs of `kernel` the current device runs at the same time (cached per
 // kernel and device).
-static int resident_pairs(const void* kernel, size_t smem_bytes) {
+static int resident_pairs(const void* kernel, size_t smem_bytes, int threads = kTnThreads) {
     static std::mutex mu;
     static std::map<std::pair<const void*, int>, int> cache;
     int dev = 0;
@@ -1090,7 +1098,7 @@ static int resident_pairs(const void* kernel, size_t smem_bytes) {
     if (it != cache.end()) return it->second;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (unsigned)sm_count(), 1, 1);
-    cfg.blockDim = dim3(kTnThreads, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1202,10 +1210,11 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
     FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T / BM, (P2 / 128) * ((g.B + 1) / 2),
                g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr, (const char*)g.u, g.H * 2};
     count_launch();
-    if (!set_smem(gemm_scan_fwd_kernel, kFsSmemBytes)) return SSM_ERR_CUDA;
-    const int pairs = resident_pairs(reinterpret_cast<const void*>(gemm_scan_fwd_kernel), kFsSmemBytes);
+    auto kern = gemm_scan_fwd_kernel;
+    if (!set_smem(kern, kFsSmemBytes)) return SSM_ERR_CUDA;
+    const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), kFsSmemBytes, kFsThreads);
     if (pairs <= 0) return SSM_ERR_CUDA;
-    gemm_scan_fwd_kernel<<<2 * min(pairs, p.nchains), kTnThreads, kFsSmemBytes, st>>>(ma, mw, p);
+    kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, p);
     return SSM_OK;
 }
 
