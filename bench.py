@@ -34,6 +34,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # Algorithmic work of each internal stage per timestep (one (b,t) row): bytes for the
 # HBM-bound scans, flops for the projections (a real GEMM with K*N = 2*H*P per row).
 STAGE_MODEL = {
+    # input projection and forward scan in one kernel: the contraction is what it has to do (the scan
+    # adds 8 flop per state and step and no HBM traffic)
+    "gemm_Bu_scan_fwd": ("tensor", lambda H, P, s: 4.0 * H * P),
     "gemm_Bu": ("tensor", lambda H, P, s: 4.0 * H * P),
     "scan_fwd": ("hbm", lambda H, P, s: 16.0 * P),
     "gemm_y": ("tensor", lambda H, P, s: 4.0 * H * P),
@@ -50,6 +53,7 @@ STAGE_MODEL = {
 # P = 256, bf16 I/O at T = 1024 (the scans choose other tile shapes at other T); an entry is None
 # once its kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_TIMESTEP = {
+    "gemm_Bu_scan_fwd": None,
     "scan_fwd": 1021.7e6 / 262144,
     "scan_bwd": 1579.9e6 / 262144,
     "gemm_Bu": 763.6e6 / 262144,
