@@ -178,7 +178,8 @@ static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
     launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
                       at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
     if (p.tc)
-        launch_pack_operands_tc(s.H, s.P, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+        // (the kernel that scans in the epilogue of the projection wants its own column order)
+        launch_pack_operands_tc(s.H, s.P, tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P), at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
                                 at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
     else
         launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),

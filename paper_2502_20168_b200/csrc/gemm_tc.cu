@@ -663,12 +663,14 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // tiles of one (sequence, 64 states) chain in time order and keeps the state between tiles; the
 // two CTAs of a pair take different sequences (the rows of an MMA need not be neighbours) and the
 // same weight tile.  Epilogue per tile, 256 threads: (1) accumulators (hi + lo) into a
-// 128 x 128 fp32 tile in shared memory, 128-byte swizzled; (2) thread (state, quarter of the
-// rows) reads its 32 rows into registers and folds them - the first quarter from the carried
-// state, the others from zero - and the quarters are joined as in the streaming scan kernels;
-// (3) it folds again and writes the hi and lo bf16 halves of its results straight to global
-// memory (a warp writes 128 contiguous bytes per row and plane), so the shared-memory tile is free
-// for the next drain as soon as everybody has read it.  T must be a multiple of 128.
+// 128 x 128 fp32 tile in shared memory, 128-byte swizzled; the weight rows are packed so that the
+// columns of two neighbouring states come out as (re, re, im, im); (2) thread (pair of states,
+// eighth of the rows) reads its 16 rows into registers and folds them with packed fp32x2
+// multiply-adds - the first group from the carried state, the others from zero - and the groups
+// are joined as in the streaming scan kernels; (3) it folds again and writes the hi and lo bf16
+// halves of its results straight to global memory (a warp writes 256 contiguous bytes per row and
+// plane), so the shared-memory tile is free for the next drain as soon as everybody has read it.
+// T must be a multiple of 128.
 struct FsParams {
     int B, T, P;
     int n_tiles;      // 2P / 128
@@ -692,14 +694,42 @@ constexpr size_t kFsSmemBytes = (size_t)kPairStages * kPairStageBytes + kFsTileB
 constexpr int kFsEpiWarps = 8;               // two per TMEM lane quarter (16 measured slower: 0.34 against 0.31 ms)
 constexpr int kFsEpiThreads = 32 * kFsEpiWarps;
 constexpr int kFsThreads = 64 + kFsEpiThreads;
-constexpr int kFsRows = BM * 64 / kFsEpiThreads;   // rows per scanning thread: 64 states x (128 / kFsRows) groups
+constexpr int kFsRows = BM * 32 / kFsEpiThreads;   // rows per scanning thread: 32 pairs of states x (128 / kFsRows) groups
+
+// Two fp32 values in one 64-bit register pair, and the packed multiply-add on them: the scan of
+// the epilogue advances two states per instruction.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+struct C2 {
+    f32x2 re, im;   // two complex numbers: (re, re), (im, im)
+};
+// a * x + b for two states at once (nai = -Im a)
+__device__ __forceinline__ C2 cstep2(f32x2 ar, f32x2 ai, f32x2 nai, C2 x, C2 b) {
+    C2 r;
+    r.re = fma2(ar, x.re, fma2(nai, x.im, b.re));
+    r.im = fma2(ar, x.im, fma2(ai, x.re, b.im));
+    return r;
+}
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kFsEpiThreads) : "memory"); }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFsThreads, 1)
-gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh, FsParams p) {
+gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
+                     const __grid_constant__ CUtensorMap tmX, FsParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float2 agg_e[kFsEpiThreads], agg_m[kFsEpiThreads], carry_s[64];
+    __shared__ float4 agg_e[kFsEpiThreads], carry_s[32];   // (re, re, im, im) of two neighbouring states
     __shared__ uint32_t masks[4];
     const Smem s = carve_smem(smem_raw, kPairStages, kFsTileBytes, 0, kPairStageBytes, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -810,31 +840,40 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
         const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
         const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
-        const int st = te & 63, sl = te >> 6;       // scan role: state of the tile, group of its rows
+        const int sp = te & 31, sl = te >> 5;       // scan role: pair of states of the tile, group of its rows
         const int prow = q * 32 + lane;             // drain role: row of the tile
         float4* T4 = reinterpret_cast<float4*>(s.staging);
-        const float2* T2 = reinterpret_cast<const float2*>(s.staging);
-        const float2 zero2 = make_float2(0.f, 0.f);
+        const C2 zero = {0ull, 0ull};
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
             const bool has_seq = b < p.B;
-            const int pg = n_tile * 64 + st;        // state
-            const float2 a = p.Abar[pg];
-            float2 aR;
-            {   // Abar^R in double
-                double re = a.x, im = a.y;
+            const int pg = n_tile * 64 + 2 * sp;    // the first of this thread's two states
+            const float2 a0 = p.Abar[pg], a1 = p.Abar[pg + 1];
+            const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
+            f32x2 pr, pi, npi;                      // Abar^R, evaluated in double
+            {
+                double re0 = a0.x, im0 = a0.y, re1 = a1.x, im1 = a1.y;
 #pragma unroll
                 for (int n = 1; n < R; n *= 2) {
-                    const double r2 = re * re - im * im, i2 = 2.0 * re * im;
-                    re = r2;
-                    im = i2;
+                    const double r0 = re0 * re0 - im0 * im0, i0 = 2.0 * re0 * im0;
+                    const double r1 = re1 * re1 - im1 * im1, i1 = 2.0 * re1 * im1;
+                    re0 = r0, im0 = i0, re1 = r1, im1 = i1;
                 }
-                aR = make_float2((float)re, (float)im);
+                pr = pack2((float)re0, (float)re1);
+                pi = pack2((float)im0, (float)im1);
+                npi = pack2(-(float)im0, -(float)im1);
             }
-            if (sl == 0) carry_s[st] = (p.x0 && has_seq) ? p.x0[(size_t)b * p.P + pg] : zero2;
+            if (sl == 0) {   // the carried state, as (re, re, im, im) of the two states
+                float2 c0 = make_float2(0.f, 0.f), c1 = c0;
+                if (p.x0 && has_seq) {
+                    c0 = p.x0[(size_t)b * p.P + pg];
+                    c1 = p.x0[(size_t)b * p.P + pg + 1];
+                }
+                carry_s[sp] = make_float4(c0.x, c1.x, c0.y, c1.y);
+            }
             for (int tb = 0; tb < p.tblocks; ++tb) {
                 const int m0 = row_of(chain, tb);
                 if (p.done && te < BM) {
@@ -843,7 +882,8 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (lane == 0) masks[te >> 5] = mk;
                 }
                 (void)mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag);
-                epi_sync();   // flags visible, tile free (everybody has read the previous one); also:
+                if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
+                epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
                               // the 256 threads leave together or not at all
                 if (*s.abort_flag) {
                     ok = false;
@@ -854,14 +894,13 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll
                 for (int g = grp; g < 4; g += kFsEpiWarps / 4) {   // 32 columns = one 128-byte group of the row
-                    const int grp = g;
                     uint32_t r[32], r2[32];
-                    tmem_ld32(t_row + (uint32_t)(grp * 32), r);
-                    tmem_ld32(t_row + (uint32_t)(BN / 2 + grp * 32), r2);
+                    tmem_ld32(t_row + (uint32_t)(g * 32), r);
+                    tmem_ld32(t_row + (uint32_t)(BN / 2 + g * 32), r2);
                     tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        T4[prow * 32 + grp * 8 + (j ^ (prow & 7))] =
+                        T4[prow * 32 + g * 8 + (j ^ (prow & 7))] =
                             make_float4(__uint_as_float(r[4 * j]) + __uint_as_float(r2[4 * j]),
                                         __uint_as_float(r[4 * j + 1]) + __uint_as_float(r2[4 * j + 1]),
                                         __uint_as_float(r[4 * j + 2]) + __uint_as_float(r2[4 * j + 2]),
@@ -871,64 +910,125 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 mbar_arrive_cluster(leader_empty[acc]);
                 if ((acc ^= 1) == 0) acc_phase ^= 1u;
                 epi_sync();
-                // (2) scan: this thread's state over its R rows
+                // (2) scan: this thread's two states over its R rows.  The flags of a row group are the
+                // same for the whole warp: a group without flags takes loops without the tests.
                 const int r0 = sl * R;
-                // (the flag tests stay in the loops even without flags: a variant compiled without them ran 10 % slower)
-                const uint32_t mask = (masks[r0 >> 5] >> (r0 & 31)) & ((R == 32) ? 0xffffffffu : ((1u << R) - 1u));
-                float2 v[R];
+                uint32_t gflags = 0;   // bit g: row group g has a flag
+                if (p.done) {
 #pragma unroll
-                for (int i = 0; i < R; ++i)
-                    v[i] = T2[(r0 + i) * 64 + ((st >> 4) * 8 + (((st & 15) >> 1) ^ ((r0 + i) & 7))) * 2 + (st & 1)];
-                float2 e = zero2, m = aR;
-                if (sl == 0) {
-                    float2 x = carry_s[st];
+                    for (int w = 0; w < 4; ++w) {
+                        const uint32_t mk = masks[w];
 #pragma unroll
-                    for (int i = 0; i < R; ++i) {
-                        if ((mask >> i) & 1u) x = zero2;
-                        v[i] = x = cfma(a, x, v[i]);
+                        for (int h = 0; h < 32 / R; ++h)
+                            if ((mk >> (h * R)) & ((1u << R) - 1u)) gflags |= 1u << (w * (32 / R) + h);
+                    }
+                }
+                const uint32_t mask = p.done ? (masks[r0 >> 5] >> (r0 & 31)) & ((1u << R) - 1u) : 0u;
+                C2 v[R];
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const int row = r0 + i;
+                    const float4 t = T4[row * 32 + ((sp & ~7) | ((sp & 7) ^ (row & 7)))];   // (re, re, im, im)
+                    v[i].re = pack2(t.x, t.y);
+                    v[i].im = pack2(t.z, t.w);
+                }
+                C2 e = zero;
+                if (sl == 0) {   // from the carried state: these results are final
+                    const float4 c = carry_s[sp];
+                    C2 x = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                    if (mask == 0u) {
+#pragma unroll
+                        for (int i = 0; i < R; ++i) v[i] = x = cstep2(ar, ai, nai, x, v[i]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < R; ++i) {
+                            if ((mask >> i) & 1u) x = zero;
+                            v[i] = x = cstep2(ar, ai, nai, x, v[i]);
+                        }
                     }
                     e = x;
-                    m = zero2;
+                } else if (mask == 0u) {
+#pragma unroll
+                    for (int i = 0; i < R; ++i) e = cstep2(ar, ai, nai, e, v[i]);
                 } else {
 #pragma unroll
                     for (int i = 0; i < R; ++i) {
-                        if ((mask >> i) & 1u) e = zero2;
-                        e = cfma(a, e, v[i]);
+                        if ((mask >> i) & 1u) e = zero;
+                        e = cstep2(ar, ai, nai, e, v[i]);
                     }
-                    if (mask != 0u) m = zero2;
                 }
-                agg_e[te] = e;
-                agg_m[te] = m;
-                epi_sync();   // pairs visible; every thread has its rows in registers
-                float2 x = e;
-                if (sl > 0) {
-                    x = agg_e[st];   // the first quarter left its final state
-                    for (int qq = 1; qq < sl; ++qq) x = cfma(agg_m[qq * 64 + st], x, agg_e[qq * 64 + st]);
+                {
+                    float e0, e1, e2, e3;
+                    unpack2(e.re, e0, e1);
+                    unpack2(e.im, e2, e3);
+                    agg_e[te] = make_float4(e0, e1, e2, e3);
                 }
-                // (3) fold again; results to global memory as hi / lo bf16 halves
-                uint32_t* out = p.x_hi + ((size_t)m0 + r0) * p.P + pg;
+                epi_sync();   // group results visible; every thread has its rows in registers
+                C2 x = e;
+                if (sl > 0) {   // state before this group's first row
+                    {
+                        const float4 c = agg_e[sp];
+                        x.re = pack2(c.x, c.y);
+                        x.im = pack2(c.z, c.w);
+                    }
 #pragma unroll
-                for (int i = 0; i < R; ++i) {
-                    float2 xv = v[i];
-                    if (sl > 0) {
-                        if ((mask >> i) & 1u) x = zero2;
-                        xv = x = cfma(a, x, v[i]);
+                    for (int g = 1; g < nsl - 1; ++g) {
+                        if (g < sl) {
+                            const float4 c = agg_e[g * 32 + sp];
+                            const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                            x = ((gflags >> g) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
+                        }
                     }
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(xv.x, xv.y);
-                    const float2 hf = __bfloat1622float2(h);
-                    const __nv_bfloat162 l = __floats2bfloat162_rn(xv.x - hf.x, xv.y - hf.y);
-                    if (has_seq) {
-                        out[(size_t)i * p.P] = *reinterpret_cast<const uint32_t*>(&h);
-                        out[p.plane + (size_t)i * p.P] = *reinterpret_cast<const uint32_t*>(&l);
+                }
+                // (3) fold again; results as hi / lo bf16 halves into this warp's part of the tile (everybody
+                // has its rows in registers by now): [plane][row][64 states], which the warp hands to the TMA unit
+                uint8_t* warp_out = s.staging + sl * (2 * R * 256);
+                uint2* out = reinterpret_cast<uint2*>(warp_out) + sp;
+                auto emit = [&](int i, C2 xv) {
+                    float re0, re1, im0, im1;
+                    unpack2(xv.re, re0, re1);
+                    unpack2(xv.im, im0, im1);
+                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(re0, im0), h1 = __floats2bfloat162_rn(re1, im1);
+                    const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+                    const __nv_bfloat162 l0 = __floats2bfloat162_rn(re0 - f0.x, im0 - f0.y);
+                    const __nv_bfloat162 l1 = __floats2bfloat162_rn(re1 - f1.x, im1 - f1.y);
+                    out[i * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                    out[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+                };
+                if (sl == 0) {
+#pragma unroll
+                    for (int i = 0; i < R; ++i) emit(i, v[i]);
+                } else if (mask == 0u) {
+#pragma unroll
+                    for (int i = 0; i < R; ++i) emit(i, x = cstep2(ar, ai, nai, x, v[i]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < R; ++i) {
+                        if ((mask >> i) & 1u) x = zero;
+                        emit(i, x = cstep2(ar, ai, nai, x, v[i]));
                     }
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0 && has_seq) {
+                    tma_store_3d_nocommit(&tmX, smem_u32(warp_out), n_tile * 64, m0 + r0, 0);
+                    tma_commit_group();
                 }
                 if (sl == nsl - 1) {
-                    // (not after the chain's last tile: by then the first quarter may already have set up the next chain)
-                    if (tb < p.tblocks - 1) carry_s[st] = x;
-                    else if (p.xT && has_seq) p.xT[(size_t)b * p.P + pg] = x;
+                    float x0r, x1r, x0i, x1i;
+                    unpack2(x.re, x0r, x1r);
+                    unpack2(x.im, x0i, x1i);
+                    // (not after the chain's last tile: by then the first group may already have set up the next chain)
+                    if (tb < p.tblocks - 1) {
+                        carry_s[sp] = make_float4(x0r, x1r, x0i, x1i);
+                    } else if (p.xT && has_seq) {
+                        p.xT[(size_t)b * p.P + pg] = make_float2(x0r, x0i);
+                        p.xT[(size_t)b * p.P + pg + 1] = make_float2(x1r, x1i);
+                    }
                 }
             }
         }
+        if (lane == 0) tma_store_wait_all();
     }
     tc_fence_before();
     __syncwarp();
@@ -1204,9 +1304,20 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
     using namespace tc;
     if (!tc_gemm_scan_fwd_supported(g.B, g.T, g.H, g.P)) return SSM_ERR_SHAPE;
     const int M = g.B * g.T, P2 = 2 * g.P;
-    CUtensorMap ma, mw;
+    CUtensorMap ma, mw, mx;
     if (!make_map(&ma, g.u, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
     if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
+    {   // the two planes of x as [2, B*T, P] 32-bit words; a warp stores 64 states x its rows x both planes
+        PFN_cuTensorMapEncodeTiled fn = encode_fn();
+        if (!fn) return SSM_ERR_CUDA;
+        cuuint64_t dims[3] = {(cuuint64_t)g.P, (cuuint64_t)M, 2};
+        cuuint64_t strides[2] = {(cuuint64_t)g.P * 4, (cuuint64_t)M * g.P * 4};
+        cuuint32_t box[3] = {64, (cuuint32_t)kFsRows, 2};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (fn(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, g.x_planes, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SSM_ERR_CUDA;
+    }
     FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T / BM, (P2 / 128) * ((g.B + 1) / 2),
                g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr, (const char*)g.u, g.H * 2};
     count_launch();
@@ -1214,7 +1325,7 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
     if (!set_smem(kern, kFsSmemBytes)) return SSM_ERR_CUDA;
     const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), kFsSmemBytes, kFsThreads);
     if (pairs <= 0) return SSM_ERR_CUDA;
-    kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, p);
+    kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, mx, p);
     return SSM_OK;
 }
 

@@ -128,7 +128,7 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 
 // discretize.cu: operands of the tensor-core path (bf16).  Wsplit_B / Wsplit_C: [4P, H] hi/lo
 // stacked forms of Bp / Cq (see GemmTcTN);  Cp, Bq: [H, 2P] single bf16.
-void launch_pack_operands_tc(int H, int P, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
+void launch_pack_operands_tc(int H, int P, bool pair_cols, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st);
 
 // glu.cu: what surrounds the GEMMs of the half-GLU gate out = v * sigmoid(GELU(v) W).
