@@ -274,3 +274,38 @@ def test_generator_is_seeded_and_shaped():
     assert 0 < d1["done"].mean() < 0.05
     assert I.draw_layer(I.C0)["done"] is None
     assert [I.shard_batch(10, r, 4) for r in range(4)] == [(0, 3), (3, 6), (6, 8), (8, 10)]
+
+
+# ---- conjugate-symmetric parameters ----------------------------------------
+def test_conjugate_pairs_fold_into_half_the_states_with_doubled_C():
+    """A system whose states come in conjugate pairs (Lambda, B, C and the initial state of state
+    p + P/2 are the conjugates of those of state p) has a real output before Re() is taken, and
+    Re(C x) over all P states equals Re(2 C x) over the first half: the variant that stores P/2
+    states is this layer with C doubled.  Gradients follow by the chain rule (dC_half = 2 x the
+    gradient of the doubled C), checked on du and on the first-half parameter gradients."""
+    d = small(seed=21, B=2, T=9, H=3, P=4, p_done=0.2, with_x0=True)
+    half = {k: d[k] for k in ("Delta", "Lambda", "Bc", "Cc", "x0")}
+    Lam = np.concatenate([half["Lambda"], np.conj(half["Lambda"])])
+    Dl = np.concatenate([half["Delta"], half["Delta"]])
+    Bc = np.concatenate([half["Bc"], np.conj(half["Bc"])], axis=0)
+    Cc = np.concatenate([half["Cc"], np.conj(half["Cc"])], axis=1)
+    x0 = np.concatenate([half["x0"], np.conj(half["x0"])], axis=1)
+    y_full, xT_full, _ = O.ssm_layer_fwd(Lam, Dl, Bc, Cc, d["D"], d["u"], d["done"], x0)
+    y_half, xT_half, _ = O.ssm_layer_fwd(half["Lambda"], half["Delta"], half["Bc"], 2.0 * half["Cc"], d["D"], d["u"],
+                                         d["done"], half["x0"])
+    P = half["Lambda"].shape[0]
+    np.testing.assert_allclose(y_full, y_half, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(xT_full[:, :P], xT_half, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(xT_full[:, P:], np.conj(xT_half), rtol=1e-12, atol=1e-12)
+    g_full = O.ssm_layer_bwd(Lam, Dl, Bc, Cc, d["D"], d["u"], d["done"], x0, d["gy"])
+    g_half = O.ssm_layer_bwd(half["Lambda"], half["Delta"], half["Bc"], 2.0 * half["Cc"], d["D"], d["u"], d["done"],
+                             half["x0"], d["gy"])
+    np.testing.assert_allclose(g_full["du"], g_half["du"], rtol=1e-11, atol=1e-11)
+    np.testing.assert_allclose(g_full["dD"], g_half["dD"], rtol=1e-11, atol=1e-11)
+    # each parameter of the half system appears twice in the full one (once conjugated): with the
+    # convention g = dL/dRe + i dL/dIm the two contributions are g and conj(g) of the pair
+    np.testing.assert_allclose(g_full["dB"][:P] + np.conj(g_full["dB"][P:]), g_half["dB"], rtol=1e-10, atol=1e-10)
+    np.testing.assert_allclose(g_full["dLambda"][:P] + np.conj(g_full["dLambda"][P:]), g_half["dLambda"], rtol=1e-10,
+                               atol=1e-10)
+    np.testing.assert_allclose(g_full["dC"][:, :P] + np.conj(g_full["dC"][:, P:]), 2.0 * g_half["dC"], rtol=1e-10,
+                               atol=1e-10)
