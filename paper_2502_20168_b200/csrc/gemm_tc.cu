@@ -670,13 +670,17 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // are joined as in the streaming scan kernels; (3) it folds again and writes the hi and lo bf16
 // halves of its results straight to global memory (a warp writes 256 contiguous bytes per row and
 // plane), so the shared-memory tile is free for the next drain as soon as everybody has read it.
-// T must be a multiple of 128.
+// T is a multiple of 128, or 16, 32 or 64: then a tile holds 128 / T whole sequences, a chain is one
+// tile, and every row group that begins a sequence starts from that sequence's initial state.
 struct FsParams {
     int B, T, P;
     int n_tiles;      // 2P / 128
     int k_blocks;     // H / 64
-    int tblocks;      // T / 128
-    int nchains;      // n_tiles * ceil(B / 2)
+    int tblocks;      // tiles per chain: T / 128, or 1
+    int unit_rows;    // rows of a chain: T, or 128 when T < 128
+    int n_units;      // chains per 64 states: B, or ceil(B * T / 128)
+    int gps;          // row groups per sequence inside a tile: 8, or T / 16
+    int nchains;      // n_tiles * ceil(n_units / 2)
     const float2* Abar;
     const uint8_t* done;
     const float2* x0;
@@ -752,22 +756,22 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *s.tmem_slot_ptr;
+    // the barriers of a kind are 8 bytes apart: addresses by arithmetic, so that no array is indexed at run time
+    const uint32_t full0 = s.full[0], empty0 = s.empty[0], tfull0 = s.tmem_full[0], tempty0 = s.tmem_empty[0];
 
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int M = p.B * p.T;
-    // chain -> (64 states, this CTA's sequence); tile tb of a chain -> first row
+    // chain -> (64 states, this CTA's sequence or, for short sequences, tile of rows); tile tb of a chain -> first row
     auto seq_of = [&](int chain) { return 2 * (chain / p.n_tiles) + (int)rank; };
     auto row_of = [&](int chain, int tb) {
         const int b = seq_of(chain);
-        return b < p.B ? b * p.T + tb * BM : M;   // no sequence (odd B): rows past the end read as zero
+        return b < p.n_units ? b * p.unit_rows + tb * BM : M;   // nothing left for this CTA: rows past the end read as zero
     };
 
     if (warp == 0) {
         if (lane == 0) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmWh);
-            uint32_t leader_full[kPairStages];
-            for (int i = 0; i < kPairStages; ++i) leader_full[i] = map_to_cta(s.full[i], 0);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -777,11 +781,12 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const int m0 = row_of(chain, tb);
                     // (no L2 prefetch of the next tile's rows here: with it the kernel ran 7 % slower)
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!(ok = mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag))) break;
-                        if (rank == 0) mbar_expect_tx(s.full[stage], 2 * kPairStageBytes);
+                        if (!(ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, s.abort_flag))) break;
+                        const uint32_t leader_full = map_to_cta(full0 + 8u * stage, 0);
+                        if (rank == 0) mbar_expect_tx(full0 + 8u * stage, 2 * kPairStageBytes);
                         const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
-                        tma_load_2d_pair(a_dst, &tmA, leader_full[stage], kb * BK, m0);
-                        tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full[stage], kb * BK, n0);
+                        tma_load_2d_pair(a_dst, &tmA, leader_full, kb * BK, m0);
+                        tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full, kb * BK, n0);
                         if (++stage == kPairStages) {
                             stage = 0;
                             phase ^= 1u;
@@ -798,11 +803,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             bool ok = true;
             for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
                 for (int tb = 0; tb < p.tblocks && ok; ++tb) {
-                    if (!(ok = mbar_wait(s.tmem_empty[acc], acc_phase ^ 1u, s.abort_flag))) break;
+                    if (!(ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, s.abort_flag))) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                        if (!(ok = mbar_wait(full0 + 8u * stage, phase, s.abort_flag))) break;
                         tc_fence_after();
                         const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
                         const uint64_t adesc = smem_desc_kmajor(a_addr);
@@ -811,20 +816,20 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         for (int k = 0; k < BK / UK; ++k)
                             umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
                                            (uint32_t)((kb | k) != 0));
-                        umma_commit_pair(s.empty[stage]);
+                        umma_commit_pair(empty0 + 8u * stage);
                         if (++stage == kPairStages) {
                             stage = 0;
                             phase ^= 1u;
                         }
                     }
                     if (!ok) break;
-                    umma_commit_pair(s.tmem_full[acc]);
+                    umma_commit_pair(tfull0 + 8u * acc);
                     if ((acc ^= 1) == 0) acc_phase ^= 1u;
                 }
             }
         }
     } else {
-        const uint32_t leader_empty[2] = {map_to_cta(s.tmem_empty[0], 0), map_to_cta(s.tmem_empty[1], 0)};
+        const uint32_t leader_empty0 = map_to_cta(tempty0, 0);
         constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
         const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
         const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
@@ -837,24 +842,27 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         bool ok = true;
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
-            const bool has_seq = b < p.B;
+            const bool has_seq = b < p.n_units;
+            const bool short_seq = p.T < BM;        // then b counts tiles of rows, not sequences
+            const int g0 = sl - sl % p.gps;         // the first row group of this group's sequence in the tile
+            const bool from_carry = sl == g0;
             const int pg = n_tile * 64 + 2 * sp;    // the first of this thread's two states
             const float2 a0 = p.Abar[pg], a1 = p.Abar[pg + 1];
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
-            f32x2 pr, pi, npi;                      // Abar^R, evaluated in double
+            f32x2 pr, pi, npi;   // Abar^R by squaring in fp32 (a few 1e-7 relative: the results leave as bf16 pairs)
             {
-                double re0 = a0.x, im0 = a0.y, re1 = a1.x, im1 = a1.y;
+                float re0 = a0.x, im0 = a0.y, re1 = a1.x, im1 = a1.y;
 #pragma unroll
                 for (int n = 1; n < R; n *= 2) {
-                    const double r0 = re0 * re0 - im0 * im0, i0 = 2.0 * re0 * im0;
-                    const double r1 = re1 * re1 - im1 * im1, i1 = 2.0 * re1 * im1;
+                    const float r0 = fmaf(re0, re0, -im0 * im0), i0 = 2.f * re0 * im0;
+                    const float r1 = fmaf(re1, re1, -im1 * im1), i1 = 2.f * re1 * im1;
                     re0 = r0, im0 = i0, re1 = r1, im1 = i1;
                 }
-                pr = pack2((float)re0, (float)re1);
-                pi = pack2((float)im0, (float)im1);
-                npi = pack2(-(float)im0, -(float)im1);
+                pr = pack2(re0, re1);
+                pi = pack2(im0, im1);
+                npi = pack2(-im0, -im1);
             }
-            if (sl == 0) {   // the carried state, as (re, re, im, im) of the two states
+            if (sl == 0 && !short_seq) {   // the carried state, as (re, re, im, im) of the two states
                 float2 c0 = make_float2(0.f, 0.f), c1 = c0;
                 if (p.x0 && has_seq) {
                     c0 = p.x0[(size_t)b * p.P + pg];
@@ -865,11 +873,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             for (int tb = 0; tb < p.tblocks; ++tb) {
                 const int m0 = row_of(chain, tb);
                 if (p.done && te < BM) {
-                    const bool f = has_seq && p.done[(size_t)m0 + te] != 0;
+                    const bool f = has_seq && m0 + te < M && p.done[(size_t)m0 + te] != 0;
                     const uint32_t mk = __ballot_sync(0xffffffffu, f);
                     if (lane == 0) masks[te >> 5] = mk;
                 }
-                (void)mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag);
+                (void)mbar_wait(tfull0 + 8u * acc, acc_phase, s.abort_flag);
                 if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
                 epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
                               // the 256 threads leave together or not at all
@@ -895,12 +903,14 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                                         __uint_as_float(r[4 * j + 3]) + __uint_as_float(r2[4 * j + 3]));
                 }
                 tc_fence_before();
-                mbar_arrive_cluster(leader_empty[acc]);
+                mbar_arrive_cluster(leader_empty0 + 8u * acc);
                 if ((acc ^= 1) == 0) acc_phase ^= 1u;
                 epi_sync();
                 // (2) scan: this thread's two states over its R rows.  The flags of a row group are the
                 // same for the whole warp: a group without flags takes loops without the tests.
                 const int r0 = sl * R;
+                const bool grp_valid = has_seq && m0 + r0 < M;           // (short sequences: the last tile may be ragged)
+                const int b_grp = short_seq ? (m0 + r0) / p.T : b;      // this group's sequence
                 uint32_t gflags = 0;   // bit g: row group g has a flag
                 if (p.done) {
 #pragma unroll
@@ -921,8 +931,16 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     v[i].im = pack2(t.z, t.w);
                 }
                 C2 e = zero;
-                if (sl == 0) {   // from the carried state: these results are final
-                    const float4 c = carry_s[sp];
+                if (from_carry) {   // from the carried or the initial state: these results are final
+                    float4 c;
+                    if (!short_seq) {
+                        c = carry_s[sp];
+                    } else if (p.x0 && grp_valid) {
+                        const float2 c0 = p.x0[(size_t)b_grp * p.P + pg], c1 = p.x0[(size_t)b_grp * p.P + pg + 1];
+                        c = make_float4(c0.x, c1.x, c0.y, c1.y);
+                    } else {
+                        c = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                     C2 x = {pack2(c.x, c.y), pack2(c.z, c.w)};
                     if (mask == 0u) {
 #pragma unroll
@@ -953,15 +971,15 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 epi_sync();   // group results visible; every thread has its rows in registers
                 C2 x = e;
-                if (sl > 0) {   // state before this group's first row
+                if (!from_carry) {   // state before this group's first row
                     {
-                        const float4 c = agg_e[sp];
+                        const float4 c = agg_e[g0 * 32 + sp];
                         x.re = pack2(c.x, c.y);
                         x.im = pack2(c.z, c.w);
                     }
 #pragma unroll
                     for (int g = 1; g < nsl - 1; ++g) {
-                        if (g < sl) {
+                        if (g > g0 && g < sl) {
                             const float4 c = agg_e[g * 32 + sp];
                             const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
                             x = ((gflags >> g) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
@@ -983,7 +1001,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     out[i * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
                     out[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
                 };
-                if (sl == 0) {
+                if (from_carry) {
 #pragma unroll
                     for (int i = 0; i < R; ++i) emit(i, v[i]);
                 } else if (mask == 0u) {
@@ -998,20 +1016,20 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0 && has_seq) {
+                if (lane == 0 && grp_valid) {
                     tma_store_3d_nocommit(&tmX, smem_u32(warp_out), n_tile * 64, m0 + r0, 0);
                     tma_commit_group();
                 }
-                if (sl == nsl - 1) {
+                if (short_seq ? (sl - g0 == p.gps - 1) : (sl == nsl - 1)) {   // the group that ends a sequence or the tile
                     float x0r, x1r, x0i, x1i;
                     unpack2(x.re, x0r, x1r);
                     unpack2(x.im, x0i, x1i);
                     // (not after the chain's last tile: by then the first group may already have set up the next chain)
-                    if (tb < p.tblocks - 1) {
+                    if (!short_seq && tb < p.tblocks - 1) {
                         carry_s[sp] = make_float4(x0r, x1r, x0i, x1i);
-                    } else if (p.xT && has_seq) {
-                        p.xT[(size_t)b * p.P + pg] = make_float2(x0r, x0i);
-                        p.xT[(size_t)b * p.P + pg + 1] = make_float2(x1r, x1i);
+                    } else if (p.xT && grp_valid) {
+                        p.xT[(size_t)b_grp * p.P + pg] = make_float2(x0r, x0i);
+                        p.xT[(size_t)b_grp * p.P + pg + 1] = make_float2(x1r, x1i);
                     }
                 }
             }
@@ -1283,9 +1301,13 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
 
+// Chains per 64 states: the sequences, or, when a 128-row tile holds several whole sequences, the tiles.
+static int fs_units(int B, int T) { return T >= tc::BM ? B : (B * T + tc::BM - 1) / tc::BM; }
+
 bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) {
-    if (T % tc::BM != 0 || H % tc::BK != 0 || P % 64 != 0) return false;
-    return (2 * P / 128) * ((B + 1) / 2) >= tc::sm_count() / 2;   // a chain for every CTA pair
+    const bool t_ok = T % tc::BM == 0 || T == 16 || T == 32 || T == 64;
+    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return false;
+    return (2 * P / 128) * ((fs_units(B, T) + 1) / 2) >= tc::sm_count() / 2;   // a chain for every CTA pair
 }
 
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
@@ -1306,7 +1328,9 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return SSM_ERR_CUDA;
     }
-    FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T / BM, (P2 / 128) * ((g.B + 1) / 2),
+    const int units = fs_units(g.B, g.T);
+    FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
+               g.T >= BM ? BM / kFsRows : g.T / kFsRows, (P2 / 128) * ((units + 1) / 2),
                g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr};
     count_launch();
     auto kern = gemm_scan_fwd_kernel;

@@ -59,17 +59,19 @@ def test_tensor_core_path_shapes_bf16(B, T, H, P):
     run(w, with_x0=True, with_gxT=True)
 
 
-@pytest.mark.parametrize("B,T,H,P", [(81, 128, 256, 128), (150, 256, 256, 64), (76, 384, 512, 128)])
+@pytest.mark.parametrize("B,T,H,P", [(81, 128, 256, 128), (150, 256, 256, 64), (76, 384, 512, 128),
+                                     (301, 64, 256, 128), (601, 32, 256, 128), (2403, 16, 256, 64)])
 def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
-    # T a multiple of 128 and enough (sequence, 64 states) chains: the input projection and the forward
-    # scan run as one kernel; odd B leaves one CTA of the last pair without a sequence
+    # Enough (sequence, 64 states) chains and T a multiple of 128, or T = 16, 32, 64 (a 128-row tile
+    # then holds whole sequences; odd B leaves the last tile ragged): the input projection and the
+    # forward scan run as one kernel.  Odd B leaves one CTA of the last pair without work.
     w = I.Workload("fused", B=B, T=T, H=H, P=P, io_dtype="bf16", p_done=0.02, seed=B + T)
 
     def flags(d):
         d["done"][0, 0] = 1
         d["done"][-1, -1] = 1
-        d["done"][1, 127] = 1        # last row of a tile
-        d["done"][2, 128 % T] = 1    # first row of a tile
+        d["done"][1, min(127, T - 1)] = 1   # last row of a tile
+        d["done"][2, 128 % T] = 1           # first row of a tile
     run(w, with_x0=True, with_gxT=True, mutate=flags)
     run(I.small_variant(w, p_done=0.0))
 
