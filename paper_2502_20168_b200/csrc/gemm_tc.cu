@@ -175,8 +175,14 @@ struct Smem {
     uint8_t* staging;     // epilogue transpose buffers
     float* diag;          // copy of the epilogue's diagonal
     uint8_t* skipbuf;     // bf16 epilogue: per epilogue warp two 32 x 32 bf16 tiles of the skip operand
-    uint32_t full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
-    uint32_t skip_full[2 * kTnEpiWarps];
+    // mbarriers of a kind sit 8 bytes apart: their addresses are computed, so that no array is indexed at
+    // run time (that would put this struct into local memory)
+    uint32_t full0, empty0, tmem_full0, tmem_empty0, skip_full0;
+    __device__ __forceinline__ uint32_t full(int i) const { return full0 + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t empty(int i) const { return empty0 + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t tmem_full(int i) const { return tmem_full0 + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t tmem_empty(int i) const { return tmem_empty0 + 8u * (uint32_t)i; }
+    __device__ __forceinline__ uint32_t skip_full(int i) const { return skip_full0 + 8u * (uint32_t)i; }
     uint32_t tmem_slot;   // where tcgen05.alloc writes the base address
     volatile int* abort_flag;
     volatile uint32_t* tmem_slot_ptr;
@@ -193,18 +199,14 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging
     s.skipbuf = s.staging + staging_bytes;
     s.diag = reinterpret_cast<float*>(s.skipbuf + skip_bytes);
     uint8_t* bars = s.skipbuf + skip_bytes + diag_bytes;
-    for (int i = 0; i < kStages; ++i) {
-        s.full[i] = smem_u32(bars + 8 * i);
-        s.empty[i] = smem_u32(bars + 8 * (kStages + i));
-    }
-    for (int i = 0; i < 2; ++i) {
-        s.tmem_full[i] = smem_u32(bars + 8 * (2 * kStages + i));
-        s.tmem_empty[i] = smem_u32(bars + 8 * (2 * kStages + 2 + i));
-    }
+    s.full0 = smem_u32(bars);
+    s.empty0 = smem_u32(bars + 8 * kStages);
+    s.tmem_full0 = smem_u32(bars + 8 * (2 * kStages));
+    s.tmem_empty0 = smem_u32(bars + 8 * (2 * kStages + 2));
     s.tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(bars + 8 * (2 * kStages + 4));
     s.tmem_slot = smem_u32(bars + 8 * (2 * kStages + 4));
     s.abort_flag = reinterpret_cast<volatile int*>(bars + 8 * (2 * kStages + 4) + 4);
-    for (int i = 0; i < 2 * kTnEpiWarps; ++i) s.skip_full[i] = smem_u32(bars + 8 * (2 * kStages + 5 + i));
+    s.skip_full0 = smem_u32(bars + 8 * (2 * kStages + 5));
     return s;
 }
 
@@ -212,14 +214,14 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* raw, int stages, int staging
 __device__ __forceinline__ uint32_t prologue(const Smem& s, int warp, int lane, int epilogue_threads) {
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) {
-            mbar_init(s.full[i], 1);
-            mbar_init(s.empty[i], 1);
+            mbar_init(s.full(i), 1);
+            mbar_init(s.empty(i), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(s.tmem_full[i], 1);
-            mbar_init(s.tmem_empty[i], epilogue_threads);
+            mbar_init(s.tmem_full(i), 1);
+            mbar_init(s.tmem_empty(i), epilogue_threads);
         }
-        for (int i = 0; i < 2 * kTnEpiWarps; ++i) mbar_init(s.skip_full[i], 1);
+        for (int i = 0; i < 2 * kTnEpiWarps; ++i) mbar_init(s.skip_full(i), 1);
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -282,7 +284,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
     uint8_t* stg_bytes = s.staging + (size_t)(warp - 2) * (tn_staging_bytes(kEpi) / kTnEpiWarps);
 
     if (kEpi == 0) {
-        if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
+        if (!mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag)) return false;
         tc_fence_after();
         float4* stg = reinterpret_cast<float4*>(stg_bytes);
 #pragma unroll
@@ -317,7 +319,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
     // ---- kEpi == 1, 2: the skip operand arrives by TMA
     const int w = warp - 2;
     uint8_t* skb = s.skipbuf + (size_t)w * 4096;   // two 2 KB skip tiles
-    const uint32_t sbar[2] = {s.skip_full[2 * w], s.skip_full[2 * w + 1]};
+    const uint32_t sbar[2] = {s.skip_full(2 * w), s.skip_full(2 * w + 1)};
     const int swz = (lane >> 1) & 3;               // 64-byte swizzle: chunk c of row `lane` sits at chunk c ^ swz
     auto fetch_skip = [&](int sl) {
         const int b = sl & 1;
@@ -328,7 +330,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         fetch_skip(0);
         if (kSlabs > 1) fetch_skip(1);
     }
-    if (!mbar_wait(s.tmem_full[acc], acc_phase, s.abort_flag)) return false;
+    if (!mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag)) return false;
     tc_fence_after();
     if (kEpi == 2) {
         // z = acc (hi + lo columns) goes out in fp32, skip * sigmoid(z) in bf16; one staging buffer each
@@ -444,11 +446,11 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
                 const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!(ok = mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag))) break;
-                    mbar_expect_tx(s.full[stage], kStageBytes);
+                    if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
+                    mbar_expect_tx(s.full(stage), kStageBytes);
                     const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
-                    tma_load_2d(a_dst, &tmA, s.full[stage], kb * BK, m0);
-                    tma_load_2d(a_dst + kABytes, &tmW, s.full[stage], kb * BK, n0);
+                    tma_load_2d(a_dst, &tmA, s.full(stage), kb * BK, m0);
+                    tma_load_2d(a_dst + kABytes, &tmW, s.full(stage), kb * BK, n0);
                     if (++stage == kTnStages) {
                         stage = 0;
                         phase ^= 1u;
@@ -463,11 +465,11 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-                if (!(ok = mbar_wait(s.tmem_empty[acc], acc_phase ^ 1u, s.abort_flag))) break;
+                if (!(ok = mbar_wait(s.tmem_empty(acc), acc_phase ^ 1u, s.abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                    if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageBytes);
                     const uint64_t adesc = smem_desc_kmajor(a_addr);
@@ -478,14 +480,14 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                         umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
                                   (uint32_t)((kb | k) != 0));
                     }
-                    umma_commit(s.empty[stage]);
+                    umma_commit(s.empty(stage));
                     if (++stage == kTnStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
                 }
                 if (!ok) break;
-                umma_commit(s.tmem_full[acc]);
+                umma_commit(s.tmem_full(acc));
                 if ((acc ^= 1) == 0) acc_phase ^= 1u;
             }
         }
@@ -499,7 +501,7 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                                     skip_phase)))
                 break;
             tc_fence_before();
-            mbar_arrive(s.tmem_empty[acc]);
+            mbar_arrive(s.tmem_empty(acc));
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
         }
         if (lane == 0) tma_store_wait_all();
@@ -539,14 +541,14 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     // barriers and tensor memory (both CTAs), then the whole pair meets
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) {
-            mbar_init(s.full[i], 1);
-            mbar_init(s.empty[i], 1);
+            mbar_init(s.full(i), 1);
+            mbar_init(s.empty(i), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(s.tmem_full[i], 1);
-            mbar_init(s.tmem_empty[i], 2 * 32 * kTnEpiWarps);
+            mbar_init(s.tmem_full(i), 1);
+            mbar_init(s.tmem_empty(i), 2 * 32 * kTnEpiWarps);
         }
-        for (int i = 0; i < 2 * kTnEpiWarps; ++i) mbar_init(s.skip_full[i], 1);
+        for (int i = 0; i < 2 * kTnEpiWarps; ++i) mbar_init(s.skip_full(i), 1);
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -567,8 +569,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         if (lane == 0) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmWh);
-            uint32_t leader_full[kPairStages];
-            for (int i = 0; i < kPairStages; ++i) leader_full[i] = map_to_cta(s.full[i], 0);
+            const uint32_t leader_full0 = map_to_cta(s.full(0), 0);   // (the leader's barriers are 8 bytes apart there too)
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -586,11 +587,11 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                 const int n0 = (tile % p.n_tiles) * BN + (int)rank * (BN / 2);
                 prefetch_a(tile + npairs);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!(ok = mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag))) break;
-                    if (rank == 0) mbar_expect_tx(s.full[stage], 2 * kPairStageBytes);
+                    if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
+                    if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kPairStageBytes);
                     const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
-                    tma_load_2d_pair(a_dst, &tmA, leader_full[stage], kb * BK, m0);
-                    tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full[stage], kb * BK, n0);
+                    tma_load_2d_pair(a_dst, &tmA, leader_full0 + 8u * stage, kb * BK, m0);
+                    tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full0 + 8u * stage, kb * BK, n0);
                     if (++stage == kPairStages) {
                         stage = 0;
                         phase ^= 1u;
@@ -605,11 +606,11 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = pair; tile < total && ok; tile += npairs) {
-                if (!(ok = mbar_wait(s.tmem_empty[acc], acc_phase ^ 1u, s.abort_flag))) break;
+                if (!(ok = mbar_wait(s.tmem_empty(acc), acc_phase ^ 1u, s.abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                    if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
                     const uint64_t adesc = smem_desc_kmajor(a_addr);
@@ -618,19 +619,19 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                     for (int k = 0; k < BK / UK; ++k)
                         umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
                                        (uint32_t)((kb | k) != 0));
-                    umma_commit_pair(s.empty[stage]);
+                    umma_commit_pair(s.empty(stage));
                     if (++stage == kPairStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
                 }
                 if (!ok) break;
-                umma_commit_pair(s.tmem_full[acc]);
+                umma_commit_pair(s.tmem_full(acc));
                 if ((acc ^= 1) == 0) acc_phase ^= 1u;
             }
         }
     } else {
-        const uint32_t leader_empty[2] = {map_to_cta(s.tmem_empty[0], 0), map_to_cta(s.tmem_empty[1], 0)};
+        const uint32_t leader_empty0 = map_to_cta(s.tmem_empty(0), 0);
         int acc = 0;
         uint32_t acc_phase = 0, skip_phase = 0;
         bool ok = true;
@@ -640,7 +641,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                                                     skip_phase)))
                 break;
             tc_fence_before();
-            mbar_arrive_cluster(leader_empty[acc]);
+            mbar_arrive_cluster(leader_empty0 + 8u * acc);
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
         }
         if (lane == 0) tma_store_wait_all();
@@ -738,12 +739,12 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const uint32_t rank = cluster_ctarank();
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) {
-            mbar_init(s.full[i], 1);
-            mbar_init(s.empty[i], 1);
+            mbar_init(s.full(i), 1);
+            mbar_init(s.empty(i), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(s.tmem_full[i], 1);
-            mbar_init(s.tmem_empty[i], 2 * kFsEpiThreads);
+            mbar_init(s.tmem_full(i), 1);
+            mbar_init(s.tmem_empty(i), 2 * kFsEpiThreads);
         }
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -756,8 +757,6 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *s.tmem_slot_ptr;
-    // the barriers of a kind are 8 bytes apart: addresses by arithmetic, so that no array is indexed at run time
-    const uint32_t full0 = s.full[0], empty0 = s.empty[0], tfull0 = s.tmem_full[0], tempty0 = s.tmem_empty[0];
 
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int M = p.B * p.T;
@@ -781,9 +780,9 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const int m0 = row_of(chain, tb);
                     // (no L2 prefetch of the next tile's rows here: with it the kernel ran 7 % slower)
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!(ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, s.abort_flag))) break;
-                        const uint32_t leader_full = map_to_cta(full0 + 8u * stage, 0);
-                        if (rank == 0) mbar_expect_tx(full0 + 8u * stage, 2 * kPairStageBytes);
+                        if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
+                        const uint32_t leader_full = map_to_cta(s.full(stage), 0);
+                        if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kPairStageBytes);
                         const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
                         tma_load_2d_pair(a_dst, &tmA, leader_full, kb * BK, m0);
                         tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full, kb * BK, n0);
@@ -803,11 +802,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             bool ok = true;
             for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
                 for (int tb = 0; tb < p.tblocks && ok; ++tb) {
-                    if (!(ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, s.abort_flag))) break;
+                    if (!(ok = mbar_wait(s.tmem_empty(acc), acc_phase ^ 1u, s.abort_flag))) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!(ok = mbar_wait(full0 + 8u * stage, phase, s.abort_flag))) break;
+                        if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                         tc_fence_after();
                         const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
                         const uint64_t adesc = smem_desc_kmajor(a_addr);
@@ -816,20 +815,20 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         for (int k = 0; k < BK / UK; ++k)
                             umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
                                            (uint32_t)((kb | k) != 0));
-                        umma_commit_pair(empty0 + 8u * stage);
+                        umma_commit_pair(s.empty(stage));
                         if (++stage == kPairStages) {
                             stage = 0;
                             phase ^= 1u;
                         }
                     }
                     if (!ok) break;
-                    umma_commit_pair(tfull0 + 8u * acc);
+                    umma_commit_pair(s.tmem_full(acc));
                     if ((acc ^= 1) == 0) acc_phase ^= 1u;
                 }
             }
         }
     } else {
-        const uint32_t leader_empty0 = map_to_cta(tempty0, 0);
+        const uint32_t leader_empty0 = map_to_cta(s.tmem_empty(0), 0);
         constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
         const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
         const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
@@ -877,7 +876,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const uint32_t mk = __ballot_sync(0xffffffffu, f);
                     if (lane == 0) masks[te >> 5] = mk;
                 }
-                (void)mbar_wait(tfull0 + 8u * acc, acc_phase, s.abort_flag);
+                (void)mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag);
                 if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
                 epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
                               // the 256 threads leave together or not at all
@@ -1080,16 +1079,16 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!mbar_wait(s.empty[stage], phase ^ 1u, s.abort_flag)) break;
-                mbar_expect_tx(s.full[stage], kStageBytes);
+                if (!mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag)) break;
+                mbar_expect_tx(s.full(stage), kStageBytes);
                 const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
                 const int row = (kb0 + kb) * BK;
 #pragma unroll
-                for (int h = 0; h < BM / 64; ++h) tma_load_2d(a_dst + h * (BK * 128), &tmA, s.full[stage], i0 + 64 * h, row);
+                for (int h = 0; h < BM / 64; ++h) tma_load_2d(a_dst + h * (BK * 128), &tmA, s.full(stage), i0 + 64 * h, row);
 #pragma unroll
                 for (int h = 0; h < kOutCols / 64; ++h) {
-                    tma_load_2d(a_dst + kABytes + h * (BK * 128), &tmBhi, s.full[stage], j0 + 64 * h, row);
-                    tma_load_2d(a_dst + kABytes + (kOutCols / 64 + h) * (BK * 128), &tmBlo, s.full[stage],
+                    tma_load_2d(a_dst + kABytes + h * (BK * 128), &tmBhi, s.full(stage), j0 + 64 * h, row);
+                    tma_load_2d(a_dst + kABytes + (kOutCols / 64 + h) * (BK * 128), &tmBlo, s.full(stage),
                                 j0 + 64 * h, row);
                 }
                 if (++stage == kStages) {
@@ -1105,7 +1104,7 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             uint32_t phase = 0;
             bool ok = true;
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!(ok = mbar_wait(s.full[stage], phase, s.abort_flag))) break;
+                if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                 tc_fence_after();
                 const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageBytes);
                 const uint64_t adesc = smem_desc_mnmajor(a_addr);
@@ -1116,13 +1115,13 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     umma_bf16(tmem_base, adesc + (uint64_t)(128 * k), bdesc + (uint64_t)(128 * k), idesc,
                               (uint32_t)((kb | k) != 0));
                 }
-                umma_commit(s.empty[stage]);
+                umma_commit(s.empty(stage));
                 if (++stage == kStages) {
                     stage = 0;
                     phase ^= 1u;
                 }
             }
-            if (ok) umma_commit(s.tmem_full[0]);
+            if (ok) umma_commit(s.tmem_full(0));
         }
     } else {
         const int q = warp & 3;
@@ -1130,7 +1129,7 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         float* dst_row = p.part + ((size_t)split * p.I + row) * p.J + j0;
         bool ok = true;
         if (nkb > 0) {
-            ok = mbar_wait(s.tmem_full[0], 0, s.abort_flag);
+            ok = mbar_wait(s.tmem_full(0), 0, s.abort_flag);
             tc_fence_after();
         }
         if (ok) {
