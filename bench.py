@@ -37,6 +37,7 @@ STAGE_MODEL = {
     # input projection and forward scan in one kernel: the contraction is what it has to do (the scan
     # adds 8 flop per state and step and no HBM traffic)
     "gemm_Bu_scan_fwd": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "gemm_gx_scan_bwd": ("tensor", lambda H, P, s: 4.0 * H * P),
     "gemm_Bu": ("tensor", lambda H, P, s: 4.0 * H * P),
     "scan_fwd": ("hbm", lambda H, P, s: 16.0 * P),
     "gemm_y": ("tensor", lambda H, P, s: 4.0 * H * P),
@@ -54,6 +55,7 @@ STAGE_MODEL = {
 # once its kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_TIMESTEP = {
     "gemm_Bu_scan_fwd": 777.8e6 / 262144,
+    "gemm_gx_scan_bwd": None,
     "scan_fwd": 1021.7e6 / 262144,
     "scan_bwd": 1579.9e6 / 262144,
     "gemm_Bu": 763.6e6 / 262144,

@@ -179,7 +179,8 @@ static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
                       at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
     if (p.tc)
         // (the kernel that scans in the epilogue of the projection wants its own column order)
-        launch_pack_operands_tc(s.H, s.P, tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P), at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+        launch_pack_operands_tc(s.H, s.P, tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P),
+                                tc_gemm_scan_bwd_supported(s.B, s.T, s.H, s.P), at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
                                 at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
     else
         launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
@@ -459,18 +460,26 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
     int rc = SSM_OK;
 
     if (p.tc) {
-        {   // gx[m, 2p+c] = sum_h gy[m,h] conj(C)_c[h,p]   (weights as hi + lo bf16)
-            StageTimer tm("gemm_gx", st);
-            GemmTcTN g{gy, at<void>(ws, p.W1), BT, P2, s.H, true, true, at<void>(ws, p.f32buf), nullptr, nullptr, hdr};
-            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
-        }
-        {
-            StageTimer tm("scan_bwd", st);
-            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done, (const float2*)x0,
-                                 at<void>(ws, p.xs), true, at<float2>(ws, p.f32buf), (const float2*)gxT,
-                                 at<void>(ws, p.gs), true, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
-                                 at<char>(ws, p.scan), st);
-            if (rc) return rc;
+        if (tc_gemm_scan_bwd_supported(s.B, s.T, s.H, s.P)) {
+            // projection and reverse scan in one kernel: s = reverse scan(gy conj(C)), g_x stays on chip
+            StageTimer tm("gemm_gx_scan_bwd", st);
+            GemmScanBwd g{gy, at<void>(ws, p.W1), s.B, s.T, s.H, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
+                          (const float2*)gxT, at<void>(ws, p.xs), at<void>(ws, p.gs), nullptr, (float2*)dx0, hdr};
+            if ((rc = launch_gemm_scan_bwd_sum(g, at<float2>(ws, p.gAbar), at<char>(ws, p.scan), st))) return rc;
+        } else {
+            {   // gx[m, 2p+c] = sum_h gy[m,h] conj(C)_c[h,p]   (weights as hi + lo bf16)
+                StageTimer tm("gemm_gx", st);
+                GemmTcTN g{gy, at<void>(ws, p.W1), BT, P2, s.H, true, true, at<void>(ws, p.f32buf), nullptr, nullptr, hdr};
+                if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+            }
+            {
+                StageTimer tm("scan_bwd", st);
+                rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done,
+                                     (const float2*)x0, at<void>(ws, p.xs), true, at<float2>(ws, p.f32buf),
+                                     (const float2*)gxT, at<void>(ws, p.gs), true, at<float2>(ws, p.gAbar), (float2*)dx0,
+                                     hdr, at<char>(ws, p.scan), st);
+                if (rc) return rc;
+            }
         }
         {   // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]
             StageTimer tm("gemm_du", st);

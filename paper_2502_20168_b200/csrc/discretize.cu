@@ -146,11 +146,11 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* W, int H, int n, int 
     W[(r + 128) * H + h] = lo;
 }
 
-// pair_cols: the rows of the Bbar operand are ordered so that the accumulator columns of two
+// pair_cols (Bbar operand), pair_cols_C (conj(C) operand): the rows of the operand are ordered so that the accumulator columns of two
 // neighbouring states come out as (re, re, im, im): the kernel that scans the accumulators in its
 // epilogue advances two states per packed instruction.  State p, component c -> row
 // (p / 64) * 128 + 4 * ((p % 64) / 2) + 2 * c + p % 2 of the [2P, H] operand.
-__global__ void pack_operands_tc_kernel(int H, int P, bool pair_cols, const float2* __restrict__ Bbar, const float2* __restrict__ Cc,
+__global__ void pack_operands_tc_kernel(int H, int P, bool pair_cols, bool pair_cols_C, const float2* __restrict__ Bbar, const float2* __restrict__ Cc,
                                         __nv_bfloat16* __restrict__ WsB, __nv_bfloat16* __restrict__ WsC,
                                         __nv_bfloat16* __restrict__ Cp, __nv_bfloat16* __restrict__ Bq) {
     const size_t n = (size_t)P * H;
@@ -169,18 +169,19 @@ __global__ void pack_operands_tc_kernel(int H, int P, bool pair_cols, const floa
             const float2 v = Cc[i];
             Cp[(size_t)h * 2 * P + 2 * p] = __float2bfloat16_rn(v.x);
             Cp[(size_t)h * 2 * P + 2 * p + 1] = __float2bfloat16_rn(-v.y);
-            store_split(WsC, H, 2 * p, h, v.x);
-            store_split(WsC, H, 2 * p + 1, h, -v.y);
+            const int n = pair_cols_C ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
+            store_split(WsC, H, n, h, v.x);
+            store_split(WsC, H, n + (pair_cols_C ? 2 : 1), h, -v.y);
         }
     }
 }
 
-void launch_pack_operands_tc(int H, int P, bool pair_cols, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
+void launch_pack_operands_tc(int H, int P, bool pair_cols, bool pair_cols_C, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st) {
     const int threads = 256;
     const int blocks = (int)(((size_t)P * H + threads - 1) / threads);
     count_launch();
-    pack_operands_tc_kernel<<<blocks, threads, 0, st>>>(H, P, pair_cols, Bbar, Cc, (__nv_bfloat16*)Wsplit_B,
+    pack_operands_tc_kernel<<<blocks, threads, 0, st>>>(H, P, pair_cols, pair_cols_C, Bbar, Cc, (__nv_bfloat16*)Wsplit_B,
                                                         (__nv_bfloat16*)Wsplit_C, (__nv_bfloat16*)Cp,
                                                         (__nv_bfloat16*)Bq);
 }

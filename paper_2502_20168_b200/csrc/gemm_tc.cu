@@ -1044,6 +1044,393 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------
+// g_x projection and reverse scan in one kernel (CTA pairs)
+// ---------------------------------------------------------------------------------------------
+// s_t = g_x,t + keep_{t+1} conj(Abar) s_{t+1} without g_x ever reaching HBM, and the sums
+// gAbar = sum_t keep_t s_t conj(x_{t-1}).  The kernel is gemm_scan_fwd_kernel run backwards: a CTA
+// walks the tiles of a chain from the last to the first, the last row group starts from the carried
+// value, rows are folded from the last to the first, and the reset that acts between rows i and
+// i + 1 is the flag of row i + 1.  What is new is x_{t-1}: once a warp has its 16 rows of g_x in
+// registers, its part of the shared-memory tile is free, and one lane has the TMA unit copy the
+// rows m - 1 ... m + 14 of both planes of x there (one row early; the row before a sequence's first
+// is replaced by x0).  In the second pass a thread reads its two states' x_{t-1}, adds
+// s_t conj(x_{t-1}) to its sums and writes the hi / lo halves of s_t to the same place, which
+// then leaves through the TMA unit as in the forward kernel.  The sums stay in registers for the
+// whole chain and are added over the row groups at its end: one entry of gA_part per (sequence,
+// state), each written once.  T must be a multiple of 128.
+struct FbParams {
+    int B, T, P;
+    int n_tiles;      // 2P / 128
+    int k_blocks;     // H / 64
+    int tblocks;      // T / 128
+    int nchains;      // n_tiles * ceil(B / 2)
+    const float2* Abar;
+    const uint8_t* done;
+    const float2* x0;     // [B, P] or NULL
+    const float2* gxT;    // [B, P] or NULL
+    float2* gA_part;      // [B, P]
+    float2* gx0;          // [B, P] or NULL
+    WsHeader* hdr;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFsThreads, 1)
+gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
+                     const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmS, FbParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ float4 agg_e[kFsEpiThreads], carry_s[32];   // (re, re, im, im) of two neighbouring states
+    __shared__ uint32_t masks[8];   // [0, 4): flags of the rows one later (the resets of the reverse scan); [4, 8): of the rows
+    __shared__ __align__(8) uint64_t xbar[kFsEpiWarps];   // one per warp: its rows of x have arrived
+    const Smem s = carve_smem(smem_raw, kPairStages, kFsTileBytes, 0, kPairStageBytes, 0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(s.full(i), 1);
+            mbar_init(s.empty(i), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s.tmem_full(i), 1);
+            mbar_init(s.tmem_empty(i), 2 * kFsEpiThreads);
+        }
+        for (int i = 0; i < kFsEpiWarps; ++i) mbar_init(smem_u32(&xbar[i]), 1);
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x < 8) masks[threadIdx.x] = 0u;
+    __syncwarp();
+    if (warp == 1) tmem_alloc_pair(s.tmem_slot, kTmemCols);
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *s.tmem_slot_ptr;
+
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int M = p.B * p.T;
+    auto seq_of = [&](int chain) { return 2 * (chain / p.n_tiles) + (int)rank; };
+    auto row_of = [&](int chain, int tb) {
+        const int b = seq_of(chain);
+        return b < p.B ? b * p.T + tb * BM : M;   // no sequence (odd B): rows past the end read as zero
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmWh);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
+                const int n0 = (chain % p.n_tiles) * BN + (int)rank * (BN / 2);
+                for (int tb = p.tblocks - 1; tb >= 0 && ok; --tb) {
+                    const int m0 = row_of(chain, tb);
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
+                        const uint32_t leader_full = map_to_cta(s.full(stage), 0);
+                        if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kPairStageBytes);
+                        const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        tma_load_2d_pair(a_dst, &tmA, leader_full, kb * BK, m0);
+                        tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full, kb * BK, n0);
+                        if (++stage == kPairStages) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = instr_desc(2 * BM, BN, 0, 0);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
+                for (int tb = 0; tb < p.tblocks && ok; ++tb) {
+                    if (!(ok = mbar_wait(s.tmem_empty(acc), acc_phase ^ 1u, s.abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
+                        tc_fence_after();
+                        const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        const uint64_t adesc = smem_desc_kmajor(a_addr);
+                        const uint64_t bdesc = smem_desc_kmajor(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < BK / UK; ++k)
+                            umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                           (uint32_t)((kb | k) != 0));
+                        umma_commit_pair(s.empty(stage));
+                        if (++stage == kPairStages) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                    if (!ok) break;
+                    umma_commit_pair(s.tmem_full(acc));
+                    if ((acc ^= 1) == 0) acc_phase ^= 1u;
+                }
+            }
+        }
+    } else {
+        const uint32_t leader_empty0 = map_to_cta(s.tmem_empty(0), 0);
+        constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
+        const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
+        const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
+        const int sp = te & 31, sl = te >> 5;       // scan role: pair of states of the tile, group of its rows
+        const int prow = q * 32 + lane;             // drain role: row of the tile
+        const bool from_carry = sl == nsl - 1;      // the last rows come first
+        float4* T4 = reinterpret_cast<float4*>(s.staging);
+        uint8_t* warp_buf = s.staging + sl * (2 * R * 256);   // this warp's rows of the tile; later x_{t-1}, then s
+        uint2* xs = reinterpret_cast<uint2*>(warp_buf) + sp;
+        const uint32_t xb = smem_u32(&xbar[sl]);
+        uint32_t xphase = 0;
+        const C2 zero = {0ull, 0ull};
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
+            const int n_tile = chain % p.n_tiles, b = seq_of(chain);
+            const bool has_seq = b < p.B;
+            const int pg = n_tile * 64 + 2 * sp;    // the first of this thread's two states
+            const float2 a0 = cconj(p.Abar[pg]), a1 = cconj(p.Abar[pg + 1]);
+            const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
+            f32x2 pr, pi, npi;   // conj(Abar)^R by squaring in fp32
+            {
+                float re0 = a0.x, im0 = a0.y, re1 = a1.x, im1 = a1.y;
+#pragma unroll
+                for (int n = 1; n < R; n *= 2) {
+                    const float r0 = fmaf(re0, re0, -im0 * im0), i0 = 2.f * re0 * im0;
+                    const float r1 = fmaf(re1, re1, -im1 * im1), i1 = 2.f * re1 * im1;
+                    re0 = r0, im0 = i0, re1 = r1, im1 = i1;
+                }
+                pr = pack2(re0, re1);
+                pi = pack2(im0, im1);
+                npi = pack2(-im0, -im1);
+            }
+            C2 g = zero;        // this thread's part of the chain's sums s_t conj(x_{t-1})
+            C2 xinit = zero;    // x0: what stands before the sequence's first row
+            if (sl == 0 && p.x0 && has_seq) {
+                const float2 c0 = p.x0[(size_t)b * p.P + pg], c1 = p.x0[(size_t)b * p.P + pg + 1];
+                xinit.re = pack2(c0.x, c1.x);
+                xinit.im = pack2(c0.y, c1.y);
+            }
+            if (from_carry) carry_s[sp] = make_float4(0.f, 0.f, 0.f, 0.f);   // nothing follows the last row
+            for (int tb = p.tblocks - 1; tb >= 0; --tb) {
+                const int m0 = row_of(chain, tb);
+                if (p.done && te < BM) {
+                    const bool f0 = has_seq && p.done[(size_t)m0 + te] != 0;
+                    const bool f1 = has_seq && tb * BM + te + 1 < p.T && p.done[(size_t)m0 + te + 1] != 0;
+                    const uint32_t mk0 = __ballot_sync(0xffffffffu, f0), mk1 = __ballot_sync(0xffffffffu, f1);
+                    if (lane == 0) {
+                        masks[te >> 5] = mk1;
+                        masks[4 + (te >> 5)] = mk0;
+                    }
+                }
+                (void)mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag);
+                if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
+                epi_sync();   // flags visible, tile free; also: the 256 threads leave together or not at all
+                if (*s.abort_flag) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7)
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll
+                for (int gq = grp; gq < 4; gq += kFsEpiWarps / 4) {   // 32 columns = one 128-byte group of the row
+                    uint32_t r[32], r2[32];
+                    tmem_ld32(t_row + (uint32_t)(gq * 32), r);
+                    tmem_ld32(t_row + (uint32_t)(BN / 2 + gq * 32), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        T4[prow * 32 + gq * 8 + (j ^ (prow & 7))] =
+                            make_float4(__uint_as_float(r[4 * j]) + __uint_as_float(r2[4 * j]),
+                                        __uint_as_float(r[4 * j + 1]) + __uint_as_float(r2[4 * j + 1]),
+                                        __uint_as_float(r[4 * j + 2]) + __uint_as_float(r2[4 * j + 2]),
+                                        __uint_as_float(r[4 * j + 3]) + __uint_as_float(r2[4 * j + 3]));
+                }
+                tc_fence_before();
+                mbar_arrive_cluster(leader_empty0 + 8u * acc);
+                if ((acc ^= 1) == 0) acc_phase ^= 1u;
+                epi_sync();
+                // (2) this thread's two states over its R rows, last row first
+                const int r0 = sl * R;
+                uint32_t gflags = 0;   // bit g: a reset acts inside or right after row group g
+                uint32_t mask = 0u, mask0 = 0u;
+                if (p.done) {
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const uint32_t mk = masks[w];
+#pragma unroll
+                        for (int h = 0; h < 32 / R; ++h)
+                            if ((mk >> (h * R)) & ((1u << R) - 1u)) gflags |= 1u << (w * (32 / R) + h);
+                    }
+                    mask = (masks[r0 >> 5] >> (r0 & 31)) & ((1u << R) - 1u);
+                    mask0 = (masks[4 + (r0 >> 5)] >> (r0 & 31)) & ((1u << R) - 1u);
+                }
+                C2 v[R];
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const int row = r0 + i;
+                    const float4 t = T4[row * 32 + ((sp & ~7) | ((sp & 7) ^ (row & 7)))];   // (re, re, im, im)
+                    v[i].re = pack2(t.x, t.y);
+                    v[i].im = pack2(t.z, t.w);
+                }
+                if (from_carry && tb == p.tblocks - 1 && p.gxT && has_seq) {   // the gradient of the final state
+                    const float2 c0 = p.gxT[(size_t)b * p.P + pg], c1 = p.gxT[(size_t)b * p.P + pg + 1];
+                    float v0, v1, v2, v3;
+                    unpack2(v[R - 1].re, v0, v1);
+                    unpack2(v[R - 1].im, v2, v3);
+                    v[R - 1].re = pack2(v0 + c0.x, v1 + c1.x);
+                    v[R - 1].im = pack2(v2 + c0.y, v3 + c1.y);
+                }
+                // the warp has its rows: rows m - 1 ... m + R - 2 of x (both planes) into its part of the tile
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_expect_tx(xb, 2 * R * 256);
+                    tma_load_3d(smem_u32(warp_buf), &tmX, xb, n_tile * 64, m0 + r0 - 1, 0);
+                }
+                C2 e = zero;
+                if (from_carry) {   // from the carried value: these results are final
+                    const float4 c = carry_s[sp];
+                    C2 x = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                    if (mask == 0u) {
+#pragma unroll
+                        for (int i = R - 1; i >= 0; --i) v[i] = x = cstep2(ar, ai, nai, x, v[i]);
+                    } else {
+#pragma unroll
+                        for (int i = R - 1; i >= 0; --i) {
+                            if ((mask >> i) & 1u) x = zero;
+                            v[i] = x = cstep2(ar, ai, nai, x, v[i]);
+                        }
+                    }
+                    e = x;
+                } else if (mask == 0u) {
+#pragma unroll
+                    for (int i = R - 1; i >= 0; --i) e = cstep2(ar, ai, nai, e, v[i]);
+                } else {
+#pragma unroll
+                    for (int i = R - 1; i >= 0; --i) {
+                        if ((mask >> i) & 1u) e = zero;
+                        e = cstep2(ar, ai, nai, e, v[i]);
+                    }
+                }
+                {
+                    float e0, e1, e2, e3;
+                    unpack2(e.re, e0, e1);
+                    unpack2(e.im, e2, e3);
+                    agg_e[te] = make_float4(e0, e1, e2, e3);
+                }
+                epi_sync();   // group results visible
+                C2 x = e;
+                if (!from_carry) {   // s of the row after this group's last
+                    {
+                        const float4 c = agg_e[(nsl - 1) * 32 + sp];
+                        x.re = pack2(c.x, c.y);
+                        x.im = pack2(c.z, c.w);
+                    }
+#pragma unroll
+                    for (int gq = nsl - 2; gq >= 1; --gq) {
+                        if (gq > sl) {
+                            const float4 c = agg_e[gq * 32 + sp];
+                            const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                            x = ((gflags >> gq) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
+                        }
+                    }
+                }
+                // (3) fold again, with x_{t-1} at hand: sums for gAbar, s as hi / lo bf16 halves in place of x
+                if (!mbar_wait(xb, xphase, s.abort_flag)) {
+                    // (the wait gave up: the flag is set, everybody leaves at the next barrier)
+                }
+                xphase ^= 1u;
+                const bool seq_start = tb == 0 && sl == 0;   // row 0 of this group is the sequence's first row
+#pragma unroll
+                for (int i = R - 1; i >= 0; --i) {
+                    C2 sv = v[i];
+                    if (!from_carry) {
+                        if ((mask >> i) & 1u) x = zero;
+                        sv = x = cstep2(ar, ai, nai, x, v[i]);
+                    }
+                    float re0, re1, im0, im1;
+                    unpack2(sv.re, re0, re1);
+                    unpack2(sv.im, im0, im1);
+                    if (!((mask0 >> i) & 1u)) {
+                        C2 xp;
+                        if (seq_start && i == 0) {
+                            xp = xinit;
+                        } else {
+                            const uint2 xh = xs[i * 32], xl = xs[(R + i) * 32];
+                            xp.re = pack2(__uint_as_float(xh.x << 16) + __uint_as_float(xl.x << 16),
+                                          __uint_as_float(xh.y << 16) + __uint_as_float(xl.y << 16));
+                            xp.im = pack2(__uint_as_float(xh.x & 0xffff0000u) + __uint_as_float(xl.x & 0xffff0000u),
+                                          __uint_as_float(xh.y & 0xffff0000u) + __uint_as_float(xl.y & 0xffff0000u));
+                        }
+                        // g += s conj(x):  re += s.re x.re + s.im x.im,  im += s.im x.re - s.re x.im
+                        g.re = fma2(sv.re, xp.re, fma2(sv.im, xp.im, g.re));
+                        g.im = fma2(sv.im, xp.re, fma2(sv.re, xp.im ^ 0x8000000080000000ull, g.im));
+                    }
+                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(re0, im0), h1 = __floats2bfloat162_rn(re1, im1);
+                    const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+                    const __nv_bfloat162 l0 = __floats2bfloat162_rn(re0 - f0.x, im0 - f0.y);
+                    const __nv_bfloat162 l1 = __floats2bfloat162_rn(re1 - f1.x, im1 - f1.y);
+                    xs[i * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                    xs[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0 && has_seq) {
+                    tma_store_3d_nocommit(&tmS, smem_u32(warp_buf), n_tile * 64, m0 + r0, 0);
+                    tma_commit_group();
+                }
+                if (sl == 0) {   // x is s of the tile's first row
+                    float x0r, x1r, x0i, x1i;
+                    unpack2(x.re, x0r, x1r);
+                    unpack2(x.im, x0i, x1i);
+                    if (tb > 0) {
+                        carry_s[sp] = make_float4(x0r, x1r, x0i, x1i);
+                    } else if (p.gx0 && has_seq) {   // what reaches the initial state: keep_0 conj(Abar) s_0
+                        const bool cut = (mask0 & 1u) != 0u;
+                        const float2 z = make_float2(0.f, 0.f);
+                        p.gx0[(size_t)b * p.P + pg] = cut ? z : cfma(a0, make_float2(x0r, x0i), z);
+                        p.gx0[(size_t)b * p.P + pg + 1] = cut ? z : cfma(a1, make_float2(x1r, x1i), z);
+                    }
+                }
+            }
+            if (!ok) break;
+            // the chain's sums over the row groups (agg_e is free: everybody is past the last tile's join)
+            epi_sync();
+            {
+                float g0, g1, g2, g3;
+                unpack2(g.re, g0, g1);
+                unpack2(g.im, g2, g3);
+                agg_e[te] = make_float4(g0, g1, g2, g3);
+            }
+            epi_sync();
+            if (sl == 0 && has_seq) {
+                float4 sum = agg_e[sp];
+#pragma unroll
+                for (int gq = 1; gq < nsl; ++gq) {
+                    const float4 c = agg_e[gq * 32 + sp];
+                    sum.x += c.x, sum.y += c.y, sum.z += c.z, sum.w += c.w;
+                }
+                p.gA_part[(size_t)b * p.P + pg] = make_float2(sum.x, sum.z);
+                p.gA_part[(size_t)b * p.P + pg + 1] = make_float2(sum.y, sum.w);
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+    }
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync_all();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+    if (threadIdx.x == 0 && *s.abort_flag && p.hdr) p.hdr->status = SSM_ERR_TIMEOUT;
+}
+
+// ---------------------------------------------------------------------------------------------
 // NT kernel (weight gradients): one 128 x 256 output tile and one slice of the rows per CTA
 // ---------------------------------------------------------------------------------------------
 struct NtParams {
@@ -1300,6 +1687,19 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
 
+// The two bf16 planes of a state tensor as [2, B*T, P] 32-bit words, in boxes of 64 states x kFsRows rows x both planes.
+static bool make_plane_map(CUtensorMap* map, const void* planes, int M, int P) {
+    PFN_cuTensorMapEncodeTiled fn = tc::encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)M, 2};
+    cuuint64_t strides[2] = {(cuuint64_t)P * 4, (cuuint64_t)M * P * 4};
+    cuuint32_t box[3] = {64, (cuuint32_t)tc::kFsRows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(planes), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Chains per 64 states: the sequences, or, when a 128-row tile holds several whole sequences, the tiles.
 static int fs_units(int B, int T) { return T >= tc::BM ? B : (B * T + tc::BM - 1) / tc::BM; }
 
@@ -1316,17 +1716,7 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
     CUtensorMap ma, mw, mx;
     if (!make_map(&ma, g.u, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
     if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
-    {   // the two planes of x as [2, B*T, P] 32-bit words; a warp stores 64 states x its rows x both planes
-        PFN_cuTensorMapEncodeTiled fn = encode_fn();
-        if (!fn) return SSM_ERR_CUDA;
-        cuuint64_t dims[3] = {(cuuint64_t)g.P, (cuuint64_t)M, 2};
-        cuuint64_t strides[2] = {(cuuint64_t)g.P * 4, (cuuint64_t)M * g.P * 4};
-        cuuint32_t box[3] = {64, (cuuint32_t)kFsRows, 2};
-        cuuint32_t estr[3] = {1, 1, 1};
-        if (fn(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, g.x_planes, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return SSM_ERR_CUDA;
-    }
+    if (!make_plane_map(&mx, g.x_planes, M, g.P)) return SSM_ERR_CUDA;
     const int units = fs_units(g.B, g.T);
     FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
                g.T >= BM ? BM / kFsRows : g.T / kFsRows, (P2 / 128) * ((units + 1) / 2),
@@ -1337,6 +1727,30 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
     const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), kFsSmemBytes, kFsThreads);
     if (pairs <= 0) return SSM_ERR_CUDA;
     kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, mx, p);
+    return SSM_OK;
+}
+
+bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) {
+    if (T % tc::BM != 0 || H % tc::BK != 0 || P % 64 != 0) return false;
+    return (2 * P / 128) * ((B + 1) / 2) >= tc::sm_count() / 2;   // a chain for every CTA pair
+}
+
+int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {
+    using namespace tc;
+    if (!tc_gemm_scan_bwd_supported(g.B, g.T, g.H, g.P)) return SSM_ERR_SHAPE;
+    const int M = g.B * g.T, P2 = 2 * g.P;
+    CUtensorMap ma, mw, mx, ms;
+    if (!make_map(&ma, g.gy, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
+    if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
+    if (!make_plane_map(&mx, g.x_planes, M, g.P) || !make_plane_map(&ms, g.s_planes, M, g.P)) return SSM_ERR_CUDA;
+    FbParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T / BM, (P2 / 128) * ((g.B + 1) / 2),
+               g.Abar, g.done, g.x0, g.gxT, g.gA_part, g.gx0, g.hdr};
+    count_launch();
+    auto kern = gemm_scan_bwd_kernel;
+    if (!set_smem(kern, kFsSmemBytes)) return SSM_ERR_CUDA;
+    const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), kFsSmemBytes, kFsThreads);
+    if (pairs <= 0) return SSM_ERR_CUDA;
+    kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, mx, ms, p);
     return SSM_OK;
 }
 

@@ -112,6 +112,28 @@ struct GemmScanFwd {
 bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P);
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st);
 
+// g_x projection and reverse scan fused (gemm_tc.cu): s = reverse scan(gy conj(C)) written as the two
+// bf16 planes of s, the sums s_t conj(x_{t-1}) per (sequence, state) in gA_part; g_x never reaches
+// memory.  T must be a multiple of 128, with enough chains (tc_gemm_scan_bwd_supported).
+struct GemmScanBwd {
+    const void* gy;         // bf16 [B*T, H]
+    const void* Wsplit;     // hi/lo stacked conj(C) operand [4P, H], rows in the pair_cols order
+    int B, T, H, P;
+    const float2* Abar;     // [P]
+    const uint8_t* done;    // [B*T] or NULL
+    const float2* x0;       // [B, P] or NULL
+    const float2* gxT;      // [B, P] or NULL
+    const void* x_planes;   // bf16 hi plane [B*T, 2P], then the lo plane
+    void* s_planes;         // out: the same layout
+    float2* gA_part;        // out [B, P]
+    float2* gx0;            // out [B, P] or NULL
+    WsHeader* hdr;
+};
+bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P);
+int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st);
+// scan.cu: the same followed by the sum of gA_part over the sequences (scratch as for launch_scan_bwd)
+int launch_gemm_scan_bwd_sum(GemmScanBwd g, float2* gAbar, void* scratch, cudaStream_t st);
+
 struct GemmTcNT {
     // part[s, i, j] = sum_{m in slice s} A[m, i] * (Bm_hi[m, j] + Bm_lo[m, j]);  A bf16 [K, I],
     // Bm_hi / Bm_lo bf16 [K, J]: the two planes of a state tensor
@@ -128,7 +150,7 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 
 // discretize.cu: operands of the tensor-core path (bf16).  Wsplit_B / Wsplit_C: [4P, H] hi/lo
 // stacked forms of Bp / Cq (see GemmTcTN);  Cp, Bq: [H, 2P] single bf16.
-void launch_pack_operands_tc(int H, int P, bool pair_cols, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
+void launch_pack_operands_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st);
 
 // glu.cu: what surrounds the GEMMs of the half-GLU gate out = v * sigmoid(GELU(v) W).

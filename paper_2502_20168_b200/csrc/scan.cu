@@ -360,4 +360,15 @@ int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
     return SSM_OK;
 }
 
+int launch_gemm_scan_bwd_sum(GemmScanBwd g, float2* gAbar, void* scratch, cudaStream_t st) {
+    const ScanPlan s = plan_scan(g.B, g.P);
+    char* base = (char*)scratch;
+    float* part = reinterpret_cast<float*>(base + s.off_part);
+    float* tmp = reinterpret_cast<float*>(base + s.off_tmp);
+    g.gA_part = reinterpret_cast<float2*>(part);
+    if (int rc = launch_gemm_scan_bwd(g, st)) return rc;
+    launch_colsum(part, g.B, 2 * g.P, (float*)gAbar, tmp, st);
+    return SSM_OK;
+}
+
 }  // namespace ssm
