@@ -1292,6 +1292,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 if (lane == 0) {
                     mbar_expect_tx(xb, 2 * R * 256);
                     tma_load_3d(smem_u32(warp_buf), &tmX, xb, n_tile * 64, m0 + r0 - 1, 0);
+                    // and the same rows of the tile before this one into L2, where the next load will find them
+                    if (tb > 0) tma_prefetch_3d(&tmX, n_tile * 64, m0 - BM + r0 - 1, 0);
                 }
                 C2 e = zero;
                 if (from_carry) {   // from the carried value: these results are final
