@@ -31,21 +31,22 @@ UNIT = "timesteps/s"
 DEFAULT_WORKLOAD = "c4_sweep_T1024_bf16"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# Algorithmic work of each internal stage per timestep (one (b,t) row): bytes for the
-# HBM-bound scans, flops for the projections (a real GEMM with K*N = 2*H*P per row).
+# Algorithmic work of each internal stage per timestep (one (b,t) row; s = bytes of an I/O element):
+# (flops, bytes).  A projection is a real GEMM with K*N = 2*H*P per row; a scan moves 16 or 24 bytes
+# per state and step.  A stage that is both (projection and scan in one kernel) names its flops and the
+# bytes it has to move (operand in, state planes in / out); the roofline that bounds it is the one whose
+# floor (work / measured peak) is the longer time.
 STAGE_MODEL = {
-    # input projection and forward scan in one kernel: the contraction is what it has to do (the scan
-    # adds 8 flop per state and step and no HBM traffic)
-    "gemm_Bu_scan_fwd": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "gemm_gx_scan_bwd": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "gemm_Bu": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "scan_fwd": ("hbm", lambda H, P, s: 16.0 * P),
-    "gemm_y": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "gemm_gx": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "scan_bwd": ("hbm", lambda H, P, s: 24.0 * P),
-    "gemm_du": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "gemm_gBbar": ("tensor", lambda H, P, s: 4.0 * H * P),
-    "gemm_gC": ("tensor", lambda H, P, s: 4.0 * H * P),
+    "gemm_Bu_scan_fwd": (lambda H, P, s: 4.0 * H * P, lambda H, P, s: H * s + 8.0 * P),      # u in, x planes out
+    "gemm_gx_scan_bwd": (lambda H, P, s: 4.0 * H * P, lambda H, P, s: H * s + 16.0 * P),     # gy, x planes in, s planes out
+    "gemm_Bu": (lambda H, P, s: 4.0 * H * P, None),
+    "scan_fwd": (None, lambda H, P, s: 16.0 * P),
+    "gemm_y": (lambda H, P, s: 4.0 * H * P, None),
+    "gemm_gx": (lambda H, P, s: 4.0 * H * P, None),
+    "scan_bwd": (None, lambda H, P, s: 24.0 * P),
+    "gemm_du": (lambda H, P, s: 4.0 * H * P, None),
+    "gemm_gBbar": (lambda H, P, s: 4.0 * H * P, None),
+    "gemm_gC": (lambda H, P, s: 4.0 * H * P, None),
 }
 
 
@@ -55,7 +56,7 @@ STAGE_MODEL = {
 # once its kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_TIMESTEP = {
     "gemm_Bu_scan_fwd": 777.8e6 / 262144,
-    "gemm_gx_scan_bwd": None,
+    "gemm_gx_scan_bwd": 1358.2e6 / 262144,
     "scan_fwd": 1021.7e6 / 262144,
     "scan_bwd": 1579.9e6 / 262144,
     "gemm_Bu": 763.6e6 / 262144,
@@ -440,18 +441,21 @@ def main():
         value = total_ts * args.steps / (ms * 1e-3)
         s_io = 2 if w.io_dtype == "bf16" else 4
         top = max((k for k in stages if k in STAGE_MODEL), key=lambda k: stages[k][1])
-        bound, work = STAGE_MODEL[top]
+        flops_fn, bytes_fn = STAGE_MODEL[top]
         n_launch, top_ms = stages[top]
         per_launch_s = top_ms * 1e-3 / n_launch
-        alg = work(w.H, w.P, s_io) * w.timesteps
         traffic = NCU_TRAFFIC_PER_TIMESTEP.get(top) if (w.T, w.H, w.P, w.io_dtype, stacked) == (1024, 512, 256, "bf16", False) else None
         traffic = None if traffic is None else traffic * w.timesteps
+        hbm_peak = float(peaks["hbm_gbs"])
+        tensor_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+        alg_flops = flops_fn(w.H, w.P, s_io) * w.timesteps if flops_fn else 0.0
+        alg_bytes = bytes_fn(w.H, w.P, s_io) * w.timesteps if bytes_fn else 0.0
+        floors_s = {"tensor": alg_flops / (tensor_peak * 1e12), "hbm": alg_bytes / (hbm_peak * 1e9)}
+        bound = max(floors_s, key=floors_s.get)
         if bound == "hbm":
-            achieved, peak, runit = alg / per_launch_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"
+            alg, achieved, peak, runit = alg_bytes, alg_bytes / per_launch_s / 1e9, hbm_peak, "GB/s"
         else:
-            achieved = alg / per_launch_s / 1e12
-            peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-            runit = "TFLOP/s"
+            alg, achieved, peak, runit = alg_flops, alg_flops / per_launch_s / 1e12, tensor_peak, "TFLOP/s"
         stage_share = {k: round(v[1] / ms, 4) for k, v in stages.items()}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -466,7 +470,8 @@ def main():
             "clocks": clocks,
             "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
                          "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
-                         "algorithmic_per_launch": alg, "launches_per_step": n_launch / args.steps,
+                         "algorithmic_per_launch": alg,
+                         "floor_ms": {k: round(v * 1e3, 4) for k, v in floors_s.items() if v > 0}, "launches_per_step": n_launch / args.steps,
                          "ms_per_launch": per_launch_s * 1e3},
             "stage_ms_per_step": {k: round(v[1] / args.steps, 4) for k, v in stages.items()},
             "stage_share": stage_share,
