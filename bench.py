@@ -292,6 +292,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--allreduce-grads", action="store_true",
+                    help="N > 1: also sum the parameter gradients over the ranks every step (one all-reduce of the "
+                         "gradient bucket, running under the next step's forward pass), as a data-parallel trainer would")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -320,9 +323,16 @@ def main():
     buf = harness.StackBuffers(d, w.io_dtype) if stacked else harness.LayerBuffers(d, w.io_dtype)
     stream = torch.cuda.current_stream()
 
+    exchange = args.allreduce_grads and world > 1 and not stacked
+    pending = []
+
     def step():
         buf.forward(stream)
+        if pending:                      # last step's gradient sum has to be out of the bucket before it is rewritten
+            pending.pop().wait()
         buf.backward(stream)
+        if exchange:
+            pending.append(harness.allreduce_param_grads(buf, async_op=True))
 
     def barrier():
         if world > 1:
@@ -343,6 +353,8 @@ def main():
     ev0.record(stream)
     for _ in range(args.steps):
         step()
+    while pending:                       # the last step's exchange belongs to the timed region
+        pending.pop().wait()
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)
@@ -463,7 +475,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
                        "p_done": w.p_done, "n_layers": w.n_layers, "l2": "inputs larger than L2 (no flush)"
-                       if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}"},
+                       if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}" + (" + gradient all-reduce" if exchange else "")},
             "e2e": {"value": total_ts * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "mode": e2e_mode},
             "gpu_launches": int(launches),

@@ -31,6 +31,29 @@ def to_np(t):
     return t.cpu().numpy()
 
 
+def grad_bucket(P: int, H: int, device="cuda"):
+    """One contiguous fp32 buffer holding dLambda[P] c64, dDelta[P], dB[P,H] c64, dC[H,P] c64, dD[H]
+    (each segment starts on a 16-byte boundary); returns (bucket, views in that order)."""
+    pad = lambda n: (n + 3) // 4 * 4
+    sizes = [2 * P, P, 2 * P * H, 2 * H * P, H]          # in floats
+    offs = np.concatenate([[0], np.cumsum([pad(n) for n in sizes])])
+    bucket = torch.zeros(int(offs[-1]), dtype=torch.float32, device=device)
+    seg = [bucket[int(o):int(o) + n] for o, n in zip(offs[:-1], sizes)]
+    cplx = lambda t, *shape: torch.view_as_complex(t.view(*shape, 2))
+    return bucket, (cplx(seg[0], P), seg[1], cplx(seg[2], P, H), cplx(seg[3], H, P), seg[4])
+
+
+def allreduce_param_grads(buf, group=None, async_op=False):
+    """Sum of the parameter gradients over the ranks of a batch-sharded (data-parallel) run: the one
+    exchange such a run has.  Sequences are independent, so every rank's gradients are the sums over
+    its own sequences and the full-batch gradients are their sum; y, du and the states stay local.
+    One all-reduce over the bucket (NCCL on GPUs; any torch.distributed backend).  With async_op the
+    returned handle is waited for before the bucket is read or written again, which lets the exchange
+    run under the next step's forward pass."""
+    import torch.distributed as dist
+    return dist.all_reduce(buf.grad_bucket, op=dist.ReduceOp.SUM, group=group, async_op=async_op)
+
+
 class LayerBuffers:
     """Device copies of one layer's inputs plus preallocated outputs and workspace."""
 
@@ -55,11 +78,9 @@ class LayerBuffers:
         self.y = torch.empty((B, T, H), dtype=io, device=device)
         self.xT = torch.empty((B, P), **c64)
         self.du = torch.empty((B, T, H), dtype=io, device=device)
-        self.dLambda = torch.empty(P, **c64)
-        self.dDelta = torch.empty(P, **f32)
-        self.dB = torch.empty((P, H), **c64)
-        self.dC = torch.empty((H, P), **c64)
-        self.dD = torch.empty(H, **f32)
+        # The five parameter gradients are views into one fp32 bucket, so that a data-parallel
+        # trainer sums them over the ranks with a single all-reduce and no packing pass.
+        self.grad_bucket, (self.dLambda, self.dDelta, self.dB, self.dC, self.dD) = grad_bucket(P, H, device)
         self.dx0 = torch.empty((B, P), **c64)
         self.ws = sb.alloc_workspace(sb.ssm_layer_workspace_bytes(self.shape), device)
 

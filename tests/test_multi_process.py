@@ -1,7 +1,9 @@
 """Host-side logic of the N > 1 path on CPU (gloo, world size 2): the batch is sharded over the
 ranks with no data-path collective, each rank's shard gives exactly the rows of the full
 result (sequences are independent), the parameter gradients add up across ranks, and the
-step time reported is the maximum over ranks."""
+step time reported is the maximum over ranks.  The second test covers the exchange a data-parallel
+trainer adds: the five parameter gradients summed over the ranks by one all-reduce of the bucket
+they live in."""
 import os
 import socket
 
@@ -38,6 +40,48 @@ def _rank_main(rank, world, port, out):
     out.put((rank, lo, hi, y, dC.numpy(), float(t)))
     dist.barrier()
     dist.destroy_process_group()
+
+
+def _bucket_rank_main(rank, world, port, out):
+    import types
+    from paper_2502_20168_b200 import harness
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    d = I.draw_layer(W)
+    lo, hi = I.shard_batch(W.B, rank, world)
+    g = O.ssm_layer_bwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], d["u"][lo:hi], d["done"][lo:hi], None,
+                        d["gy"][lo:hi])
+    bucket, views = harness.grad_bucket(W.P, W.H, "cpu")
+    names = ("dLambda", "dDelta", "dB", "dC", "dD")
+    for name, v in zip(names, views):          # this rank's gradients, where the layer's backward would put them
+        v.copy_(torch.from_numpy(np.ascontiguousarray(g[name])).to(v.dtype))
+    buf = types.SimpleNamespace(grad_bucket=bucket)
+    work = harness.allreduce_param_grads(buf, async_op=True)
+    work.wait()
+    out.put((rank, {name: v.numpy().copy() for name, v in zip(names, views)}))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_parameter_gradients_summed_over_two_ranks_by_one_bucket_allreduce():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_bucket_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = [q.get(timeout=120) for _ in procs]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    d = I.draw_layer(W)
+    g = O.ssm_layer_bwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], d["u"], d["done"], None, d["gy"])
+    for rank, grads in got:
+        for name, v in grads.items():          # fp32 bucket against the float64 full-batch gradients
+            ref = g[name]
+            assert v.shape == ref.shape, name
+            assert np.max(np.abs(v - ref) / (1.0 + np.abs(ref))) < 1e-5, (rank, name)
 
 
 def test_batch_sharding_over_two_ranks():
