@@ -327,6 +327,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         tma_load_2d(smem_u32(skb + b * 2048), tmSkip, sbar[b], n_out0 + (slab0 + sl) * 32, row0);
     };
     if (lane == 0) {
+        fence_async_smem();   // (the lanes' reads of the previous tile's last slabs: fenced and joined there)
         fetch_skip(0);
         if (kSlabs > 1) fetch_skip(1);
     }
@@ -348,8 +349,14 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
 #pragma unroll
             for (int j = 0; j < 4; ++j) sk[j] = *reinterpret_cast<const uint4*>(skb + b * 2048 + lane * 64 + ((j ^ swz) << 4));
             tmem_ld_wait();
+            // The refill below is a write of the async proxy over what these lanes have just read through the
+            // generic proxy: without the proxy fences it can land before a lane's read has been served.
+            fence_async_smem();
             __syncwarp();
-            if (lane == 0 && sl + 2 < kSlabs) fetch_skip(sl + 2);
+            if (lane == 0 && sl + 2 < kSlabs) {
+                fence_async_smem();
+                fetch_skip(sl + 2);
+            }
             if (lane == 0) tma_store_wait_read();   // the previous slab has left both staging buffers
             __syncwarp();
             uint4 o[4];
@@ -389,8 +396,16 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
 #pragma unroll
         for (int j = 0; j < 4; ++j) sk[j] = *reinterpret_cast<const uint4*>(skb + b * 2048 + lane * 64 + ((j ^ swz) << 4));
         tmem_ld_wait();
-        __syncwarp();   // every lane has its skip row: the buffer can take the slab after next
-        if (lane == 0 && sl + 2 < kSlabs) fetch_skip(sl + 2);
+        // Every lane has asked for its skip row; the buffer takes the slab after next.  That refill is a
+        // write of the async proxy over data just read through the generic proxy: the proxy fences order the
+        // two (without them the refill was seen to land before a lane's read had been served, when another
+        // kernel shared the SMs and the skip rows came from L2).
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0 && sl + 2 < kSlabs) {
+            fence_async_smem();
+            fetch_skip(sl + 2);
+        }
         uint4 o[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
