@@ -138,3 +138,35 @@ def test_layer_step_replays_from_a_cuda_graph():
         sb_res = buf.results()
         for k in ("y", "du", "dLambda", "dDelta", "dB", "dC", "dD"):
             assert np.array_equal(eager[k], sb_res[k]), k
+
+
+def test_backward_results_do_not_depend_on_a_kernel_running_beside_it():
+    """Another stream keeps the GPU busy with reductions over the same gy and u while the backward
+    pass runs: every result has to come out bit for bit as in a quiet run.  (Shared-memory buffers
+    that the TMA unit refills right after the lanes have read them are where timing could show:
+    the sweep point with 64 long sequences is the one where it once did.)"""
+    import torch
+    from paper_2502_20168_b200 import binding as sb, harness
+    w = [c for c in I.C4 if c.T == 4096][0]
+    buf = harness.LayerBuffers(I.draw_layer(w), w.io_dtype)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    with torch.cuda.stream(main):
+        buf.forward(main); buf.backward(main)
+    torch.cuda.synchronize()
+    sb.ssm_check(buf.ws)
+    quiet = buf.results()
+    acc = torch.zeros(w.H, dtype=torch.float32, device="cuda")
+    for rep in range(3):
+        for k in ("du", "dLambda", "dB", "dC", "dD"):
+            getattr(buf, k).zero_()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for _ in range(12 + 4 * rep):
+                acc += torch.sum(buf.gy.view(-1, w.H) * buf.u.view(-1, w.H), dim=0, dtype=torch.float32)
+        with torch.cuda.stream(main):
+            buf.backward(main)
+        torch.cuda.synchronize()
+        sb.ssm_check(buf.ws)
+        busy = buf.results()
+        for k in ("du", "dLambda", "dDelta", "dB", "dC", "dD"):
+            assert np.array_equal(quiet[k], busy[k]), (rep, k)
