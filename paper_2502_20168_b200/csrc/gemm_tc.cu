@@ -1243,29 +1243,40 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     }
                 }
                 (void)mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag);
+                tc_fence_after();
+                // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7).
+                // A warp drains two groups of 32 columns (hi + lo halves each): the first group's loads are in
+                // flight while it waits for the tile to be free, the second group's while it stores the first.
+                static_assert(kFsEpiWarps == 8, "two 32-column groups per warp");
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+                uint32_t ra[32], ra2[32], rb[32], rb2[32];
+                tmem_ld32(t_row + (uint32_t)(grp * 32), ra);
+                tmem_ld32(t_row + (uint32_t)(BN / 2 + grp * 32), ra2);
                 if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
-                epi_sync();   // flags visible, tile free; also: the 256 threads leave together or not at all
+                epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
+                              // the 256 threads leave together or not at all
+                tmem_ld_wait();
                 if (*s.abort_flag) {
                     ok = false;
                     break;
                 }
-                tc_fence_after();
-                // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7)
-                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+                tmem_ld32(t_row + (uint32_t)((grp + 2) * 32), rb);
+                tmem_ld32(t_row + (uint32_t)(BN / 2 + (grp + 2) * 32), rb2);
 #pragma unroll
-                for (int gq = grp; gq < 4; gq += kFsEpiWarps / 4) {   // 32 columns = one 128-byte group of the row
-                    uint32_t r[32], r2[32];
-                    tmem_ld32(t_row + (uint32_t)(gq * 32), r);
-                    tmem_ld32(t_row + (uint32_t)(BN / 2 + gq * 32), r2);
-                    tmem_ld_wait();
+                for (int j = 0; j < 8; ++j)
+                    T4[prow * 32 + grp * 8 + (j ^ (prow & 7))] =
+                        make_float4(__uint_as_float(ra[4 * j]) + __uint_as_float(ra2[4 * j]),
+                                    __uint_as_float(ra[4 * j + 1]) + __uint_as_float(ra2[4 * j + 1]),
+                                    __uint_as_float(ra[4 * j + 2]) + __uint_as_float(ra2[4 * j + 2]),
+                                    __uint_as_float(ra[4 * j + 3]) + __uint_as_float(ra2[4 * j + 3]));
+                tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        T4[prow * 32 + gq * 8 + (j ^ (prow & 7))] =
-                            make_float4(__uint_as_float(r[4 * j]) + __uint_as_float(r2[4 * j]),
-                                        __uint_as_float(r[4 * j + 1]) + __uint_as_float(r2[4 * j + 1]),
-                                        __uint_as_float(r[4 * j + 2]) + __uint_as_float(r2[4 * j + 2]),
-                                        __uint_as_float(r[4 * j + 3]) + __uint_as_float(r2[4 * j + 3]));
-                }
+                for (int j = 0; j < 8; ++j)
+                    T4[prow * 32 + (grp + 2) * 8 + (j ^ (prow & 7))] =
+                        make_float4(__uint_as_float(rb[4 * j]) + __uint_as_float(rb2[4 * j]),
+                                    __uint_as_float(rb[4 * j + 1]) + __uint_as_float(rb2[4 * j + 1]),
+                                    __uint_as_float(rb[4 * j + 2]) + __uint_as_float(rb2[4 * j + 2]),
+                                    __uint_as_float(rb[4 * j + 3]) + __uint_as_float(rb2[4 * j + 3]));
                 tc_fence_before();
                 mbar_arrive_cluster(leader_empty0 + 8u * acc);
                 if ((acc ^= 1) == 0) acc_phase ^= 1u;

@@ -156,12 +156,12 @@ def test_backward_results_do_not_depend_on_a_kernel_running_beside_it():
     sb.ssm_check(buf.ws)
     quiet = buf.results()
     acc = torch.zeros(w.H, dtype=torch.float32, device="cuda")
-    for rep in range(3):
+    for rep in range(6):
         for k in ("du", "dLambda", "dB", "dC", "dD"):
             getattr(buf, k).zero_()
         torch.cuda.synchronize()
         with torch.cuda.stream(side):
-            for _ in range(12 + 4 * rep):
+            for _ in range(8 + 3 * rep):
                 acc += torch.sum(buf.gy.view(-1, w.H) * buf.u.view(-1, w.H), dim=0, dtype=torch.float32)
         with torch.cuda.stream(main):
             buf.backward(main)
