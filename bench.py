@@ -56,13 +56,13 @@ STAGE_MODEL = {
 # once its kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_TIMESTEP = {
     "gemm_Bu_scan_fwd": 777.8e6 / 262144,
-    "gemm_gx_scan_bwd": 1358.2e6 / 262144,
+    "gemm_gx_scan_bwd": 1326.6e6 / 262144,
     "scan_fwd": 1021.7e6 / 262144,
     "scan_bwd": 1579.9e6 / 262144,
     "gemm_Bu": 763.6e6 / 262144,
     "gemm_gx": 763.6e6 / 262144,
-    "gemm_y": 793.0e6 / 262144,
-    "gemm_du": 793.0e6 / 262144,
+    "gemm_y": None,      # (proxy fences added to the bf16 epilogue since the capture: 793.0 MB before)
+    "gemm_du": None,
     "gemm_gBbar": 813.4e6 / 262144,
     "gemm_gC": 813.4e6 / 262144,
 }
