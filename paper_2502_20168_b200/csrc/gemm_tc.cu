@@ -1,3 +1,4 @@
+#include <type_traits>
 // bf16 projections on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
 // memory, operands staged in shared memory by TMA).  Two kernels:
 //
@@ -730,6 +731,16 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 struct C2 {
     f32x2 re, im;   // two complex numbers: (re, re), (im, im)
 };
@@ -1224,6 +1235,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 npi = pack2(-im0, -im1);
             }
             C2 g = zero;        // this thread's part of the chain's sums s_t conj(x_{t-1})
+            f32x2 gim_neg = 0ull;   // the part of Im g that enters with a minus sign, summed apart
             C2 xinit = zero;    // x0: what stands before the sequence's first row
             if (sl == 0 && p.x0 && has_seq) {
                 const float2 c0 = p.x0[(size_t)b * p.P + pg], c1 = p.x0[(size_t)b * p.P + pg + 1];
@@ -1375,38 +1387,51 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 xphase ^= 1u;
                 const bool seq_start = tb == 0 && sl == 0;   // row 0 of this group is the sequence's first row
+                // A tile without flags (the common case) takes the loop without the per-row tests.
+                auto fold_rows = [&](auto with_flags) {
+                    constexpr bool kFlags = decltype(with_flags)::value;
 #pragma unroll
-                for (int i = R - 1; i >= 0; --i) {
-                    C2 sv = v[i];
-                    if (!from_carry) {
-                        if ((mask >> i) & 1u) x = zero;
-                        sv = x = cstep2(ar, ai, nai, x, v[i]);
-                    }
-                    float re0, re1, im0, im1;
-                    unpack2(sv.re, re0, re1);
-                    unpack2(sv.im, im0, im1);
-                    if (!((mask0 >> i) & 1u)) {
-                        C2 xp;
-                        if (seq_start && i == 0) {
-                            xp = xinit;
-                        } else {
-                            const uint2 xh = xs[i * 32], xl = xs[(R + i) * 32];
-                            xp.re = pack2(__uint_as_float(xh.x << 16) + __uint_as_float(xl.x << 16),
-                                          __uint_as_float(xh.y << 16) + __uint_as_float(xl.y << 16));
-                            xp.im = pack2(__uint_as_float(xh.x & 0xffff0000u) + __uint_as_float(xl.x & 0xffff0000u),
-                                          __uint_as_float(xh.y & 0xffff0000u) + __uint_as_float(xl.y & 0xffff0000u));
+                    for (int i = R - 1; i >= 0; --i) {
+                        C2 sv = v[i];
+                        if (!from_carry) {
+                            if (kFlags && ((mask >> i) & 1u)) x = zero;
+                            sv = x = cstep2(ar, ai, nai, x, v[i]);
                         }
-                        // g += s conj(x):  re += s.re x.re + s.im x.im,  im += s.im x.re - s.re x.im
-                        g.re = fma2(sv.re, xp.re, fma2(sv.im, xp.im, g.re));
-                        g.im = fma2(sv.im, xp.re, fma2(sv.re, xp.im ^ 0x8000000080000000ull, g.im));
+                        if (!kFlags || !((mask0 >> i) & 1u)) {
+                            C2 xp;
+                            if (seq_start && i == 0) {
+                                xp = xinit;
+                            } else {
+                                const uint2 xh = xs[i * 32], xl = xs[(R + i) * 32];
+                                xp.re = add2(pack2(__uint_as_float(xh.x << 16), __uint_as_float(xh.y << 16)),
+                                             pack2(__uint_as_float(xl.x << 16), __uint_as_float(xl.y << 16)));
+                                xp.im = add2(pack2(__uint_as_float(xh.x & 0xffff0000u), __uint_as_float(xh.y & 0xffff0000u)),
+                                             pack2(__uint_as_float(xl.x & 0xffff0000u), __uint_as_float(xl.y & 0xffff0000u)));
+                            }
+                            // g += s conj(x):  re += s.re x.re + s.im x.im,  im += s.im x.re - s.re x.im (two sums)
+                            g.re = fma2(sv.re, xp.re, fma2(sv.im, xp.im, g.re));
+                            g.im = fma2(sv.im, xp.re, g.im);
+                            gim_neg = fma2(sv.re, xp.im, gim_neg);
+                        }
+                        float re0, re1, im0, im1;
+                        unpack2(sv.re, re0, re1);
+                        unpack2(sv.im, im0, im1);
+                        const __nv_bfloat162 h0 = __floats2bfloat162_rn(re0, im0), h1 = __floats2bfloat162_rn(re1, im1);
+                        const uint32_t hb0 = *reinterpret_cast<const uint32_t*>(&h0), hb1 = *reinterpret_cast<const uint32_t*>(&h1);
+                        const f32x2 lre = sub2(sv.re, pack2(__uint_as_float(hb0 << 16), __uint_as_float(hb1 << 16)));
+                        const f32x2 lim = sub2(sv.im, pack2(__uint_as_float(hb0 & 0xffff0000u), __uint_as_float(hb1 & 0xffff0000u)));
+                        float lr0, lr1, li0, li1;
+                        unpack2(lre, lr0, lr1);
+                        unpack2(lim, li0, li1);
+                        const __nv_bfloat162 l0 = __floats2bfloat162_rn(lr0, li0), l1 = __floats2bfloat162_rn(lr1, li1);
+                        xs[i * 32] = make_uint2(hb0, hb1);
+                        xs[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
                     }
-                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(re0, im0), h1 = __floats2bfloat162_rn(re1, im1);
-                    const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
-                    const __nv_bfloat162 l0 = __floats2bfloat162_rn(re0 - f0.x, im0 - f0.y);
-                    const __nv_bfloat162 l1 = __floats2bfloat162_rn(re1 - f1.x, im1 - f1.y);
-                    xs[i * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-                    xs[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
-                }
+                };
+                if ((mask | mask0) == 0u)
+                    fold_rows(std::false_type{});
+                else
+                    fold_rows(std::true_type{});
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0 && has_seq) {
@@ -1433,7 +1458,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             {
                 float g0, g1, g2, g3;
                 unpack2(g.re, g0, g1);
-                unpack2(g.im, g2, g3);
+                unpack2(sub2(g.im, gim_neg), g2, g3);
                 agg_e[te] = make_float4(g0, g1, g2, g3);
             }
             epi_sync();
