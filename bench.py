@@ -56,7 +56,7 @@ STAGE_MODEL = {
 # once its kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_TIMESTEP = {
     "gemm_Bu_scan_fwd": 777.8e6 / 262144,
-    "gemm_gx_scan_bwd": 1326.6e6 / 262144,
+    "gemm_gx_scan_bwd": 1327.6e6 / 262144,
     "scan_fwd": 1021.7e6 / 262144,
     "scan_bwd": 1579.9e6 / 262144,
     "gemm_Bu": 763.6e6 / 262144,
