@@ -133,8 +133,8 @@ def oracle_sample_run(d, n_seq):
     u, gy = d["u"][:n_seq], d["gy"][:n_seq]
     t0 = time.perf_counter()
     if "params" in d:      # stacked model
-        _, cache = O.stack_fwd(d["params"], d["ln_weight"], d["ln_bias"], u, done, round_io=I.round_to_bf16)
-        O.stack_bwd(d["params"], d["ln_weight"], d["ln_bias"], cache, done, gy, round_io=I.round_to_bf16)
+        _, cache = O.stack_fwd(d["params"], d["ln_weight"], d["ln_bias"], u, done)
+        O.stack_bwd(d["params"], d["ln_weight"], d["ln_bias"], cache, done, gy)
         return time.perf_counter() - t0
     O.ssm_layer_fwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], u, done, None)
     O.ssm_layer_bwd(d["Lambda"], d["Delta"], d["Bc"], d["Cc"], d["D"], u, done, None, gy)

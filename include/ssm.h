@@ -15,9 +15,13 @@
  *
  * Conventions shared by every entry point
  *  - All data pointers are DEVICE pointers owned by the caller; `shape` is a HOST
- *    pointer.  The library allocates no memory, keeps no global state and never
- *    synchronises the host (except ssm_check).  Work is enqueued on `stream`
+ *    pointer.  The entry points allocate no device memory and never synchronise the host
+ *    (except ssm_check, ssm_check_static and ssm_profile_end).  Work is enqueued on `stream`
  *    (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *  - What the library keeps per process: small host-side caches filled on first use per
+ *    device (SM count, kernel attributes, the tensor-map encoder's address), the launch
+ *    counter and the event pool of the measurement helpers, and one fixed device array of
+ *    SSM_STATIC_SCRATCH_BYTES per GPU for ssm_scan_bwd_static.  Results never depend on them.
  *  - Tensors are dense, row-major, last index fastest.  Complex numbers are
  *    interleaved (re, im) float pairs, bit-compatible with float2 / complex64.
  *  - Parameters, states and their gradients are always fp32.  Only u, y, gy, du follow
@@ -130,12 +134,16 @@ int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* don
  *  - All calls on a device share the one array.  The library clears what has to start at
  *    zero on every call, but two calls whose GPU work overlaps (different streams) race on
  *    it: issue them on one stream or order them yourself.
+ *  - A bounded device-side wait that gives up records SSM_ERR_TIMEOUT in the array's first word;
+ *    ssm_check_static(stream) reads it back (it synchronises `stream`, allocates nothing, and
+ *    reports the most recent call on the current device, since every call clears the word).
  * Arguments are those of ssm_scan_bwd minus the workspace. */
 #define SSM_STATIC_SCRATCH_BYTES (8u << 20)
 int ssm_scan_bwd_static(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* done,
                         const ssm_c64* x0, const ssm_c64* x, const ssm_c64* gx,
                         const ssm_c64* gxT, ssm_c64* gBu, ssm_c64* gAbar, ssm_c64* gx0,
                         void* stream);
+int ssm_check_static(void* stream);
 
 /* ---- the whole layer: Sec. III-B Eq. 3 with the resets of Sec. IV-A ----------------
  * Forward: discretise, Bu = Bbar u, scan, y = Re(C x) + D u.  u, y are [B,T,H] in
@@ -197,8 +205,10 @@ int ssm_glu_bwd(const ssm_shape* shape, const float* W, const void* v, const voi
  * (exact erf GELU, LayerNorm over the H features with eps 1e-5), the same done flags in every
  * layer and a zero initial state.  The paper wraps its S5 SSM in a block of nonlinearity and
  * gating (Appendix "S5 Sequence Layer", whose schematic is a half-GLU); this post-norm
- * residual block is the stacked configuration the benchmark defines.  Tensors between layers
- * (v, u_l and, in the backward pass, their gradients) are stored in io_dtype; arithmetic is fp32.
+ * residual block is the stacked configuration the benchmark defines.  u, out, gout and du are in
+ * io_dtype; what passes between the layers stays in fp32 inside the workspace (rounded to bf16
+ * there, two correct evaluations differ by more than the bf16 tolerance in the parameter
+ * gradients of the layers below).
  * `params` / `grads` are HOST arrays of n_layers structs holding DEVICE pointers.  The
  * workspace filled by ssm_stack_fwd is read by ssm_stack_bwd.  Backward: from gout[B,T,H] to
  * du[B,T,H] and every layer's parameter gradients (overwritten). */

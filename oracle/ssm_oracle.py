@@ -270,9 +270,10 @@ def _identity(a):
 def stack_fwd(params, ln_weight, ln_bias, u, done=None, round_io=_identity):
     """n layers of  v = SSM(u);  out = LayerNorm(u + GELU(v)) * w + b.
 
-    `round_io` models the storage precision of every tensor that crosses a layer
-    boundary or is kept for the backward pass (v and out); identity = all float64.
-    Returns (out, cache).
+    `round_io` (identity by default = all float64) models a storage precision for the
+    tensors that are a layer's inputs and outputs: the SSM output v and the block output.
+    It exists to study what such roundings do to the gradients; the CUDA path keeps these
+    tensors in fp32 and is compared with the default.  Returns (out, cache).
     """
     cache = []
     act = np.asarray(u, F64)
@@ -289,8 +290,9 @@ def stack_fwd(params, ln_weight, ln_bias, u, done=None, round_io=_identity):
 def stack_bwd(params, ln_weight, ln_bias, cache, done, gout, round_io=_identity):
     """Backward of `stack_fwd` (rounding treated as identity in the derivative).
 
-    Per layer, top down:  gz = LN'(gout);  gv = round(gz * GELU'(v));  the SSM backward
-    takes gv;  the gradient handed to the layer below is round(round(gz) + du_ssm).
+    Per layer, top down:  gz = LN'(gout);  gv = round(gz * GELU'(v)) is the SSM layer's
+    incoming gradient;  the gradient handed to the layer below is round(gz + du_ssm): only what
+    enters or leaves a layer is rounded, nothing inside it.
     Returns (du, [per-layer dict(dLambda, dDelta, dB, dC, dD, dln_weight, dln_bias)]).
     """
     g = np.asarray(gout, F64)
@@ -300,7 +302,7 @@ def stack_bwd(params, ln_weight, ln_bias, cache, done, gout, round_io=_identity)
         gz, gw, gb = layernorm_bwd(g, c["zhat"], c["rstd"], np.asarray(ln_weight[l], F64))
         gv = round_io(gz * gelu_grad(c["v"])).astype(F64)
         r = ssm_layer_bwd(p["Lambda"], p["Delta"], p["Bc"], p["Cc"], p["D"], c["u"], done, None, gv)
-        g = round_io(round_io(gz).astype(F64) + r["du"]).astype(F64)
+        g = round_io(gz + r["du"]).astype(F64)
         grads[l] = {k: r[k] for k in ("dLambda", "dDelta", "dB", "dC", "dD")}
         grads[l]["dln_weight"] = gw
         grads[l]["dln_bias"] = gb

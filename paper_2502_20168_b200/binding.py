@@ -25,7 +25,7 @@ EXPORTS = (
     "ssm_status_string", "ssm_check", "ssm_discretize", "ssm_discretize_bwd",
     "ssm_scan_workspace_bytes", "ssm_scan_fwd", "ssm_scan_bwd",
     "ssm_layer_workspace_bytes", "ssm_layer_fwd", "ssm_layer_bwd",
-    "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static",
+    "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static", "ssm_check_static",
     "ssm_stack_workspace_bytes", "ssm_stack_fwd", "ssm_stack_bwd",
     "ssm_step_workspace_bytes", "ssm_step_prepare", "ssm_step",
     "ssm_glu_workspace_bytes", "ssm_glu_fwd", "ssm_glu_bwd",
@@ -83,6 +83,8 @@ def _load() -> ctypes.CDLL:
     lib.ssm_layer_bwd.argtypes = [S] + [P] * 11 + [c_size_t] + [P] * 8
     lib.ssm_scan_bwd_static.restype = c_int
     lib.ssm_scan_bwd_static.argtypes = [S] + [P] * 10
+    lib.ssm_check_static.restype = c_int
+    lib.ssm_check_static.argtypes = [P]
     lib.ssm_stack_workspace_bytes.restype = c_size_t
     lib.ssm_stack_workspace_bytes.argtypes = [S, c_int]
     lib.ssm_stack_fwd.restype = c_int
@@ -191,6 +193,11 @@ def ssm_scan_bwd_static(shape, Abar, done, x0, x, gx, gxT, gBu, gAbar, gx0, stre
     raises SsmError(SSM_ERR_TOO_LARGE) when the shape needs more than SSM_STATIC_SCRATCH_BYTES)."""
     _ok(_lib.ssm_scan_bwd_static(byref(shape), _ptr(Abar), _ptr(done), _ptr(x0), _ptr(x), _ptr(gx), _ptr(gxT),
                                  _ptr(gBu), _ptr(gAbar), _ptr(gx0), _stream(stream)), "ssm_scan_bwd_static")
+
+
+def ssm_check_static(stream=None) -> None:
+    """Status of the most recent ssm_scan_bwd_static call on the current device (synchronises `stream`)."""
+    _ok(_lib.ssm_check_static(_stream(stream)), "ssm_check_static")
 
 
 def ssm_layer_workspace_bytes(shape) -> int:

@@ -189,10 +189,22 @@ static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
 
 // Launch sequence of one layer's forward pass from a prepared workspace.  `hdr` receives the
 // status of bounded waits.
-static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D, const void* u, const uint8_t* done,
-                         const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr, cudaStream_t st) {
-    const bool bf16 = s.io_dtype == SSM_BF16;
+// Storage types of the tensors a layer reads and writes.  For the entry points of a single layer all
+// of them are shape->io_dtype; inside a stack only the stack's own input and outputs are.
+struct LayerIo {
+    bool u_bf16, y_bf16;      // forward: u in, y out
+    bool gy_bf16, du_bf16;    // backward: gy in, du out
+};
+static LayerIo layer_io(const ssm_shape& s) {
+    const bool b = s.io_dtype == SSM_BF16;
+    return {b, b, b, b};
+}
+
+static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const LayerIo& io, const float* D, const void* u,
+                         const uint8_t* done, const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr,
+                         cudaStream_t st) {
     const int BT = s.B * s.T, P2 = 2 * s.P;
+    if (p.tc && !(io.u_bf16 && io.y_bf16)) return SSM_ERR_DTYPE;   // the tensor-core path reads and writes bf16
     int rc = SSM_OK;
     if (p.tc && tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P)) {
         {   // projection and scan in one kernel: x = scan(u Bbar^T), Bu stays on chip
@@ -227,8 +239,8 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D,
     } else {
         {
             StageTimer tm("gemm_Bu", st);
-            GemmTN g1{u, bf16, s.H, at<void>(ws, p.W0), false, s.H, BT, P2, s.H, Epi::StoreF32,
-                      at<void>(ws, p.xs), false, nullptr, nullptr, nullptr};
+            GemmTN g1{u, io.u_bf16, s.H, at<void>(ws, p.W0), false, s.H, BT, P2, s.H, Epi::StoreF32,
+                      at<void>(ws, p.xs), false, nullptr, nullptr, false, nullptr};
             launch_gemm_tn(g1, st);
         }
         {
@@ -241,7 +253,7 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D,
         {
             StageTimer tm("gemm_y", st);
             GemmTN g2{at<void>(ws, p.xs), false, P2, at<void>(ws, p.W2), false, P2, BT, s.H, P2, Epi::AddDiagIo,
-                      y, bf16, D, u, nullptr};
+                      y, io.y_bf16, D, u, io.u_bf16, nullptr};
             launch_gemm_tn(g2, st);
         }
     }
@@ -249,11 +261,12 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const float* D,
     return SSM_OK;
 }
 
-static int layer_fwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
-                          const ssm_c64* Bc, const ssm_c64* Cc, const float* D, const void* u, const uint8_t* done,
-                          const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr, cudaStream_t st) {
+static int layer_fwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo& io, const ssm_c64* Lambda,
+                          const float* Delta, const ssm_c64* Bc, const ssm_c64* Cc, const float* D, const void* u,
+                          const uint8_t* done, const ssm_c64* x0, void* y, ssm_c64* xT, void* ws, WsHeader* hdr,
+                          cudaStream_t st) {
     layer_prepare(s, p, Lambda, Delta, Bc, Cc, ws, st);
-    return layer_fwd_run(s, p, D, u, done, x0, y, xT, ws, hdr, st);
+    return layer_fwd_run(s, p, io, D, u, done, x0, y, xT, ws, hdr, st);
 }
 
 SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const float* Delta, const ssm_c64* Bc,
@@ -270,7 +283,7 @@ SSM_API int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     cudaStream_t st = (cudaStream_t)stream;
     WsHeader* hdr = at<WsHeader>(ws, p.hdr);
     if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return SSM_ERR_CUDA;
-    return layer_fwd_impl(s, p, Lambda, Delta, Bc, Cc, D, u, done, x0, y, xT, ws, hdr, st);
+    return layer_fwd_impl(s, p, layer_io(s), Lambda, Delta, Bc, Cc, D, u, done, x0, y, xT, ws, hdr, st);
 }
 
 // Single-step mode: the layer's forward launch sequence for T = 1 from operands prepared once.
@@ -310,7 +323,8 @@ SSM_API int ssm_step(const ssm_shape* shape, const float* D, const void* u, cons
     const LayerPlan p = plan_layer(s);
     if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
     // each (trajectory, state) is read as x0 and written as xT by the same thread, so x_next may be x_prev
-    return layer_fwd_run(s, p, D, u, done, x_prev, y, x_next, ws, at<WsHeader>(ws, p.hdr), (cudaStream_t)stream);
+    return layer_fwd_run(s, p, layer_io(s), D, u, done, x_prev, y, x_next, ws, at<WsHeader>(ws, p.hdr),
+                         (cudaStream_t)stream);
 }
 
 // ---- half-GLU gate -----------------------------------------------------------------------
@@ -381,7 +395,7 @@ SSM_API int ssm_glu_fwd(const ssm_shape* shape, const float* W, const void* v, v
             if (int rc = launch_gemm_tc_tn(g, st)) return rc;
         } else {
             GemmTN g{at<void>(ws, p.x1), false, s.H, at<void>(ws, p.Wt), false, s.H, M, s.H, s.H, Epi::StoreF32,
-                     at<void>(ws, p.z), false, nullptr, nullptr, nullptr};
+                     at<void>(ws, p.z), false, nullptr, nullptr, false, nullptr};
             launch_gemm_tn(g, st);
         }
     }
@@ -417,7 +431,7 @@ SSM_API int ssm_glu_bwd(const ssm_shape* shape, const float* W, const void* v, c
             if (int rc = launch_gemm_tc_tn(g, st)) return rc;
         } else {
             GemmTN g{at<void>(ws, p.gz), false, s.H, W, false, s.H, M, s.H, s.H, Epi::StoreF32,
-                     at<void>(ws, p.gx1), false, nullptr, nullptr, nullptr};
+                     at<void>(ws, p.gx1), false, nullptr, nullptr, false, nullptr};
             launch_gemm_tn(g, st);
         }
     }
@@ -446,15 +460,15 @@ SSM_API int ssm_glu_bwd(const ssm_shape* shape, const float* W, const void* v, c
     return SSM_OK;
 }
 
-// Launch sequence of one layer's backward pass.  du_add (io dtype, may be NULL) is added to du
-// before it is rounded (the residual branch of a stacked model).
-static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
-                          const ssm_c64* Bc, const float* D, const void* u, const uint8_t* done, const ssm_c64* x0,
-                          const void* gy, const ssm_c64* gxT, const void* du_add, void* ws, WsHeader* hdr, void* du,
-                          ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD, ssm_c64* dx0,
-                          cudaStream_t st) {
-    const bool bf16 = s.io_dtype == SSM_BF16;
+// Launch sequence of one layer's backward pass.  du_add (fp32 [B,T,H], may be NULL) is added to du
+// before it is stored (the gradient of the residual branch of a stacked model).
+static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo& io, const ssm_c64* Lambda,
+                          const float* Delta, const ssm_c64* Bc, const float* D, const void* u, const uint8_t* done,
+                          const ssm_c64* x0, const void* gy, const ssm_c64* gxT, const float* du_add, void* ws,
+                          WsHeader* hdr, void* du, ssm_c64* dLambda, float* dDelta, ssm_c64* dB, ssm_c64* dC, float* dD,
+                          ssm_c64* dx0, cudaStream_t st) {
     const int BT = s.B * s.T, P2 = 2 * s.P;
+    if (p.tc && !(io.u_bf16 && io.gy_bf16 && io.du_bf16)) return SSM_ERR_DTYPE;
     float* part = at<float>(ws, p.part);
     const size_t plane = (size_t)BT * s.P * 4;   // bytes of one bf16 plane of a state tensor
     int rc = SSM_OK;
@@ -502,8 +516,8 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
     } else {
         {
             StageTimer tm("gemm_gx", st);
-            GemmTN g3{gy, bf16, s.H, at<void>(ws, p.W1), false, s.H, BT, P2, s.H, Epi::StoreF32,
-                      at<void>(ws, p.gs), false, nullptr, nullptr, nullptr};
+            GemmTN g3{gy, io.gy_bf16, s.H, at<void>(ws, p.W1), false, s.H, BT, P2, s.H, Epi::StoreF32,
+                      at<void>(ws, p.gs), false, nullptr, nullptr, false, nullptr};
             launch_gemm_tn(g3, st);
         }
         {
@@ -517,25 +531,25 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
         {
             StageTimer tm("gemm_du", st);
             GemmTN g4{at<void>(ws, p.gs), false, P2, at<void>(ws, p.W3), false, P2, BT, s.H, P2, Epi::AddDiagIo,
-                      du, bf16, D, gy, du_add};
+                      du, io.du_bf16, D, gy, io.gy_bf16, du_add};
             launch_gemm_tn(g4, st);
         }
         {
             StageTimer tm("gemm_gBbar", st);
-            GemmNT g5{u, bf16, s.H, at<void>(ws, p.gs), false, P2, BT, p.splits, part};
+            GemmNT g5{u, io.u_bf16, s.H, at<void>(ws, p.gs), false, P2, BT, p.splits, part};
             launch_gemm_nt(g5, st);
             launch_splitk_reduce(part, p.splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
         }
         {
             StageTimer tm("gemm_gC", st);
-            GemmNT g6{gy, bf16, s.H, at<void>(ws, p.xs), false, P2, BT, p.splits, part};
+            GemmNT g6{gy, io.gy_bf16, s.H, at<void>(ws, p.xs), false, P2, BT, p.splits, part};
             launch_gemm_nt(g6, st);
             launch_splitk_reduce(part, p.splits, s.H, P2, 1, (float2*)dC, st);
         }
     }
     {   // dD[h] = sum_m gy[m,h] u[m,h];  then the adjoint of the discretisation
         StageTimer tm("gD_and_discretize_bwd", st);
-        launch_dot_columns(bf16, gy, u, BT, s.H, dD, at<float>(ws, p.dot), st);
+        launch_dot_columns(io.gy_bf16, gy, io.u_bf16, u, BT, s.H, dD, at<float>(ws, p.dot), st);
         launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
                               at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);
     }
@@ -560,35 +574,44 @@ SSM_API int ssm_layer_bwd(const ssm_shape* shape, const ssm_c64* Lambda, const f
     if (int rc = check_ws(ws, ws_bytes, p.total)) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     WsHeader* hdr = at<WsHeader>(ws, p.hdr);
-    return layer_bwd_impl(s, p, Lambda, Delta, Bc, D, u, done, x0, gy, gxT, nullptr, ws, hdr, du, dLambda, dDelta, dB,
-                          dC, dD, dx0, st);
+    return layer_bwd_impl(s, p, layer_io(s), Lambda, Delta, Bc, D, u, done, x0, gy, gxT, nullptr, ws, hdr, du, dLambda,
+                          dDelta, dB, dC, dD, dx0, st);
 }
 
 // ---- stacked model -----------------------------------------------------------------------------
 namespace {
 
-// The layers of a stack run on the fp32 CUDA-core path: what is stored between and inside the
-// blocks is rounded to the I/O type, and a value that lands on the other side of a rounding
-// boundary than in an exact evaluation shifts the parameter-gradient sums by more than the
-// tolerance allows unless the arithmetic in front of every rounding is accurate to fp32 level.
+// Storage inside a stack.  Only the stack's input u, its output, gout and du are in the I/O type.
+// Everything that passes between the layers (the SSM outputs v, the layer inputs, the gradients
+// handed from a layer to the one below) is fp32: stored in bf16, a value that rounds to the other
+// neighbour than in an exact evaluation is a legitimate difference between two correct runs, and the
+// layers that follow amplify such differences in the parameter-gradient sums beyond the tolerance of
+// the I/O type.  The layers therefore run with fp32 inputs and outputs (except for the first layer's
+// input and the last gradient), on the fp32 path of the layer.
 struct StackPlan {
     size_t layer_ws;   // bytes of one layer workspace
-    size_t act;        // bytes of one [B,T,H] io tensor
-    size_t hdr, layers, acts, vs, stats, gzr, gv, g0, g1, tmp, total;
+    size_t act;        // bytes of one fp32 [B,T,H] tensor
+    size_t hdr, layers, acts, vs, stats, gz, gv, g0, g1, tmp, total;
 };
+
+ssm_shape stack_layer_shape(const ssm_shape& s) {
+    ssm_shape t = s;
+    t.io_dtype = SSM_F32;
+    return t;
+}
 
 StackPlan plan_stack(const ssm_shape& s, int L) {
     StackPlan p{};
     size_t off = 0;
     const size_t BT = (size_t)s.B * s.T;
-    p.layer_ws = align_up(plan_layer(s, false).total, 256);
-    p.act = align_up(BT * s.H * (s.io_dtype == SSM_BF16 ? 2 : 4), 256);
+    p.layer_ws = align_up(plan_layer(stack_layer_shape(s), false).total, 256);
+    p.act = align_up(BT * s.H * 4, 256);
     p.hdr = take(off, sizeof(WsHeader));
     p.layers = take(off, p.layer_ws * L);
     p.acts = take(off, p.act * (L > 1 ? L - 1 : 0));   // inputs of layers 1 .. L-1
     p.vs = take(off, p.act * L);                       // SSM outputs
     p.stats = take(off, align_up(BT * 4, 256) * 2 * L);   // mean and 1/std of every row, per layer
-    p.gzr = take(off, p.act);
+    p.gz = take(off, p.act);
     p.gv = take(off, p.act);
     p.g0 = take(off, p.act);
     p.g1 = take(off, p.act);
@@ -626,7 +649,8 @@ SSM_API int ssm_stack_fwd(const ssm_shape* shape, int n_layers, const ssm_stack_
     const ssm_shape& s = *shape;
     const StackPlan sp = plan_stack(s, n_layers);
     if (int rc = check_ws(ws, ws_bytes, sp.total)) return rc;
-    const LayerPlan lp = plan_layer(s, false);
+    const ssm_shape ls = stack_layer_shape(s);
+    const LayerPlan lp = plan_layer(ls, false);
     cudaStream_t st = (cudaStream_t)stream;
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T;
@@ -636,14 +660,16 @@ SSM_API int ssm_stack_fwd(const ssm_shape* shape, int n_layers, const ssm_stack_
     const void* in = u;
     for (int l = 0; l < n_layers; ++l) {
         const ssm_stack_params& q = params[l];
+        const bool first = l == 0, last = l == n_layers - 1;
         void* lws = at<void>(ws, sp.layers + sp.layer_ws * l);
-        void* v = at<void>(ws, sp.vs + sp.act * l);
-        void* o = (l == n_layers - 1) ? out : at<void>(ws, sp.acts + sp.act * l);
-        if (int rc = layer_fwd_impl(s, lp, q.Lambda, q.Delta, q.Bc, q.Cc, q.D, in, done, nullptr, v, nullptr, lws, hdr, st))
+        float* v = at<float>(ws, sp.vs + sp.act * l);
+        void* o = last ? out : at<void>(ws, sp.acts + sp.act * l);
+        const LayerIo io{first && bf16, false, false, false};
+        if (int rc = layer_fwd_impl(ls, lp, io, q.Lambda, q.Delta, q.Bc, q.Cc, q.D, in, done, nullptr, v, nullptr, lws, hdr, st))
             return rc;
         StageTimer tm("stack_gelu_ln_fwd", st);
-        launch_stack_fwd(bf16, BT, s.H, in, v, q.ln_weight, q.ln_bias, o, at<float>(ws, sp.stats + stat * (2 * l)),
-                         at<float>(ws, sp.stats + stat * (2 * l + 1)), st);
+        launch_stack_fwd(first && bf16, last && bf16, BT, s.H, in, v, q.ln_weight, q.ln_bias, o,
+                         at<float>(ws, sp.stats + stat * (2 * l)), at<float>(ws, sp.stats + stat * (2 * l + 1)), st);
         in = o;
     }
     SSM_RETURN_IF_CUDA_ERROR();
@@ -666,7 +692,8 @@ SSM_API int ssm_stack_bwd(const ssm_shape* shape, int n_layers, const ssm_stack_
     const ssm_shape& s = *shape;
     const StackPlan sp = plan_stack(s, n_layers);
     if (int rc = check_ws(ws, ws_bytes, sp.total)) return rc;
-    const LayerPlan lp = plan_layer(s, false);
+    const ssm_shape ls = stack_layer_shape(s);
+    const LayerPlan lp = plan_layer(ls, false);
     cudaStream_t st = (cudaStream_t)stream;
     const bool bf16 = s.io_dtype == SSM_BF16;
     const int BT = s.B * s.T;
@@ -676,18 +703,21 @@ SSM_API int ssm_stack_bwd(const ssm_shape* shape, int n_layers, const ssm_stack_
     for (int l = n_layers - 1; l >= 0; --l) {
         const ssm_stack_params& q = params[l];
         const ssm_stack_grads& gr = grads[l];
+        const bool first = l == 0, top = l == n_layers - 1;
         void* lws = at<void>(ws, sp.layers + sp.layer_ws * l);
-        const void* in = (l == 0) ? u : at<void>(ws, sp.acts + sp.act * (l - 1));
-        const void* v = at<void>(ws, sp.vs + sp.act * l);
-        void* gnext = (l == 0) ? du : at<void>(ws, (l & 1) ? sp.g1 : sp.g0);
+        const void* in = first ? u : at<void>(ws, sp.acts + sp.act * (l - 1));
+        const float* v = at<float>(ws, sp.vs + sp.act * l);
+        void* gnext = first ? du : at<void>(ws, (l & 1) ? sp.g1 : sp.g0);
         {
             StageTimer tm("stack_gelu_ln_bwd", st);
-            launch_stack_bwd(bf16, BT, s.H, g, in, v, q.ln_weight, at<float>(ws, sp.stats + stat * (2 * l)),
-                             at<float>(ws, sp.stats + stat * (2 * l + 1)), at<void>(ws, sp.gzr), at<void>(ws, sp.gv),
-                             gr.dln_weight, gr.dln_bias, at<float>(ws, sp.tmp), st);
+            launch_stack_bwd(top && bf16, first && bf16, BT, s.H, g, in, v, q.ln_weight,
+                             at<float>(ws, sp.stats + stat * (2 * l)), at<float>(ws, sp.stats + stat * (2 * l + 1)),
+                             at<float>(ws, sp.gz), at<float>(ws, sp.gv), gr.dln_weight, gr.dln_bias, at<float>(ws, sp.tmp), st);
         }
-        if (int rc = layer_bwd_impl(s, lp, q.Lambda, q.Delta, q.Bc, q.D, in, done, nullptr, at<void>(ws, sp.gv), nullptr,
-                                    at<void>(ws, sp.gzr), lws, hdr, gnext, gr.dLambda, gr.dDelta, gr.dB, gr.dC, gr.dD,
+        // the gradient handed down: gz (residual branch) + du of the SSM, summed in fp32 in the du epilogue
+        const LayerIo io{first && bf16, false, false, first && bf16};
+        if (int rc = layer_bwd_impl(ls, lp, io, q.Lambda, q.Delta, q.Bc, q.D, in, done, nullptr, at<void>(ws, sp.gv), nullptr,
+                                    at<float>(ws, sp.gz), lws, hdr, gnext, gr.dLambda, gr.dDelta, gr.dB, gr.dC, gr.dD,
                                     nullptr, st))
             return rc;
         g = gnext;

@@ -51,6 +51,8 @@ inline bool misaligned(const void* p, size_t a = 16) { return (reinterpret_cast<
 
 // Measurement hooks (profile.cu): launch counter and optional per-stage event timing.
 void count_launch(int n = 1);
+// Number of SMs of the current device, cached per device ordinal (148 where no device answers).
+int device_sm_count();
 // Raises a kernel's dynamic shared-memory limit, once per (kernel, device) (device_setup.cu).
 bool set_max_dynamic_smem(const void* kernel, size_t bytes);
 class StageTimer {

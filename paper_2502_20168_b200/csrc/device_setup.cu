@@ -25,4 +25,27 @@ bool set_max_dynamic_smem(const void* kernel, size_t bytes) {
     return true;
 }
 
+// Workspace layouts, operand packing order and kernel choices depend on the SM count, so it is
+// looked up for the device that is current, once per ordinal.
+int device_sm_count() {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static int cache[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            return 148;
+        }
+        cache[dev] = n;
+    }
+    return cache[dev];
+}
+
 }  // namespace ssm

@@ -32,13 +32,14 @@ struct EpiArgs {
 };
 
 // out[m,n] = sum_k A[m,k] Bm[n,k]; both operands K-contiguous.  K % 4 == 0.
-template <typename TA, typename TB, typename TO, bool kAddDiag>
+// TO: type of out; TS: type of the skip operand; the addend, where there is one, is fp32.
+template <typename TA, typename TB, typename TO, typename TS, bool kAddDiag>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_tn_kernel(const TA* __restrict__ A, int lda, const TB* __restrict__ Bm, int ldb, int M, int N, int K,
                EpiArgs e) {
     __shared__ __align__(16) float As[TK][TM + 4];
     __shared__ __align__(16) float Bs[TK][TN + 4];
-    const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+    const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;   // rows along x: grid.y is limited to 65535
     const int tid = threadIdx.x;
     const int lr = tid >> 2;         // 0..63: row of the tile this thread loads
     const int lk = (tid & 3) * 4;    // 0,4,8,12: k offset
@@ -77,9 +78,9 @@ gemm_tn_kernel(const TA* __restrict__ A, int lda, const TB* __restrict__ Bm, int
             if (n >= N) continue;
             float v = acc[i][j];
             if (kAddDiag) {
-                const TO* skip = reinterpret_cast<const TO*>(e.skip);
-                v = fmaf(e.diag[n], to_f32<TO>(skip[(size_t)m * e.ldo + n]), v);
-                if (e.add) v += to_f32<TO>(reinterpret_cast<const TO*>(e.add)[(size_t)m * e.ldo + n]);
+                const TS* skip = reinterpret_cast<const TS*>(e.skip);
+                v = fmaf(e.diag[n], to_f32<TS>(skip[(size_t)m * e.ldo + n]), v);
+                if (e.add) v += reinterpret_cast<const float*>(e.add)[(size_t)m * e.ldo + n];
             }
             out[(size_t)m * e.ldo + n] = from_f32<TO>(v);
         }
@@ -88,17 +89,22 @@ gemm_tn_kernel(const TA* __restrict__ A, int lda, const TB* __restrict__ Bm, int
 
 template <typename TA, typename TB>
 static void dispatch_tn(const GemmTN& g, cudaStream_t st) {
-    dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM);
+    dim3 grid((g.M + TM - 1) / TM, (g.N + TN - 1) / TN);
     count_launch();
     EpiArgs e{g.out, g.diag, g.skip, g.add, g.N};
     const TA* A = (const TA*)g.A;
     const TB* Bm = (const TB*)g.Bm;
+    using bf = __nv_bfloat16;
     if (g.epi == Epi::StoreF32)
-        gemm_tn_kernel<TA, TB, float, false><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
+        gemm_tn_kernel<TA, TB, float, float, false><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
+    else if (g.out_bf16 && g.skip_bf16)
+        gemm_tn_kernel<TA, TB, bf, bf, true><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
     else if (g.out_bf16)
-        gemm_tn_kernel<TA, TB, __nv_bfloat16, true><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
+        gemm_tn_kernel<TA, TB, bf, float, true><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
+    else if (g.skip_bf16)
+        gemm_tn_kernel<TA, TB, float, bf, true><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
     else
-        gemm_tn_kernel<TA, TB, float, true><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
+        gemm_tn_kernel<TA, TB, float, float, true><<<grid, kGemmThreads, 0, st>>>(A, g.lda, Bm, g.ldb, g.M, g.N, g.K, e);
 }
 
 void launch_gemm_tn(const GemmTN& g, cudaStream_t st) {

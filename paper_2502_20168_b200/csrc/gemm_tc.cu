@@ -1620,16 +1620,7 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
+static int sm_count() { return device_sm_count(); }
 
 // How many clusters of two CTAs of `kernel` the current device runs at the same time (cached per
 // kernel and device).

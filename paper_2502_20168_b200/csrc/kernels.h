@@ -42,8 +42,8 @@ int launch_scan_bwd_stream(int B, int T, int P, const float2* Abar, const float2
 // out[c] = sum_r in[r, c]; `tmp` must hold colsum_tmp_floats(R, C) floats.  Deterministic.
 void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaStream_t st);
 size_t colsum_tmp_floats(int R, int C);
-// out[c] = sum_m a[m,c]*b[m,c] (a, b in io dtype).
-void launch_dot_columns(bool bf16, const void* a, const void* b, int M, int C, float* out, float* tmp,
+// out[c] = sum_m a[m,c]*b[m,c]; a and b each fp32 or bf16.
+void launch_dot_columns(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* out, float* tmp,
                         cudaStream_t st);
 size_t dot_columns_tmp_floats(int M, int C);
 
@@ -57,8 +57,8 @@ struct GemmTN {
     int M, N, K;
     Epi epi;
     void* out; bool out_bf16;            // StoreF32 ignores out_bf16
-    const float* diag; const void* skip; // io dtype = out dtype
-    const void* add;                     // optional, io dtype
+    const float* diag; const void* skip; bool skip_bf16;
+    const float* add;                    // optional, fp32 [M, N]
 };
 void launch_gemm_tn(const GemmTN& g, cudaStream_t st);
 
@@ -168,12 +168,14 @@ void launch_glu_gv(bool io_bf16, size_t n, const void* v, const void* gout, cons
 void launch_glu_reduce(const float* part, int splits, size_t n, float* out, cudaStream_t st);
 
 // stack.cu: out = LayerNorm(u + GELU(v)) * w + b per row of H features, and its backward
-// (gzr = round(LN'(g)), gv = round(gz * GELU'(v)), dw, db).  tmp: stack_tmp_floats(M, H) floats.
+// (gz = LN'(g), gv = gz * GELU'(v), dw, db).  v, gz, gv are fp32; u, out and g are fp32 or bf16 as
+// flagged (only the stack's own input, output and output gradient are in the I/O type).
+// tmp: stack_tmp_floats(M, H) floats.
 size_t stack_tmp_floats(int M, int H);
-void launch_stack_fwd(bool bf16, int M, int H, const void* u, const void* v, const float* w, const float* b, void* out,
-                      float* mu, float* rstd, cudaStream_t st);
-void launch_stack_bwd(bool bf16, int M, int H, const void* g, const void* u, const void* v, const float* w,
-                      const float* mu, const float* rstd, void* gzr, void* gv, float* dw, float* db, float* tmp,
-                      cudaStream_t st);
+void launch_stack_fwd(bool u_bf16, bool out_bf16, int M, int H, const void* u, const float* v, const float* w,
+                      const float* b, void* out, float* mu, float* rstd, cudaStream_t st);
+void launch_stack_bwd(bool g_bf16, bool u_bf16, int M, int H, const void* g, const void* u, const float* v,
+                      const float* w, const float* mu, const float* rstd, float* gz, float* gv, float* dw, float* db,
+                      float* tmp, cudaStream_t st);
 
 }  // namespace ssm

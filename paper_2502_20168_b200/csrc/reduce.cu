@@ -5,13 +5,13 @@ namespace ssm {
 
 constexpr int kRowsPerBlock = 64;
 
-// block = 32 columns x 8 row lanes; grid.x = ceil(C/32), grid.y = row groups.
+// block = 32 columns x 8 row lanes; grid.x = row groups (the dimension that grows with B*T), grid.y = ceil(C/32).
 // out[g, c] = sum of in[r, c] for r in group g.
 __global__ void colsum_kernel(const float* __restrict__ in, int R, int C, int rows_per_group,
                               float* __restrict__ out) {
     __shared__ float sm[8][33];
-    const int c = blockIdx.x * 32 + threadIdx.x;
-    const int r0 = blockIdx.y * rows_per_group;
+    const int c = blockIdx.y * 32 + threadIdx.x;
+    const int r0 = blockIdx.x * rows_per_group;
     const int r1 = min(R, r0 + rows_per_group);
     float acc = 0.f;
     if (c < C)
@@ -22,7 +22,7 @@ __global__ void colsum_kernel(const float* __restrict__ in, int R, int C, int ro
         float t = 0.f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x];
-        out[(size_t)blockIdx.y * C + c] = t;
+        out[(size_t)blockIdx.x * C + c] = t;
     }
 }
 
@@ -33,13 +33,13 @@ void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaSt
     const int gx = (C + 31) / 32;
     if (R <= kRowsPerBlock * 2) {
         count_launch();
-        colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(in, R, C, R, out);
+        colsum_kernel<<<dim3(1, gx), blk, 0, st>>>(in, R, C, R, out);
         return;
     }
     const int groups = (R + kRowsPerBlock - 1) / kRowsPerBlock;
     count_launch(2);
-    colsum_kernel<<<dim3(gx, groups), blk, 0, st>>>(in, R, C, kRowsPerBlock, tmp);
-    colsum_kernel<<<dim3(gx, 1), blk, 0, st>>>(tmp, groups, C, groups, out);
+    colsum_kernel<<<dim3(groups, gx), blk, 0, st>>>(in, R, C, kRowsPerBlock, tmp);
+    colsum_kernel<<<dim3(1, gx), blk, 0, st>>>(tmp, groups, C, groups, out);
 }
 
 // part[g, c] = sum_{m in group g} a[m, c] * b[m, c].  A thread owns 4 neighbouring columns
@@ -60,20 +60,20 @@ __device__ __forceinline__ void load_quad<__nv_bfloat16>(const __nv_bfloat16* p,
     v[0] = lo.x; v[1] = lo.y; v[2] = hi.x; v[3] = hi.y;
 }
 
-template <typename T>
+template <typename TA, typename TB>
 __global__ void __launch_bounds__(256)
-dot_columns_kernel(const T* __restrict__ a, const T* __restrict__ b, int M, int C, float* __restrict__ part) {
+dot_columns_kernel(const TA* __restrict__ a, const TB* __restrict__ b, int M, int C, float* __restrict__ part) {
     __shared__ float4 sm[8][33];
-    const int c = (blockIdx.x * 32 + threadIdx.x) * 4;
-    const int r0 = blockIdx.y * kDotRows;
+    const int c = (blockIdx.y * 32 + threadIdx.x) * 4;
+    const int r0 = blockIdx.x * kDotRows;
     const int r1 = min(M, r0 + kDotRows);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     if (c < C) {
 #pragma unroll 4
         for (int r = r0 + threadIdx.y; r < r1; r += 8) {
             float va[4], vb[4];
-            load_quad<T>(a + (size_t)r * C + c, va);
-            load_quad<T>(b + (size_t)r * C + c, vb);
+            load_quad<TA>(a + (size_t)r * C + c, va);
+            load_quad<TB>(b + (size_t)r * C + c, vb);
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[i] = fmaf(va[i], vb[i], acc[i]);
         }
@@ -87,7 +87,7 @@ dot_columns_kernel(const T* __restrict__ a, const T* __restrict__ b, int M, int 
             const float4 v = sm[i][threadIdx.x];
             t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
         }
-        *reinterpret_cast<float4*>(part + (size_t)blockIdx.y * C + c) = t;
+        *reinterpret_cast<float4*>(part + (size_t)blockIdx.x * C + c) = t;
     }
 }
 
@@ -98,15 +98,20 @@ size_t dot_columns_tmp_floats(int M, int C) {
     return (size_t)g * C + colsum_tmp_floats(g, C);
 }
 
-void launch_dot_columns(bool bf16, const void* a, const void* b, int M, int C, float* out, float* tmp,
+void launch_dot_columns(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* out, float* tmp,
                         cudaStream_t st) {
+    using bf = __nv_bfloat16;
     const int g = dot_groups(M);
-    dim3 blk(32, 8), grid((C + 127) / 128, g);
+    dim3 blk(32, 8), grid(g, (C + 127) / 128);   // row groups along x: no 65535 limit there
     count_launch();
-    if (bf16)
-        dot_columns_kernel<__nv_bfloat16><<<grid, blk, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, M, C, tmp);
+    if (a_bf16 && b_bf16)
+        dot_columns_kernel<bf, bf><<<grid, blk, 0, st>>>((const bf*)a, (const bf*)b, M, C, tmp);
+    else if (a_bf16)
+        dot_columns_kernel<bf, float><<<grid, blk, 0, st>>>((const bf*)a, (const float*)b, M, C, tmp);
+    else if (b_bf16)
+        dot_columns_kernel<float, bf><<<grid, blk, 0, st>>>((const float*)a, (const bf*)b, M, C, tmp);
     else
-        dot_columns_kernel<float><<<grid, blk, 0, st>>>((const float*)a, (const float*)b, M, C, tmp);
+        dot_columns_kernel<float, float><<<grid, blk, 0, st>>>((const float*)a, (const float*)b, M, C, tmp);
     launch_colsum(tmp, g, C, out, tmp + (size_t)g * C, st);
 }
 

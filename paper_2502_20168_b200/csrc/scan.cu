@@ -247,8 +247,8 @@ scan_bwd_seq1_kernel(int B, int T, int P, const float2* __restrict__ Abar, const
 template <typename XT>
 __global__ void __launch_bounds__(256)
 scan_fwd_step_kernel(int B, int P2, const float4* __restrict__ Abar, const float4* __restrict__ Alo,
-                     const float4* __restrict__ Bu, const uint8_t* __restrict__ done, const float4* x0, XT* x,
-                     float4* xT) {
+                     const float4* Bu /* may be the array x is written to */, const uint8_t* __restrict__ done,
+                     const float4* x0, XT* x, float4* xT) {
     const int idx = blockIdx.x * 256 + threadIdx.x;
     if (idx >= B * P2) return;
     const int b = idx / P2, pp = idx - b * P2;

@@ -41,6 +41,18 @@ int static_scratch_for_current_device(void** out) {
 
 }  // namespace
 
+// The status word of ssm_scan_bwd_static's kernels sits at the start of the static array, which
+// the caller has no pointer to: this reads it back (and synchronises `stream`, like ssm_check).
+SSM_API int ssm_check_static(void* stream) {
+    void* base = nullptr;
+    if (int rc = static_scratch_for_current_device(&base)) return rc;
+    int status = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&status, base, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SSM_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SSM_ERR_CUDA;
+    return status == 0 ? SSM_OK : SSM_ERR_TIMEOUT;
+}
+
 SSM_API int ssm_scan_bwd_static(const ssm_shape* shape, const ssm_c64* Abar, const uint8_t* done,
                                 const ssm_c64* x0, const ssm_c64* x, const ssm_c64* gx, const ssm_c64* gxT,
                                 ssm_c64* gBu, ssm_c64* gAbar, ssm_c64* gx0, void* stream) {

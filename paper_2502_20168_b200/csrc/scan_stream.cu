@@ -486,18 +486,7 @@ scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const _
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
-            (void)cudaGetLastError();
-            n = 148;
-        }
-    }
-    return n;
-}
+int sm_count() { return device_sm_count(); }
 
 constexpr int kCtasPerSm = 2;
 

@@ -76,6 +76,44 @@ def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
     run(I.small_variant(w, p_done=0.0))
 
 
+@pytest.mark.parametrize("io,B,T,H,P", [("f32", 3, 50, 40, 24), ("bf16", 80, 128, 256, 128), ("bf16", 5, 77, 256, 128)])
+def test_conjugate_symmetric_variant_is_the_layer_with_half_the_states_and_doubled_C(io, B, T, H, P):
+    """A system whose P states come in conjugate pairs is stored as its first P/2 states and run as
+    this layer with C doubled (y = 2 Re(C_half x_half)).  The CUDA layer called that way is compared
+    with the oracle on the FULL P-state system: y and du as they are, x_T on the stored half, and the
+    half system's parameter gradients as the sums over each pair (g and conj(g)); the gradient with
+    respect to C_half is twice the gradient the layer returns for the doubled C."""
+    from oracle import ssm_oracle as O
+    from paper_2502_20168_b200 import harness
+    Ph = P // 2
+    w = I.Workload("conj", B=B, T=T, H=H, P=Ph, io_dtype=io, p_done=0.03, seed=B + T + P)
+    d = I.draw_layer(w, with_x0=True, with_gxT=False)
+    Lam = np.concatenate([d["Lambda"], np.conj(d["Lambda"])])
+    Dl = np.concatenate([d["Delta"], d["Delta"]])
+    Bc = np.concatenate([d["Bc"], np.conj(d["Bc"])], axis=0)
+    Cc = np.concatenate([d["Cc"], np.conj(d["Cc"])], axis=1)
+    x0 = np.concatenate([d["x0"], np.conj(d["x0"])], axis=1)
+    y, xT, _ = O.ssm_layer_fwd(Lam, Dl, Bc, Cc, d["D"], d["u"], d["done"], x0)
+    g = O.ssm_layer_bwd(Lam, Dl, Bc, Cc, d["D"], d["u"], d["done"], x0, d["gy"])
+    half = dict(d)
+    half["Cc"] = (2.0 * d["Cc"]).astype(np.complex64)      # exact in fp32
+    res = harness.run_layer(half, io, with_x0=True)
+    tol = TOL[io]
+    pair = lambda a, ax: np.take(a, range(Ph), axis=ax) + np.conj(np.take(a, range(Ph, P), axis=ax))
+    errs = {
+        "y": assert_close("y", res["y"], y, tol),
+        "xT": assert_close("xT", res["xT"], xT[:, :Ph], tol),
+        "du": assert_close("du", res["du"], g["du"], tol),
+        "dD": assert_close("dD", res["dD"], g["dD"], tol),
+        "dB": assert_close("dB", res["dB"], pair(g["dB"], 0), tol),
+        "dLambda": assert_close("dLambda", res["dLambda"], pair(g["dLambda"], 0), tol),
+        "dDelta": assert_close("dDelta", res["dDelta"], g["dDelta"][:Ph] + g["dDelta"][Ph:], tol),
+        "dC_half": assert_close("dC_half", 2.0 * res["dC"], pair(g["dC"], 1), tol),
+        "dx0": assert_close("dx0", res["dx0"], pair(g["dx0"], 1), tol),
+    }
+    print(w.name, {k: f"{v:.1e}" for k, v in errs.items()})
+
+
 @pytest.mark.parametrize("io", ["f32", "bf16"])
 def test_every_step_flagged_and_no_flags(io):
     w = I.Workload("all", B=2, T=40, H=32, P=16, io_dtype=io, p_done=0.5, seed=5)

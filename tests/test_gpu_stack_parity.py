@@ -1,13 +1,8 @@
-"""Stacked model (SSM -> GELU -> residual -> LayerNorm per layer) on the GPU vs the oracle with
-the same storage roundings.
-
-What is compared at the 2e-2 / 1e-4 tolerance is each layer block on the oracle's own inputs
-(layer input and incoming gradient taken from the oracle's run), so that only in-layer
-arithmetic differs.  End to end, a rounding to the storage type that falls on the other side
-of a boundary than in the oracle is amplified by the layers that follow (see
-test_oracle_stack_rounding.py).  The end-to-end comparison is therefore only a sanity bound:
-n_layers times the tolerance for out and du, twice that for the parameter gradients (sums over
-all rows, in which the displaced roundings add up)."""
+"""Stacked model (SSM -> GELU -> residual -> LayerNorm per layer) on the GPU against the float64
+oracle, end to end: the stack's output, the input gradient and every layer's parameter gradients
+at the tolerance of the I/O type, elementwise.  The oracle runs in float64 throughout (no storage
+rounding anywhere); the CUDA path keeps what passes between the layers in fp32 and rounds only the
+stack's own output and input gradient to the I/O type."""
 import numpy as np
 import pytest
 
@@ -36,35 +31,16 @@ def run(w, perturb_ln=True):
     from paper_2502_20168_b200 import harness
     d = draw(w, perturb_ln)
     L = w.n_layers
-    rnd = I.round_to_bf16 if w.io_dtype == "bf16" else (lambda a: np.asarray(a, np.float32))
     tol = TOL[w.io_dtype]
-    out, cache = O.stack_fwd(d["params"], d["ln_weight"], d["ln_bias"], d["u"], d["done"], round_io=rnd)
-    du, grads = O.stack_bwd(d["params"], d["ln_weight"], d["ln_bias"], cache, d["done"], d["gy"], round_io=rnd)
-
-    # each block alone, on the oracle's inputs
-    g = np.asarray(d["gy"], np.float64)
-    for l in range(L - 1, -1, -1):
-        sl = slice(l, l + 1)
-        o_ref, c_ref = O.stack_fwd(d["params"][sl], d["ln_weight"][sl], d["ln_bias"][sl], cache[l]["u"], d["done"],
-                                   round_io=rnd)
-        g_ref, gr_ref = O.stack_bwd(d["params"][sl], d["ln_weight"][sl], d["ln_bias"][sl], c_ref, d["done"], g,
-                                    round_io=rnd)
-        one = {"params": d["params"][sl], "ln_weight": d["ln_weight"][sl], "ln_bias": d["ln_bias"][sl],
-               "u": cache[l]["u"].astype(np.float32), "gy": g.astype(np.float32), "done": d["done"]}
-        res = harness.run_stack(one, w.io_dtype)
-        assert_close(f"layer {l} out", res["out"], o_ref, tol)
-        assert_close(f"layer {l} du", res["du"], g_ref, tol)
-        for k in GRADS:
-            assert_close(f"layer {l} {k}", res["grads"][0][k], gr_ref[0][k], tol)
-        g = g_ref
-
-    # the whole stack
+    out, cache = O.stack_fwd(d["params"], d["ln_weight"], d["ln_bias"], d["u"], d["done"])
+    du, grads = O.stack_bwd(d["params"], d["ln_weight"], d["ln_bias"], cache, d["done"], d["gy"])
     res = harness.run_stack(d, w.io_dtype)
-    errs = {"out": assert_close("out", res["out"], out, L * tol), "du": assert_close("du", res["du"], du, L * tol)}
+    errs = {"out": assert_close("out", res["out"], out, tol), "du": assert_close("du", res["du"], du, tol)}
     for l in range(L):
         for k in GRADS:
-            errs[f"{k}{l}"] = assert_close(f"stack layer {l} {k}", res["grads"][l][k], grads[l][k], 2 * L * tol)
-    print(w.name, {k: f"{v:.1e}" for k, v in errs.items() if v > tol / 10})
+            errs[f"{k}[{l}]"] = assert_close(f"layer {l} {k}", res["grads"][l][k], grads[l][k], tol)
+    print(w.name, {k: f"{v:.1e}" for k, v in errs.items()})
+    return errs
 
 
 def test_c2_stack_of_four_bf16():

@@ -1,10 +1,11 @@
-"""Why the stacked configuration is compared block by block: with tensors stored as bf16
-between the blocks, a value that rounds to the other neighbour is a legitimate difference
-between two correct evaluations, and the following layers amplify it.  The oracle is run
-twice on the stacked workload, the second time with a relative perturbation of 1e-7 (fp32
-rounding level) in front of every storage rounding; the two runs differ by more than the
-2e-2 tolerance in some parameter gradient, while each block taken alone on identical inputs
-stays far inside it."""
+"""Why the stacked configuration keeps fp32 between its layers: with the tensors that pass from
+layer to layer stored as bf16, a value that rounds to the other neighbour is a legitimate
+difference between two correct evaluations, and the following layers amplify it.  The oracle is
+run twice on the stacked workload with bf16 storage roundings switched on, the second time with a
+relative perturbation of 1e-7 (fp32 rounding level) in front of every rounding; the two runs
+differ by more than the 2e-2 tolerance in some parameter gradient, while each block taken alone
+on identical inputs stays far inside it.  A comparison at 2e-2 end to end is therefore only
+meaningful without those roundings, which is how the CUDA path stores its inter-layer tensors."""
 import numpy as np
 
 from oracle import ssm_oracle as O
