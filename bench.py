@@ -284,6 +284,111 @@ def time_half_glu(w, torch, sb, steps=10):
             "stage_ms_per_step": {k: round(v_[1] / steps, 4) for k, v_ in stages.items()}}
 
 
+def time_workload(w, torch, sb, harness, steps=10, warmup=3, graph=False):
+    """Forward + backward of one named workload with inputs drawn on the device: CUDA-event time per
+    step, launches per step and the library's per-stage times.  With `graph` also the time of the step
+    captured once in a CUDA graph and replayed (no host work per launch)."""
+    d = harness.device_drawn(w)
+    buf = harness.StackBuffers(d, w.io_dtype) if w.n_layers > 1 else harness.LayerBuffers(d, w.io_dtype)
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        buf.forward(stream)
+        buf.backward(stream)
+    torch.cuda.synchronize()
+    sb.ssm_check(buf.ws)
+    n0 = sb.ssm_launch_count()
+    sb.ssm_profile_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        buf.forward(stream)
+        buf.backward(stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    stages = sb.ssm_profile_end()
+    ms = e0.elapsed_time(e1) / steps
+    out = {"B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype, "n_layers": w.n_layers,
+           "ms_per_step": round(ms, 5), "timesteps_per_sec": w.timesteps / (ms * 1e-3),
+           "launches_per_step": (sb.ssm_launch_count() - n0) / steps,
+           "stage_ms_per_step": {k: round(v[1] / steps, 5) for k, v in stages.items()}}
+    if graph:
+        out["graph_ms_per_step"] = replay_ms(buf, torch, stream)
+    sb.ssm_check(buf.ws)
+    return out
+
+
+def replay_ms(buf, torch, stream, reps=20):
+    """A forward + backward captured once in a CUDA graph and replayed: milliseconds per replay."""
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        buf.forward(side)
+        buf.backward(side)
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(reps):
+        g.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    return round(g0.elapsed_time(g1) / reps, 5)
+
+
+def scan_stage_summary(r, peaks):
+    """The two scan stages of a timed layer step (fused with their projections, or apart) as
+    algorithmic GB/s and as fractions of the measured copy rate and of the nominal 8 TB/s."""
+    s_io = 2 if r["io_dtype"] == "bf16" else 4
+    n = r["B"] * r["T"]
+    out = {}
+    for key in ("gemm_Bu_scan_fwd", "scan_fwd", "gemm_gx_scan_bwd", "scan_bwd"):
+        ms = r["stage_ms_per_step"].get(key)
+        if ms:
+            gbs = STAGE_MODEL[key][1](r["H"], r["P"], s_io) * n / (ms * 1e-3) / 1e9
+            out[key] = {"ms": ms, "algorithmic_GBps": round(gbs, 1), "frac_of_measured_copy": round(gbs / peaks["hbm_gbs"], 4),
+                        "frac_of_8TBps": round(gbs / 8000.0, 4)}
+    return out
+
+
+def time_scans_alone(T, torch, sb, peaks, P=256, rows=262144, steps=10):
+    """ssm_scan_fwd / ssm_scan_bwd on their own (B * T = rows, fp32 complex states in and out):
+    16 P bytes per timestep forward (Bu in, x out), 24 P backward (g_x and x in, s out)."""
+    B = rows // T
+    shape = sb.make_shape(B, T, 8, P, "f32")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(T)
+    cplx = lambda *s: torch.view_as_complex(torch.randn(s + (2,), device="cuda", generator=g))
+    lam = -(0.01 + 0.99 * torch.rand(P, device="cuda", generator=g)) + 1j * 3.14159 * torch.rand(P, device="cuda", generator=g)
+    dt = torch.exp(torch.log(torch.tensor(1e-3)) + torch.rand(P, device="cuda", generator=g) * torch.log(torch.tensor(100.0)))
+    Abar = torch.exp(lam * dt).to(torch.complex64)
+    Bu, gx = cplx(B, T, P), cplx(B, T, P)
+    x, s = torch.empty_like(Bu), torch.empty_like(Bu)
+    gA = torch.empty(P, dtype=torch.complex64, device="cuda")
+    ws = sb.alloc_workspace(sb.ssm_scan_workspace_bytes(shape))
+    stream = torch.cuda.current_stream()
+    res = {"B": B, "T": T, "P": P}
+    for name, call, bytes_per_ts in (
+            ("ssm_scan_fwd", lambda: sb.ssm_scan_fwd(shape, Abar, Bu, None, None, x, None, ws, stream), 16.0 * P),
+            ("ssm_scan_bwd", lambda: sb.ssm_scan_bwd(shape, Abar, None, None, x, gx, None, s, gA, None, ws, stream), 24.0 * P)):
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            call()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        sb.ssm_check(ws)
+        ms = e0.elapsed_time(e1) / steps
+        gbs = bytes_per_ts * rows / (ms * 1e-3) / 1e9
+        res[name] = {"ms": round(ms, 5), "algorithmic_GBps": round(gbs, 1),
+                     "frac_of_measured_copy": round(gbs / peaks["hbm_gbs"], 4), "frac_of_8TBps": round(gbs / 8000.0, 4)}
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -292,6 +397,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the extra measurements reported beside the headline (sweep, scans alone, other configs)")
     ap.add_argument("--allreduce-grads", action="store_true",
                     help="N > 1: also sum the parameter gradients over the ranks every step (one all-reduce of the "
                          "gradient bucket, running under the next step's forward pass), as a data-parallel trainer would")
@@ -472,7 +579,9 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None,
+            "dtype": "bf16-io/bf16-hi+lo-mma/f32-acc+state" if w.io_dtype == "bf16" and not stacked else "f32",
+            "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
                        "p_done": w.p_done, "n_layers": w.n_layers, "l2": "inputs larger than L2 (no flush)"
                        if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}" + (" + gradient all-reduce" if exchange else "")},
@@ -482,6 +591,7 @@ def main():
             "clocks": clocks,
             "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
                          "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
+                         "frac_of_8TBps": (achieved / 8000.0) if bound == "hbm" else None,
                          "algorithmic_per_launch": alg,
                          "floor_ms": {k: round(v * 1e3, 4) for k, v in floors_s.items() if v > 0}, "launches_per_step": n_launch / args.steps,
                          "ms_per_launch": per_launch_s * 1e3},
@@ -493,6 +603,22 @@ def main():
             del buf
             torch.cuda.empty_cache()
             line["half_glu"] = time_half_glu(w, torch, sb)
+        if world == 1 and not args.no_extras:
+            # evidence beside the headline: the whole scan-scaling sweep, the scan entry points on their own,
+            # and the other configurations (eager; the small ones also replayed from a CUDA graph)
+            buf = None
+            torch.cuda.empty_cache()
+            sweep = {}
+            for c in I.C4:
+                r = time_workload(c, torch, sb, harness)
+                sweep[c.name] = {"ms_per_step": r["ms_per_step"], "timesteps_per_sec": r["timesteps_per_sec"],
+                                 "launches_per_step": r["launches_per_step"], "scan_stages": scan_stage_summary(r, peaks)}
+                torch.cuda.empty_cache()
+            line["sweep"] = sweep
+            line["scan_alone"] = {f"T{t}": time_scans_alone(t, torch, sb, peaks) for t in (1024, 16384)}
+            torch.cuda.empty_cache()
+            line["configs"] = {c.name: time_workload(c, torch, sb, harness, steps=20, graph=True)
+                               for c in (I.C0, I.C1, I.C2, I.C3, I.PAPER_STATE, I.PAPER_VISION)}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, max(1, 262144 // w.T)))))
         print(json.dumps(line))

@@ -386,33 +386,38 @@ scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const _
         const float2* in = reinterpret_cast<const float2*>(stage) + row0 * G + col;
 #pragma unroll
         for (int i = 0; i < r; ++i) v[i] = in[i * G];
-        // One true pass over this thread's rows from carry `cc`; results to `out(i, s_i)`.
+        // One true pass over this thread's rows from carry `cc` (= keep conj(Abar) s of the row after the
+        // thread's last); results to `out(i, s_i)`.  Inside the thread's rows the recurrence is one fused
+        // multiply-add per step, s_i = conj(Abar) s_{i+1} + gx_i (one rounding, as in the forward scan); the
+        // carry form conj(Abar) s is only taken at the thread's two ends.
         auto true_pass = [&](float2 cc, auto&& out) -> float2 {
             if (plain) {
+                float2 sv = cadd(v[r - 1], cc);
 #pragma unroll
                 for (int i = r - 1; i >= 0; --i) {
-                    const float2 sv = cadd(v[i], cc);
+                    if (i < r - 1) sv = rstep<kPair>(ac, acl, sv, v[i]);
                     out(i, sv);
                     g = cfma(sv, cconj(TileIO<XS>::get(xtile, R, G, row0 + i, col)), g);
-                    cc = rstep<kPair>(ac, acl, sv, zero2);
                 }
-            } else {
-#pragma unroll
-                for (int i = r - 1; i >= 0; --i)
-                    if (i < valid) {
-                        const float2 sv = cadd(v[i], cc);
-                        out(i, sv);
-                        if ((mask >> i) & 1u) {
-                            cc = zero2;
-                        } else {
-                            const float2 xprev =
-                                (c == 0 && row0 + i == 0) ? xinit : TileIO<XS>::get(xtile, R, G, row0 + i, col);
-                            g = cfma(sv, cconj(xprev), g);
-                            cc = rstep<kPair>(ac, acl, sv, zero2);
-                        }
-                    }
+                return rstep<kPair>(ac, acl, sv, zero2);
             }
-            return cc;
+            float2 sv = zero2;
+            bool have = false, cut = false;   // have: sv is s of the row after row i; cut: that row carries a flag
+#pragma unroll
+            for (int i = r - 1; i >= 0; --i)
+                if (i < valid) {
+                    sv = !have ? cadd(v[i], cc) : (cut ? v[i] : rstep<kPair>(ac, acl, sv, v[i]));
+                    have = true;
+                    out(i, sv);
+                    cut = (mask >> i) & 1u;
+                    if (!cut) {
+                        const float2 xprev =
+                            (c == 0 && row0 + i == 0) ? xinit : TileIO<XS>::get(xtile, R, G, row0 + i, col);
+                        g = cfma(sv, cconj(xprev), g);
+                    }
+                }
+            if (!have) return cc;   // no row of this thread lies inside the sequence
+            return cut ? zero2 : rstep<kPair>(ac, acl, sv, zero2);
         };
         float2 e, m = aR, ml = aRl;
         if (first) {
@@ -420,14 +425,20 @@ scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const _
             m = zero2;
             ml = zero2;
         } else if (plain) {
-            e = rstep<kPair>(ac, acl, v[r - 1], zero2);
+            float2 sv = v[r - 1];
 #pragma unroll
-            for (int i = r - 2; i >= 0; --i) e = rstep<kPair>(ac, acl, cadd(v[i], e), zero2);
+            for (int i = r - 2; i >= 0; --i) sv = rstep<kPair>(ac, acl, sv, v[i]);
+            e = rstep<kPair>(ac, acl, sv, zero2);
         } else {
-            e = zero2;
+            float2 sv = zero2;
+            bool cut = true;   // nothing enters from beyond the thread's rows in this pass
 #pragma unroll
             for (int i = r - 1; i >= 0; --i)
-                if (i < valid) e = ((mask >> i) & 1u) ? zero2 : rstep<kPair>(ac, acl, cadd(v[i], e), zero2);
+                if (i < valid) {
+                    sv = cut ? v[i] : rstep<kPair>(ac, acl, sv, v[i]);
+                    cut = (mask >> i) & 1u;
+                }
+            e = (valid == 0 || cut) ? zero2 : rstep<kPair>(ac, acl, sv, zero2);
             if (mask != 0u) {
                 m = zero2;
                 ml = zero2;

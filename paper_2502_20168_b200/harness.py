@@ -16,6 +16,8 @@ _IO = {"f32": torch.float32, "bf16": torch.bfloat16}
 def to_dev(a, dtype=None, device="cuda"):
     if a is None:
         return None
+    if isinstance(a, torch.Tensor):      # already a tensor (inputs drawn on the device)
+        return (a if dtype is None else a.to(dtype)).to(device).contiguous()
     t = torch.from_numpy(np.ascontiguousarray(a))
     if dtype is not None:
         t = t.to(dtype)
@@ -96,6 +98,21 @@ class LayerBuffers:
     def results(self) -> dict:
         return {k: to_np(getattr(self, k)) for k in
                 ("y", "xT", "du", "dLambda", "dDelta", "dB", "dC", "dD", "dx0")}
+
+
+def device_drawn(w, device="cuda") -> dict:
+    """A workload's tensors for timing runs: the parameters drawn on the host as always, u, gy and the
+    done flags drawn on the device (same distributions; the large tensors never exist on the host).
+    Returns a dict that LayerBuffers / StackBuffers accept."""
+    from . import inputs as I
+    d = I.draw_layer(I.small_variant(w, B=1, T=1))
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed)
+    io = _IO[w.io_dtype]
+    d["u"] = torch.randn((w.B, w.T, w.H), device=device, generator=g).to(io)
+    d["gy"] = torch.randn((w.B, w.T, w.H), device=device, generator=g).to(io)
+    d["done"] = (torch.rand((w.B, w.T), device=device, generator=g) < w.p_done).to(torch.uint8) if w.p_done > 0 else None
+    return d
 
 
 def run_layer(d: dict, io_dtype: str, with_x0=False, with_gxT=False) -> dict:

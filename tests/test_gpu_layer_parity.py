@@ -76,7 +76,7 @@ def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
     run(I.small_variant(w, p_done=0.0))
 
 
-@pytest.mark.parametrize("io,B,T,H,P", [("f32", 3, 50, 40, 24), ("bf16", 80, 128, 256, 128), ("bf16", 5, 77, 256, 128)])
+@pytest.mark.parametrize("io,B,T,H,P", [("f32", 3, 50, 40, 48), ("bf16", 80, 128, 256, 128), ("bf16", 5, 77, 256, 256)])
 def test_conjugate_symmetric_variant_is_the_layer_with_half_the_states_and_doubled_C(io, B, T, H, P):
     """A system whose P states come in conjugate pairs is stored as its first P/2 states and run as
     this layer with C doubled (y = 2 Re(C_half x_half)).  The CUDA layer called that way is compared
