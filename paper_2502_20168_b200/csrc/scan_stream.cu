@@ -272,7 +272,7 @@ scan_fwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_in, const 
         }
         sm.agg_e[tid] = e;
         sm.agg_m[tid] = m;
-        if (kPair) sm.agg_ml[tid] = ml;
+        sm.agg_ml[tid] = ml;
         if (tid == 0 && n > 0) {   // the store of the previous tile has read its stage by now: recycle it
             tma_store_wait_read_n<0>();
             mbar_arrive(smem_u32(&sm.empty[s_prev]));
@@ -287,7 +287,9 @@ scan_fwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_in, const 
             st = sm.agg_e[col];   // group 0 left its final state
             for (int q = 1; q < sl; ++q) {
                 const int o = q * G + col;
-                st = rstep<kPair>(sm.agg_m[o], kPair ? sm.agg_ml[o] : zero2, st, sm.agg_e[o]);
+                // the group multiplier Abar^r always as an fp32 pair: its rounding error is the same at every
+                // join of a chain, so with a single fp32 it grows linearly with the sequence length
+                st = cfma2(sm.agg_m[o], sm.agg_ml[o], st, sm.agg_e[o]);
             }
             if (plain) {
 #pragma unroll
@@ -448,7 +450,7 @@ scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const _
         }
         sm.agg_e[tid] = e;
         sm.agg_m[tid] = m;
-        if (kPair) sm.agg_ml[tid] = ml;
+        sm.agg_ml[tid] = ml;
         if (tid == 0 && n > 0) {   // the store of the previous tile has read its stage by now: recycle it
             tma_store_wait_read_n<0>();
             mbar_arrive(smem_u32(&sm.empty[s_prev]));
@@ -463,7 +465,7 @@ scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const _
             cc = sm.agg_e[(slices - 1) * G + col];   // the last group left its final carry
             for (int q = slices - 2; q > sl; --q) {
                 const int o = q * G + col;
-                cc = rstep<kPair>(sm.agg_m[o], kPair ? sm.agg_ml[o] : zero2, cc, sm.agg_e[o]);
+                cc = cfma2(sm.agg_m[o], sm.agg_ml[o], cc, sm.agg_e[o]);   // (multiplier as an fp32 pair, as in the forward scan)
             }
             cc = true_pass(cc, [&](int i, float2 sv) { TileIO<XS>::put(stage, R, G, row0 + i, col, sv); });
         }
