@@ -1,4 +1,6 @@
 // C-ABI entry points (see include/ssm.h): argument checks, workspace layout, launch order.
+#include <algorithm>
+
 #include "kernels.h"
 
 using namespace ssm;
@@ -55,8 +57,12 @@ LayerPlan plan_layer(const ssm_shape& s, bool allow_tc = true) {
     p.gAbar = take(off, (size_t)s.P * 8);
     p.gBbar = take(off, PH * 8);
     p.scan = take(off, scan_scratch_bytes(s.B, s.T, s.P));
-    p.part = take(off, (size_t)p.splits * 2 * PH * 4);
-    p.dot = take(off, dot_columns_tmp_floats((int)BT, s.H) * 4);
+    p.part = take(off, (size_t)2 * p.splits * 2 * PH * 4);   // split-K partials of gBbar, then those of dC
+    {   // dD: partial column sums of gy * u, from the stand-alone kernel or from the epilogue of the du projection
+        const size_t rows = (size_t)tc_tn_dot_max_rows();
+        const size_t fused = rows * s.H + colsum_tmp_floats((int)rows, s.H);
+        p.dot = take(off, std::max(dot_columns_tmp_floats((int)BT, s.H), fused) * 4);
+    }
     p.total = off;
     return p;
 }
@@ -175,16 +181,19 @@ SSM_API size_t ssm_layer_workspace_bytes(const ssm_shape* shape) {
 static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64* Lambda, const float* Delta,
                           const ssm_c64* Bc, const ssm_c64* Cc, void* ws, cudaStream_t st) {
     StageTimer tm("discretize_pack", st);
+    if (p.tc) {
+        // one kernel (the kernels that scan in the epilogue of a projection want their own column order)
+        launch_discretize_pack_tc(s.H, s.P, tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P),
+                                  tc_gemm_scan_bwd_supported(s.B, s.T, s.H, s.P), (const float2*)Lambda, Delta,
+                                  (const float2*)Bc, (const float2*)Cc, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo),
+                                  at<float2>(ws, p.Bbar), at<void>(ws, p.W0), at<void>(ws, p.W1), at<void>(ws, p.W2),
+                                  at<void>(ws, p.W3), st);
+        return;
+    }
     launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
                       at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
-    if (p.tc)
-        // (the kernel that scans in the epilogue of the projection wants its own column order)
-        launch_pack_operands_tc(s.H, s.P, tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P),
-                                tc_gemm_scan_bwd_supported(s.B, s.T, s.H, s.P), at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
-                                at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
-    else
-        launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
-                             at<void>(ws, p.W3), at<void>(ws, p.W2), at<void>(ws, p.W1), st);
+    launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
+                         at<void>(ws, p.W3), at<void>(ws, p.W2), at<void>(ws, p.W1), st);
 }
 
 // Launch sequence of one layer's forward pass from a prepared workspace.  `hdr` receives the
@@ -469,9 +478,15 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo&
                           ssm_c64* dx0, cudaStream_t st) {
     const int BT = s.B * s.T, P2 = 2 * s.P;
     if (p.tc && !(io.u_bf16 && io.gy_bf16 && io.du_bf16)) return SSM_ERR_DTYPE;
-    float* part = at<float>(ws, p.part);
+    float* part = at<float>(ws, p.part);                       // split-K partials of gBbar ...
+    float* part_c = part + (size_t)p.splits * 2 * s.P * s.H;   // ... and of dC
     const size_t plane = (size_t)BT * s.P * 4;   // bytes of one bf16 plane of a state tensor
     int rc = SSM_OK;
+    // The last sums (gAbar over the sequences, dD over row groups, the two split-K sums) are left to the two
+    // kernels at the end of the pass: what the stages leave are rows of partial sums.
+    const float2* gA_part = nullptr;
+    const float* dD_part = nullptr;
+    int gA_rows = 0, dD_rows = 0;
 
     if (p.tc) {
         if (tc_gemm_scan_bwd_supported(s.B, s.T, s.H, s.P)) {
@@ -479,7 +494,7 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo&
             StageTimer tm("gemm_gx_scan_bwd", st);
             GemmScanBwd g{gy, at<void>(ws, p.W1), s.B, s.T, s.H, s.P, at<float2>(ws, p.Abar), done, (const float2*)x0,
                           (const float2*)gxT, at<void>(ws, p.xs), at<void>(ws, p.gs), nullptr, (float2*)dx0, hdr};
-            if ((rc = launch_gemm_scan_bwd_sum(g, at<float2>(ws, p.gAbar), at<char>(ws, p.scan), st))) return rc;
+            if ((rc = launch_gemm_scan_bwd_part(g, at<char>(ws, p.scan), &gA_part, &gA_rows, st))) return rc;
         } else {
             {   // gx[m, 2p+c] = sum_h gy[m,h] conj(C)_c[h,p]   (weights as hi + lo bf16)
                 StageTimer tm("gemm_gx", st);
@@ -491,27 +506,36 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo&
                 rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done,
                                      (const float2*)x0, at<void>(ws, p.xs), true, at<float2>(ws, p.f32buf),
                                      (const float2*)gxT, at<void>(ws, p.gs), true, at<float2>(ws, p.gAbar), (float2*)dx0,
-                                     hdr, at<char>(ws, p.scan), st);
+                                     hdr, at<char>(ws, p.scan), st, &gA_part, &gA_rows);
                 if (rc) return rc;
             }
         }
-        {   // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h]
+        {   // du[m,h] = sum_k s[m,k] Bq[h,k] + D[h] gy[m,h];  where the kernel can, also dD[h] = sum_m gy[m,h] u[m,h]
+            // from the tiles of gy its epilogue holds anyway (one more operand tile, u, beside each)
             StageTimer tm("gemm_du", st);
             if (du_add) return SSM_ERR_SHAPE;   // the residual addend exists only on the CUDA-core path (stacks)
             GemmTcTN g{at<void>(ws, p.gs), at<void>(ws, p.W3), BT, s.H, P2, false, false, du, D, gy, hdr};
+            int rows = 0;
+            if (tc_tn_dot_supported(BT, s.H, P2)) {
+                g.dot = u;
+                g.dot_part = at<float>(ws, p.dot);
+                g.dot_rows = &rows;
+            }
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+            if (g.dot) {
+                dD_part = at<float>(ws, p.dot);
+                dD_rows = rows;
+            }
         }
         {   // gBbar[p,h] = sum_m s[m,p] u[m,h]
             StageTimer tm("gemm_gBbar", st);
             GemmTcNT g{u, s.H, at<void>(ws, p.gs), at<void>(ws, p.gs + plane), P2, BT, p.splits, part, hdr};
             if ((rc = launch_gemm_tc_nt(g, st))) return rc;
-            launch_splitk_reduce(part, p.splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
         }
         {   // dC[h,p] = sum_m gy[m,h] conj(x[m,p])
             StageTimer tm("gemm_gC", st);
-            GemmTcNT g{gy, s.H, at<void>(ws, p.xs), at<void>(ws, p.xs + plane), P2, BT, p.splits, part, hdr};
+            GemmTcNT g{gy, s.H, at<void>(ws, p.xs), at<void>(ws, p.xs + plane), P2, BT, p.splits, part_c, hdr};
             if ((rc = launch_gemm_tc_nt(g, st))) return rc;
-            launch_splitk_reduce(part, p.splits, s.H, P2, 1, (float2*)dC, st);
         }
     } else {
         {
@@ -525,7 +549,7 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo&
             rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done, (const float2*)x0,
                                  at<void>(ws, p.xs), false, at<float2>(ws, p.gs), (const float2*)gxT,
                                  at<void>(ws, p.gs), false, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
-                                 at<char>(ws, p.scan), st);
+                                 at<char>(ws, p.scan), st, &gA_part, &gA_rows);
             if (rc) return rc;
         }
         {
@@ -538,20 +562,24 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo&
             StageTimer tm("gemm_gBbar", st);
             GemmNT g5{u, io.u_bf16, s.H, at<void>(ws, p.gs), false, P2, BT, p.splits, part};
             launch_gemm_nt(g5, st);
-            launch_splitk_reduce(part, p.splits, s.H, P2, 0, at<float2>(ws, p.gBbar), st);
         }
         {
             StageTimer tm("gemm_gC", st);
-            GemmNT g6{gy, io.gy_bf16, s.H, at<void>(ws, p.xs), false, P2, BT, p.splits, part};
+            GemmNT g6{gy, io.gy_bf16, s.H, at<void>(ws, p.xs), false, P2, BT, p.splits, part_c};
             launch_gemm_nt(g6, st);
-            launch_splitk_reduce(part, p.splits, s.H, P2, 1, (float2*)dC, st);
         }
     }
-    {   // dD[h] = sum_m gy[m,h] u[m,h];  then the adjoint of the discretisation
+    {   // dD[h] = sum_m gy[m,h] u[m,h] (unless the du projection left its partial sums already), the two split-K
+        // sums, then the adjoint of the discretisation with the sums of gAbar and dD folded in
         StageTimer tm("gD_and_discretize_bwd", st);
-        launch_dot_columns(io.gy_bf16, gy, io.u_bf16, u, BT, s.H, dD, at<float>(ws, p.dot), st);
-        launch_discretize_bwd(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.gAbar),
-                              at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, st);
+        if (!dD_part) {
+            float* tmp = at<float>(ws, p.dot);
+            int groups = launch_dot_columns_partial(io.gy_bf16, gy, io.u_bf16, u, BT, s.H, tmp, st);
+            dD_part = launch_reduce_rows(tmp, groups, s.H, tmp + (size_t)groups * s.H, kMaxPartialRows, &dD_rows, st);
+        }
+        launch_splitk_reduce2(part, part_c, p.splits, s.H, P2, at<float2>(ws, p.gBbar), (float2*)dC, st);
+        launch_layer_finalize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, gA_part, gA_rows,
+                              at<float2>(ws, p.gBbar), (float2*)dLambda, dDelta, (float2*)dB, dD_part, dD_rows, dD, st);
     }
     SSM_RETURN_IF_CUDA_ERROR();
     return SSM_OK;

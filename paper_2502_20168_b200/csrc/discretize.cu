@@ -49,14 +49,41 @@ __global__ void discretize_kernel(int H, const float2* __restrict__ Lambda, cons
     for (int h = threadIdx.x; h < H; h += blockDim.x) Bbar[(size_t)p * H + h] = cmul(g, Bc[(size_t)p * H + h]);
 }
 
-// Adjoint.  One block per state p.
-__global__ void discretize_bwd_kernel(int H, const float2* __restrict__ Lambda, const float* __restrict__ Delta,
-                                      const float2* __restrict__ Bc, const float2* __restrict__ gAbar,
+// Adjoint.  One block per state p.  gAbar arrives as gA_rows rows of partial sums ([gA_rows, P], summed here
+// in a fixed order; one row = the finished gradient).  Blocks past the P states (if any) finish dD the same
+// way: dD[h] = sum of the dD_rows rows of dD_part ([dD_rows, H]).
+__global__ void discretize_bwd_kernel(int H, int P, const float2* __restrict__ Lambda, const float* __restrict__ Delta,
+                                      const float2* __restrict__ Bc, const float2* __restrict__ gAbar, int gA_rows,
                                       const float2* __restrict__ gBbar, float2* __restrict__ dLambda,
-                                      float* __restrict__ dDelta, float2* __restrict__ dB) {
+                                      float* __restrict__ dDelta, float2* __restrict__ dB,
+                                      const float* __restrict__ dD_part, int dD_rows, float* __restrict__ dD) {
     __shared__ float2 gamma_s;
     __shared__ float red[2][32];
+    __shared__ double redA[2][32];
+    if ((int)blockIdx.x >= P) {   // columns of dD
+        const int h = ((int)blockIdx.x - P) * blockDim.x + threadIdx.x;
+        if (h < H) {
+            float acc = 0.f;
+            for (int r = 0; r < dD_rows; ++r) acc += dD_part[(size_t)r * H + h];
+            dD[h] = acc;
+        }
+        return;
+    }
     const int p = blockIdx.x;
+    double gar_t = 0.0, gai_t = 0.0;   // this thread's rows of the partial sums of gAbar[p]
+    for (int r = threadIdx.x; r < gA_rows; r += blockDim.x) {
+        const float2 v = gAbar[(size_t)r * P + p];
+        gar_t += (double)v.x;
+        gai_t += (double)v.y;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        gar_t += __shfl_xor_sync(0xffffffffu, gar_t, o);
+        gai_t += __shfl_xor_sync(0xffffffffu, gai_t, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        redA[0][threadIdx.x >> 5] = gar_t;
+        redA[1][threadIdx.x >> 5] = gai_t;
+    }
     const float2 lam = Lambda[p];
     const float dt = Delta[p];
     ZohTerms z = {};
@@ -91,7 +118,11 @@ __global__ void discretize_bwd_kernel(int H, const float2* __restrict__ Lambda, 
             ggi += red[1][w];
         }
         const double lr = lam.x, li = lam.y, d = dt;
-        const double gar = gAbar[p].x, gai = gAbar[p].y;
+        double gar = 0.0, gai = 0.0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+            gar += redA[0][w];
+            gai += redA[1][w];
+        }
         // dgamma/dLambda = (Delta Abar - gamma) / Lambda     (= (Delta Abar Lambda - (Abar-1)) / Lambda^2)
         const double nr = d * z.ar - z.gr, ni = d * z.ai - z.gi;
         const double n = lr * lr + li * li;
@@ -176,6 +207,50 @@ __global__ void pack_operands_tc_kernel(int H, int P, bool pair_cols, bool pair_
     }
 }
 
+// Discretisation and operand packing of the tensor-core path in one kernel: block p computes Abar_p and
+// gamma_p (double precision, one thread), then the row p of Bbar with its packed forms and the packed forms
+// of column p of C.
+__global__ void __launch_bounds__(128)
+discretize_pack_tc_kernel(int H, int P, bool pair_cols, bool pair_cols_C, const float2* __restrict__ Lambda,
+                          const float* __restrict__ Delta, const float2* __restrict__ Bc, const float2* __restrict__ Cc,
+                          float2* __restrict__ Abar, float2* __restrict__ Abar_lo, float2* __restrict__ Bbar,
+                          __nv_bfloat16* __restrict__ WsB, __nv_bfloat16* __restrict__ WsC,
+                          __nv_bfloat16* __restrict__ Cp, __nv_bfloat16* __restrict__ Bq) {
+    __shared__ float2 gamma_s;
+    const int p = blockIdx.x;
+    if (threadIdx.x == 0) {
+        ZohTerms z = zoh_terms(Lambda[p], Delta[p]);
+        const float2 ah = make_float2((float)z.ar, (float)z.ai);
+        Abar[p] = ah;
+        if (Abar_lo) Abar_lo[p] = make_float2((float)(z.ar - (double)ah.x), (float)(z.ai - (double)ah.y));
+        gamma_s = make_float2((float)z.gr, (float)z.gi);
+    }
+    __syncthreads();
+    const float2 g = gamma_s;
+    const int nB = pair_cols ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
+    const int nC = pair_cols_C ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
+    for (int h = threadIdx.x; h < H; h += blockDim.x) {
+        const float2 v = cmul(g, Bc[(size_t)p * H + h]);
+        Bbar[(size_t)p * H + h] = v;
+        store_split(WsB, H, nB, h, v.x);
+        store_split(WsB, H, nB + (pair_cols ? 2 : 1), h, v.y);
+        *reinterpret_cast<__nv_bfloat162*>(Bq + (size_t)h * 2 * P + 2 * p) = __floats2bfloat162_rn(v.x, v.y);
+        const float2 c = Cc[(size_t)h * P + p];
+        *reinterpret_cast<__nv_bfloat162*>(Cp + (size_t)h * 2 * P + 2 * p) = __floats2bfloat162_rn(c.x, -c.y);
+        store_split(WsC, H, nC, h, c.x);
+        store_split(WsC, H, nC + (pair_cols_C ? 2 : 1), h, -c.y);
+    }
+}
+
+void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
+                               const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
+                               void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st) {
+    count_launch();
+    discretize_pack_tc_kernel<<<P, 128, 0, st>>>(H, P, pair_cols_B, pair_cols_C, Lambda, Delta, Bc, Cc, Abar, Abar_lo, Bbar,
+                                                 (__nv_bfloat16*)Wsplit_B, (__nv_bfloat16*)Wsplit_C, (__nv_bfloat16*)Cp,
+                                                 (__nv_bfloat16*)Bq);
+}
+
 void launch_pack_operands_tc(int H, int P, bool pair_cols, bool pair_cols_C, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st) {
     const int threads = 256;
@@ -196,7 +271,17 @@ void launch_discretize_bwd(int H, int P, const float2* Lambda, const float* Delt
                            const float2* gAbar, const float2* gBbar, float2* dLambda, float* dDelta, float2* dB,
                            cudaStream_t st) {
     count_launch();
-    discretize_bwd_kernel<<<P, 128, 0, st>>>(H, Lambda, Delta, Bc, gAbar, gBbar, dLambda, dDelta, dB);
+    discretize_bwd_kernel<<<P, 128, 0, st>>>(H, P, Lambda, Delta, Bc, gAbar, 1, gBbar, dLambda, dDelta, dB, nullptr, 0,
+                                             nullptr);
+}
+
+void launch_layer_finalize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
+                           const float2* gA_part, int gA_rows, const float2* gBbar, float2* dLambda, float* dDelta,
+                           float2* dB, const float* dD_part, int dD_rows, float* dD, cudaStream_t st) {
+    count_launch();
+    const int extra = dD_part ? (H + 127) / 128 : 0;
+    discretize_bwd_kernel<<<P + extra, 128, 0, st>>>(H, P, Lambda, Delta, Bc, gA_part, gA_rows, gBbar, dLambda, dDelta, dB,
+                                                     dD_part, dD_rows, dD);
 }
 
 void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const float2* Cc, void* Bp, void* Bq,

@@ -196,6 +196,33 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
     }
 }
 
+// Both weight-gradient reductions of a layer in one launch: blockIdx.y = 0 sums part0 into out0 in mode 0,
+// blockIdx.y = 1 sums part1 into out1 in mode 1.
+__global__ void splitk_reduce2_kernel(const float* __restrict__ part0, const float* __restrict__ part1, int splits,
+                                      int I, int J, float* __restrict__ out0, float* __restrict__ out1) {
+    const size_t n = (size_t)I * J;
+    const int mode = blockIdx.y;
+    const float* part = mode ? part1 : part0;
+    float* out = mode ? out1 : out0;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        float acc = 0.f;
+        for (int s = 0; s < splits; ++s) acc += part[(size_t)s * n + e];
+        const int i = (int)(e / J), j = (int)(e % J);
+        if (mode == 0)
+            out[((size_t)(j >> 1) * I + i) * 2 + (j & 1)] = acc;
+        else
+            out[((size_t)i * (J >> 1) + (j >> 1)) * 2 + (j & 1)] = (j & 1) ? -acc : acc;
+    }
+}
+
+void launch_splitk_reduce2(const float* part0, const float* part1, int splits, int I, int J, float2* out0, float2* out1,
+                           cudaStream_t st) {
+    const int threads = 256;
+    const int blocks = (int)(((size_t)I * J + threads - 1) / threads);
+    count_launch();
+    splitk_reduce2_kernel<<<dim3(blocks, 2), threads, 0, st>>>(part0, part1, splits, I, J, (float*)out0, (float*)out1);
+}
+
 void launch_splitk_reduce(const float* part, int splits, int I, int J, int mode, float2* out, cudaStream_t st) {
     const int threads = 256;
     const int blocks = (int)(((size_t)I * J + threads - 1) / threads);

@@ -42,9 +42,14 @@ constexpr int kStagingBytes = kTnEpiWarps * 32 * 32 * 4;  // per epilogue warp: 
 constexpr int kMaxDiag = 4096;                  // widest output whose diagonal fits the shared copy
 constexpr int kSkipBytes = kTnEpiWarps * 2 * 32 * 32 * 2;   // two 32 x 32 bf16 skip tiles per epilogue warp
 // Epilogues of the TN kernels: 0 = fp32 result; 1 = bf16(acc + diag * skip); 2 = fp32 result AND
-// a gated bf16 result skip * sigmoid(acc) (needs a staging buffer for each).
-__host__ __device__ constexpr int tn_skip_bytes(int epi) { return epi == 0 ? 0 : kSkipBytes; }
-__host__ __device__ constexpr int tn_diag_bytes(int epi) { return epi == 1 ? kMaxDiag * 4 : 0; }
+// a gated bf16 result skip * sigmoid(acc) (needs a staging buffer for each); 3 = epilogue 1 AND the
+// column sums of skip * dot over the rows this CTA drains (a second operand tile beside every skip
+// tile, per-warp sums in shared memory): CTA pairs only, outputs of at most kDotMaxN columns.
+constexpr int kDotMaxN = 1024;
+__host__ __device__ constexpr int tn_skip_bytes(int epi) { return epi == 0 ? 0 : (epi == 3 ? 2 * kSkipBytes : kSkipBytes); }
+__host__ __device__ constexpr int tn_diag_bytes(int epi) {
+    return epi == 1 ? kMaxDiag * 4 : (epi == 3 ? kDotMaxN * 4 + kTnEpiWarps * (kDotMaxN / 2) * 4 : 0);
+}
 __host__ __device__ constexpr int tn_staging_bytes(int epi) { return epi == 2 ? kStagingBytes + kStagingBytes / 2 : kStagingBytes; }
 constexpr size_t tn_smem_bytes(int epi) {
     return (size_t)kTnStages * kStageBytes + tn_staging_bytes(epi) + tn_skip_bytes(epi) + tn_diag_bytes(epi) +
@@ -258,6 +263,7 @@ struct TnParams {
     WsHeader* hdr;
     const char* a_base;   // A as bytes; rows are K * 2 bytes apart and contiguous
     int a_row_bytes;
+    float* dot_part;      // epilogue 3: [CTAs, ldo] column sums of skip * dot, one row per CTA
 };
 
 // One epilogue warp's share of a finished accumulator tile: rows m0 + 32 (warp % 4) .. + 31, one half
@@ -317,15 +323,17 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         return true;
     }
 
-    // ---- kEpi == 1, 2: the skip operand arrives by TMA
+    // ---- kEpi == 1, 2, 3: the skip operand arrives by TMA (kEpi 3: and the dot operand beside it)
+    constexpr bool kDot = kEpi == 3;
     const int w = warp - 2;
-    uint8_t* skb = s.skipbuf + (size_t)w * 4096;   // two 2 KB skip tiles
+    uint8_t* skb = s.skipbuf + (size_t)w * (kDot ? 8192 : 4096);   // two 2 KB skip tiles (then two dot tiles)
     const uint32_t sbar[2] = {s.skip_full(2 * w), s.skip_full(2 * w + 1)};
     const int swz = (lane >> 1) & 3;               // 64-byte swizzle: chunk c of row `lane` sits at chunk c ^ swz
     auto fetch_skip = [&](int sl) {
         const int b = sl & 1;
-        mbar_expect_tx(sbar[b], 2048);
+        mbar_expect_tx(sbar[b], kDot ? 4096 : 2048);
         tma_load_2d(smem_u32(skb + b * 2048), tmSkip, sbar[b], n_out0 + (slab0 + sl) * 32, row0);
+        if (kDot) tma_load_2d(smem_u32(skb + 4096 + b * 2048), tmGate, sbar[b], n_out0 + (slab0 + sl) * 32, row0);
     };
     if (lane == 0) {
         fence_async_smem();   // (the lanes' reads of the previous tile's last slabs: fenced and joined there)
@@ -396,6 +404,21 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         uint4 sk[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) sk[j] = *reinterpret_cast<const uint4*>(skb + b * 2048 + lane * 64 + ((j ^ swz) << 4));
+        float prod[kDot ? 32 : 1];
+        if (kDot) {   // skip * dot for this lane's row of the slab
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 dt = *reinterpret_cast<const uint4*>(skb + 4096 + b * 2048 + lane * 64 + ((j ^ swz) << 4));
+                const __nv_bfloat162* s2 = reinterpret_cast<const __nv_bfloat162*>(&sk[j]);
+                const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&dt);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 a = __bfloat1622float2(s2[e]), c2 = __bfloat1622float2(d2[e]);
+                    prod[8 * j + 2 * e] = a.x * c2.x;
+                    prod[8 * j + 2 * e + 1] = a.y * c2.y;
+                }
+            }
+        }
         tmem_ld_wait();
         // Every lane has asked for its skip row; the buffer takes the slab after next.  That refill is a
         // write of the async proxy over data just read through the generic proxy: the proxy fences order the
@@ -430,6 +453,24 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         fence_async_smem();
         __syncwarp();
         if (lane == 0 && row0 < p.M) tma_store_2d(tmOut, smem_u32(ob), n_out0 + c, row0);
+        if (kDot) {
+            // Column sums over the warp's 32 rows: at every halving step a lane keeps the half of its values
+            // that its lane bit selects and adds the other lane's; lane l ends with the sum of column l.
+#pragma unroll
+            for (int h = 16; h >= 1; h >>= 1) {
+                const bool upper = (lane & h) != 0;
+#pragma unroll
+                for (int j = 0; j < h; ++j) {
+                    const float send = upper ? prod[j] : prod[j + h];
+                    const float keep = upper ? prod[j + h] : prod[j];
+                    prod[j] = keep + __shfl_xor_sync(0xffffffffu, send, h);
+                }
+            }
+            // this warp's own sums (it always drains the same half of a tile's columns): rows outside M were
+            // read as zero
+            float* acc_col = s.diag + kDotMaxN + (size_t)w * (kDotMaxN / 2) + (n_out0 / BN) * (BN / 2) + sl * 32 + lane;
+            *acc_col += prod[0];
+        }
     }
     return true;
 }
@@ -537,8 +578,13 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 // leader's `tmem_empty` barriers.
 constexpr int kPairStages = 4;
 constexpr int kPairStageBytes = kABytes + kBBytes / 2;
+// (the epilogue with the column sums gives one operand stage up for its second operand tiles and its sums)
+#ifndef SSM_PAIR_STAGES_BF16_EPILOGUE
+#define SSM_PAIR_STAGES_BF16_EPILOGUE 4
+#endif
+__host__ __device__ constexpr int pair_stages(int epi) { return epi == 3 ? 3 : (epi == 1 ? SSM_PAIR_STAGES_BF16_EPILOGUE : kPairStages); }
 constexpr size_t pair_smem_bytes(int epi) {
-    return (size_t)kPairStages * kPairStageBytes + tn_staging_bytes(epi) + tn_skip_bytes(epi) + tn_diag_bytes(epi) + 1024 +
+    return (size_t)pair_stages(epi) * kPairStageBytes + tn_staging_bytes(epi) + tn_skip_bytes(epi) + tn_diag_bytes(epi) + 1024 +
            256;
 }
 
@@ -548,12 +594,15 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                        const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmSkip,
                        const __grid_constant__ CUtensorMap tmGate, TnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, kPairStages, tn_staging_bytes(kEpi), tn_diag_bytes(kEpi), kPairStageBytes,
+    constexpr int kSt = pair_stages(kEpi);
+    const Smem s = carve_smem(smem_raw, kSt, tn_staging_bytes(kEpi), tn_diag_bytes(kEpi), kPairStageBytes,
                               tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
-    if (kEpi == 1)
+    if (kEpi == 1 || kEpi == 3)
         for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
+    if (kEpi == 3)   // the epilogue warps' column sums start at zero
+        for (int i = threadIdx.x; i < kTnEpiWarps * (kDotMaxN / 2); i += kTnThreads) s.diag[kDotMaxN + i] = 0.f;
     // barriers and tensor memory (both CTAs), then the whole pair meets
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) {
@@ -596,6 +645,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                 const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM;
                 const int rows = min(BM, p.M - m0);
                 if (rows > 0) l2_prefetch_bulk(p.a_base + (size_t)m0 * p.a_row_bytes, (uint32_t)rows * p.a_row_bytes);
+                // (asking L2 for the epilogue's operand rows as well made the bf16-epilogue kernels 15 - 30 % slower)
             };
             prefetch_a(pair);
             for (int tile = pair; tile < total && ok; tile += npairs) {
@@ -608,7 +658,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                     const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
                     tma_load_2d_pair(a_dst, &tmA, leader_full0 + 8u * stage, kb * BK, m0);
                     tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full0 + 8u * stage, kb * BK, n0);
-                    if (++stage == kPairStages) {
+                    if (++stage == kSt) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -636,7 +686,7 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                         umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
                                        (uint32_t)((kb | k) != 0));
                     umma_commit_pair(s.empty(stage));
-                    if (++stage == kPairStages) {
+                    if (++stage == kSt) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -661,6 +711,19 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             if ((acc ^= 1) == 0) acc_phase ^= 1u;
         }
         if (lane == 0) tma_store_wait_all();
+        if (kEpi == 3) {
+            // this CTA's column sums: the four warps that drain a column half added in a fixed order, one row
+            // of p.dot_part per CTA (the sum over the CTAs follows in another kernel)
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kTnEpiWarps) : "memory");
+            const float* sums = s.diag + kDotMaxN;
+            for (int n = threadIdx.x - 64; n < p.ldo; n += 32 * kTnEpiWarps) {
+                const int half = (n % BN) / (BN / 2), idx = (n / BN) * (BN / 2) + n % (BN / 2);
+                float t = 0.f;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) t += sums[(size_t)(4 * half + q) * (kDotMaxN / 2) + idx];
+                p.dot_part[(size_t)blockIdx.x * p.ldo + n] = t;
+            }
+        }
     }
     // nobody leaves (or frees tensor memory) while the other CTA may still signal or compute
     tc_fence_before();
@@ -1666,6 +1729,13 @@ bool tc_tn_supported(int M, int N_out, int K, bool split_w) {
 
 static int pair_tiles_of(int M, int n_tiles) { return ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * n_tiles; }
 
+// The bf16 epilogue can also sum skip * dot over the rows (one partial row per CTA) where the pair kernel
+// runs and the output is at most kDotMaxN wide.
+bool tc_tn_dot_supported(int M, int N_out, int K) {
+    return tc_tn_supported(M, N_out, K, false) && N_out <= tc::kDotMaxN && pair_tiles_of(M, N_out / tc::BN) >= tc::sm_count() / 2;
+}
+int tc_tn_dot_max_rows() { return 2 * tc::sm_count(); }
+
 bool tc_tn_gate_supported(int M, int N_out, int K) {
     return tc_tn_supported(M, N_out, K, true) && pair_tiles_of(M, N_out / (tc::BN / 2)) >= tc::sm_count() / 2;
 }
@@ -1674,8 +1744,9 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     using namespace tc;
     const int out_cols = g.split_w ? BN / 2 : BN;
     const int n_tiles = g.N_out / out_cols;
-    const int epi = g.gate_out ? 2 : (g.store_f32 ? 0 : 1);
-    if (epi == 1 && (g.split_w || !g.diag || !g.skip)) return SSM_ERR_SHAPE;
+    const int epi = g.gate_out ? 2 : (g.store_f32 ? 0 : (g.dot ? 3 : 1));
+    if ((epi == 1 || epi == 3) && (g.split_w || !g.diag || !g.skip)) return SSM_ERR_SHAPE;
+    if (epi == 3 && (!g.dot_part || !g.dot_rows || !tc_tn_dot_supported(g.M, g.N_out, g.K))) return SSM_ERR_SHAPE;
     if (epi == 2 && (!g.split_w || !g.store_f32 || !g.skip || !tc_tn_gate_supported(g.M, g.N_out, g.K))) return SSM_ERR_SHAPE;
     CUtensorMap ma, mw, mo, ms, mg;
     if (!make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, BK, BM)) return SSM_ERR_CUDA;
@@ -1690,7 +1761,9 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
         return SSM_ERR_CUDA;
     if (epi == 2 && !make_map(&mg, g.gate_out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B))
         return SSM_ERR_CUDA;
-    TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.diag, g.hdr, (const char*)g.A, g.K * 2};
+    if (epi == 3 && !make_map(&mg, g.dot, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B))
+        return SSM_ERR_CUDA;   // (the dot operand travels in the map slot of the gated result)
+    TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.diag, g.hdr, (const char*)g.A, g.K * 2, g.dot_part};
     const int m_tiles = (g.M + BM - 1) / BM;
     const int pair_tiles = pair_tiles_of(g.M, n_tiles);
     bool ok = true;
@@ -1707,8 +1780,10 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
         const int pairs = ok ? resident_pairs(reinterpret_cast<const void*>(kern), smem) : 0;              \
         ok = ok && pairs > 0;                                                                              \
         if (ok) kern<<<2 * min(pairs, pair_tiles), kTnThreads, smem, st>>>(ma, mw, mo, ms, mg, p);         \
+        if (ok && g.dot_rows) *g.dot_rows = 2 * min(pairs, pair_tiles);                                    \
     } while (0)
-        if (epi == 2) SSM_LAUNCH_PAIR(2, true);
+        if (epi == 3) SSM_LAUNCH_PAIR(3, false);
+        else if (epi == 2) SSM_LAUNCH_PAIR(2, true);
         else if (epi == 1) SSM_LAUNCH_PAIR(1, false);
         else if (g.split_w) SSM_LAUNCH_PAIR(0, true);
         else SSM_LAUNCH_PAIR(0, false);
@@ -1744,13 +1819,20 @@ static bool make_plane_map(CUtensorMap* map, const void* planes, int M, int P) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Fewest (sequence, 64 states) chain pairs for which the kernels that scan in the epilogue of a projection
+// are taken: below it too many CTA pairs would idle while a few walk their chains tile by tile.
+#ifndef SSM_FUSED_MIN_PAIRS
+#define SSM_FUSED_MIN_PAIRS 32   // measured: 32 pairs (16 sequences of 256 states) still beat the separate kernels
+#endif
+static int fused_min_pairs() { return SSM_FUSED_MIN_PAIRS; }
+
 // Chains per 64 states: the sequences, or, when a 128-row tile holds several whole sequences, the tiles.
 static int fs_units(int B, int T) { return T >= tc::BM ? B : (B * T + tc::BM - 1) / tc::BM; }
 
 bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) {
     const bool t_ok = T % tc::BM == 0 || T == 16 || T == 32 || T == 64;
     if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return false;
-    return (2 * P / 128) * ((fs_units(B, T) + 1) / 2) >= tc::sm_count() / 2;   // a chain for every CTA pair
+    return (2 * P / 128) * ((fs_units(B, T) + 1) / 2) >= fused_min_pairs();
 }
 
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
@@ -1776,7 +1858,7 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
 
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) {
     if (T % tc::BM != 0 || H % tc::BK != 0 || P % 64 != 0) return false;
-    return (2 * P / 128) * ((B + 1) / 2) >= tc::sm_count() / 2;   // a chain for every CTA pair
+    return (2 * P / 128) * ((B + 1) / 2) >= fused_min_pairs();
 }
 
 int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {

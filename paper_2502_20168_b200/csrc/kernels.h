@@ -12,6 +12,12 @@ void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, c
 void launch_discretize_bwd(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
                            const float2* gAbar, const float2* gBbar, float2* dLambda, float* dDelta, float2* dB,
                            cudaStream_t st);
+// The adjoint of the discretisation with the last sums of the layer's backward pass folded in: gAbar comes
+// as gA_rows rows of partial sums [gA_rows, P] (one row: the finished gradient), and dD, if dD_part is given,
+// as dD_rows rows [dD_rows, H]; both are summed here in a fixed order.
+void launch_layer_finalize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
+                           const float2* gA_part, int gA_rows, const float2* gBbar, float2* dLambda, float* dDelta,
+                           float2* dB, const float* dD_part, int dD_rows, float* dD, cudaStream_t st);
 void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const float2* Cc, void* Bp, void* Bq,
                           void* Cp, void* Cq, cudaStream_t st);
 
@@ -23,9 +29,13 @@ int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
                     const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr, void* scratch,
                     cudaStream_t st);
 // x and gBu are stored both as fp32 pairs or both as bf16 pairs (x_bf16 == s_bf16).
+// With gA_part / gA_rows (both or neither) the sum over the sequences is left to the caller: *gA_part points
+// at *gA_rows <= kMaxPartialRows rows of P partial sums inside `scratch`, and gAbar is not written.
+constexpr int kMaxPartialRows = 512;
 int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done, const float2* x0,
                     const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
-                    float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st);
+                    float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st,
+                    const float2** gA_part = nullptr, int* gA_rows = nullptr);
 
 // scan_stream.cu: the scans as TMA-fed streaming kernels (a CTA walks whole sequences; all
 // parallelism over time is inside the CTA).  `ticket`: one int of scratch.  The backward pass
@@ -42,10 +52,16 @@ int launch_scan_bwd_stream(int B, int T, int P, const float2* Abar, const float2
 // out[c] = sum_r in[r, c]; `tmp` must hold colsum_tmp_floats(R, C) floats.  Deterministic.
 void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaStream_t st);
 size_t colsum_tmp_floats(int R, int C);
+// Reduces [R, C] partial sums to at most `limit` rows (groups of rows summed in a fixed order; `in` and `tmp`,
+// colsum_tmp_floats(R, C) floats, are both overwritten); returns where the rows are, *rows_out how many.
+const float* launch_reduce_rows(float* in, int R, int C, float* tmp, int limit, int* rows_out, cudaStream_t st);
 // out[c] = sum_m a[m,c]*b[m,c]; a and b each fp32 or bf16.
 void launch_dot_columns(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* out, float* tmp,
                         cudaStream_t st);
 size_t dot_columns_tmp_floats(int M, int C);
+// The group sums only: tmp[g, c] for g < the returned number of groups.
+int launch_dot_columns_partial(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* tmp,
+                               cudaStream_t st);
 
 // gemm_simt.cu: fp32-accumulate CUDA-core GEMMs (exact enough for the fp32 workloads and the
 // fallback for shapes the tensor-core path does not take).
@@ -74,6 +90,9 @@ void launch_gemm_nt(const GemmNT& g, cudaStream_t st);
 // mode 0: complex out[J/2, I]: out[j/2, i].(re if j even else im) = sum_s part[s,i,j]
 // mode 1: complex out[I, J/2]: out[i, j/2] likewise, with the imaginary part negated
 void launch_splitk_reduce(const float* part, int splits, int I, int J, int mode, float2* out, cudaStream_t st);
+// part0 in mode 0 into out0 and part1 in mode 1 into out1, one launch
+void launch_splitk_reduce2(const float* part0, const float* part1, int splits, int I, int J, float2* out0, float2* out1,
+                           cudaStream_t st);
 
 // gemm_tc.cu: bf16 projections on tcgen05 tensor cores (operands by TMA, accumulators in TMEM).
 struct GemmTcTN {
@@ -90,8 +109,16 @@ struct GemmTcTN {
     // Gate (with store_f32, split_w and skip): besides the fp32 result also gate_out[m, n] =
     // bf16(skip[m, n] * sigmoid(acc)).  Only where tc_tn_gate_supported says so.
     void* gate_out = nullptr;
+    // Column sums (with the bf16 epilogue, where tc_tn_dot_supported says so): dot_part[c, n] = sum over the
+    // rows m that CTA c drained of skip[m, n] * dot[m, n]; *dot_rows receives the number of rows c written
+    // (at most tc_tn_dot_max_rows()).  dot: bf16 [M, N_out].
+    const void* dot = nullptr;
+    float* dot_part = nullptr;
+    int* dot_rows = nullptr;
 };
 bool tc_tn_supported(int M, int N_out, int K, bool split_w);
+bool tc_tn_dot_supported(int M, int N_out, int K);
+int tc_tn_dot_max_rows();
 bool tc_tn_gate_supported(int M, int N_out, int K);
 int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st);
 
@@ -131,8 +158,9 @@ struct GemmScanBwd {
 };
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P);
 int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st);
-// scan.cu: the same followed by the sum of gA_part over the sequences (scratch as for launch_scan_bwd)
-int launch_gemm_scan_bwd_sum(GemmScanBwd g, float2* gAbar, void* scratch, cudaStream_t st);
+// scan.cu: the same with gA_part placed in `scratch` (as for launch_scan_bwd) and brought down to
+// *gA_rows <= kMaxPartialRows rows at *gA_part_out; the caller sums those.
+int launch_gemm_scan_bwd_part(GemmScanBwd g, void* scratch, const float2** gA_part_out, int* gA_rows, cudaStream_t st);
 
 struct GemmTcNT {
     // part[s, i, j] = sum_{m in slice s} A[m, i] * (Bm_hi[m, j] + Bm_lo[m, j]);  A bf16 [K, I],
@@ -152,6 +180,10 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 // stacked forms of Bp / Cq (see GemmTcTN);  Cp, Bq: [H, 2P] single bf16.
 void launch_pack_operands_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
                              void* Cp, void* Bq, cudaStream_t st);
+// launch_discretize and launch_pack_operands_tc in one kernel.
+void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
+                               const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
+                               void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st);
 
 // glu.cu: what surrounds the GEMMs of the half-GLU gate out = v * sigmoid(GELU(v) W).
 // Tensor-core path (may be NULL): Wt2 [2H, 2H], the hi/lo stacked operand of z = [x1_hi | x1_lo] W, and

@@ -42,6 +42,27 @@ void launch_colsum(const float* in, int R, int C, float* out, float* tmp, cudaSt
     colsum_kernel<<<dim3(1, gx), blk, 0, st>>>(tmp, groups, C, groups, out);
 }
 
+// Brings a [R, C] array of partial sums down to at most `limit` rows by summing groups of kRowsPerBlock rows
+// (fixed order), alternating between `in` and `tmp` (colsum_tmp_floats(R, C) floats); both are overwritten.
+// Returns where the remaining rows are and how many.
+const float* launch_reduce_rows(float* in, int R, int C, float* tmp, int limit, int* rows_out, cudaStream_t st) {
+    dim3 blk(32, 8);
+    const int gx = (C + 31) / 32;
+    float* cur = in;
+    float* other = tmp;
+    while (R > limit) {
+        const int groups = (R + kRowsPerBlock - 1) / kRowsPerBlock;
+        count_launch();
+        colsum_kernel<<<dim3(groups, gx), blk, 0, st>>>(cur, R, C, kRowsPerBlock, other);
+        float* t = cur;
+        cur = other;
+        other = t;
+        R = groups;
+    }
+    *rows_out = R;
+    return cur;
+}
+
 // part[g, c] = sum_{m in group g} a[m, c] * b[m, c].  A thread owns 4 neighbouring columns
 // (16 bytes of fp32, 8 bytes of bf16 per load); block = 32 column quads x 8 row lanes.
 constexpr int kDotRows = 128;
@@ -113,6 +134,24 @@ void launch_dot_columns(bool a_bf16, const void* a, bool b_bf16, const void* b, 
     else
         dot_columns_kernel<float, float><<<grid, blk, 0, st>>>((const float*)a, (const float*)b, M, C, tmp);
     launch_colsum(tmp, g, C, out, tmp + (size_t)g * C, st);
+}
+
+// The same without the final sum: the group sums stay in tmp[0 .. groups * C); returns the number of groups.
+int launch_dot_columns_partial(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* tmp,
+                               cudaStream_t st) {
+    using bf = __nv_bfloat16;
+    const int g = dot_groups(M);
+    dim3 blk(32, 8), grid(g, (C + 127) / 128);
+    count_launch();
+    if (a_bf16 && b_bf16)
+        dot_columns_kernel<bf, bf><<<grid, blk, 0, st>>>((const bf*)a, (const bf*)b, M, C, tmp);
+    else if (a_bf16)
+        dot_columns_kernel<bf, float><<<grid, blk, 0, st>>>((const bf*)a, (const float*)b, M, C, tmp);
+    else if (b_bf16)
+        dot_columns_kernel<float, bf><<<grid, blk, 0, st>>>((const float*)a, (const bf*)b, M, C, tmp);
+    else
+        dot_columns_kernel<float, float><<<grid, blk, 0, st>>>((const float*)a, (const float*)b, M, C, tmp);
+    return g;
 }
 
 }  // namespace ssm

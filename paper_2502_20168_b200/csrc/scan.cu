@@ -336,7 +336,8 @@ int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
 
 int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, const uint8_t* done, const float2* x0,
                     const void* x, bool x_bf16, const float2* gx, const float2* gxT, void* gBu, bool s_bf16,
-                    float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st) {
+                    float2* gAbar, float2* gx0, WsHeader* hdr, void* scratch, cudaStream_t st,
+                    const float2** gA_part, int* gA_rows) {
     const ScanPlan s = plan_scan(B, P);
     char* base = (char*)scratch;
     float* part = reinterpret_cast<float*>(base + s.off_part);
@@ -356,18 +357,21 @@ int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
             scan_bwd_seq1_kernel<float2><<<blocks1, kSeqThreads, 0, st>>>(
                 B, T, P, Abar, Alo, done, x0, (const float2*)x, gx, gxT, (float2*)gBu, (float2*)part, gx0);
     }
-    launch_colsum(part, B, 2 * P, (float*)gAbar, tmp, st);
+    if (gA_part && gA_rows)
+        *gA_part = reinterpret_cast<const float2*>(launch_reduce_rows(part, B, 2 * P, tmp, kMaxPartialRows, gA_rows, st));
+    else
+        launch_colsum(part, B, 2 * P, (float*)gAbar, tmp, st);
     return SSM_OK;
 }
 
-int launch_gemm_scan_bwd_sum(GemmScanBwd g, float2* gAbar, void* scratch, cudaStream_t st) {
+int launch_gemm_scan_bwd_part(GemmScanBwd g, void* scratch, const float2** gA_part_out, int* gA_rows, cudaStream_t st) {
     const ScanPlan s = plan_scan(g.B, g.P);
     char* base = (char*)scratch;
     float* part = reinterpret_cast<float*>(base + s.off_part);
     float* tmp = reinterpret_cast<float*>(base + s.off_tmp);
     g.gA_part = reinterpret_cast<float2*>(part);
     if (int rc = launch_gemm_scan_bwd(g, st)) return rc;
-    launch_colsum(part, g.B, 2 * g.P, (float*)gAbar, tmp, st);
+    *gA_part_out = reinterpret_cast<const float2*>(launch_reduce_rows(part, g.B, 2 * g.P, tmp, kMaxPartialRows, gA_rows, st));
     return SSM_OK;
 }
 
