@@ -13,11 +13,28 @@ namespace {
 //  * tensor-core path (bf16 I/O and tile-sized H, P): projections on tcgen05, states Bu / g_x
 //    in one fp32 buffer, x and s kept as bf16 pairs;
 //  * CUDA-core path (fp32 I/O, or odd shapes): fp32 weights and states throughout.
+//  * plane path (fp32 I/O and tile-sized H, P with enough rows): the same projections on tcgen05 as sums
+//    of products of bf16 planes (three planes per fp32 value: exact), fp32 states, scans as on the
+//    CUDA-core path.
 struct LayerPlan {
     bool tc;
+    bool planes;
     int splits;
     size_t hdr, Abar, Alo, Bbar, W0, W1, W2, W3, f32buf, xs, gs, gAbar, gBbar, scan, part, dot, total;
+    size_t u3, gy3, x3, s3, acc;   // plane path: planes of u, gy, x, s and the fp32 result of a projection
 };
+
+#ifndef SSM_PLANES_MIN_ROWS
+#define SSM_PLANES_MIN_ROWS 1   // fewest B*T rows for which fp32 layers take the plane path
+#endif
+bool planes_supported(const ssm_shape& s) {
+    const long long BT = (long long)s.B * s.T;
+    return s.H % 256 == 0 && s.P % 128 == 0 && s.H <= tc_max_n() && 2 * s.P <= tc_max_n() && BT >= SSM_PLANES_MIN_ROWS;
+}
+// Product schedules (plane of the first operand, plane of the second, four bits each, smallest terms first):
+// fp32 x fp32 = lo hi, hi lo, mid mid, mid hi, hi mid, hi hi;  bf16 x fp32 = hi lo, hi mid, hi hi.
+constexpr uint32_t kProd6A = 0x001102u, kProd6B = 0x010120u;
+constexpr uint32_t kProd3A = 0x000u, kProd3B = 0x012u;
 
 size_t take(size_t& off, size_t bytes) {
     const size_t at = off;
@@ -32,7 +49,8 @@ LayerPlan plan_layer(const ssm_shape& s, bool allow_tc = true) {
     const int P2 = 2 * s.P;
     p.tc = allow_tc && s.io_dtype == SSM_BF16 && tc_tn_supported((int)BT, P2, s.H, true) &&
            tc_tn_supported((int)BT, s.H, P2, false) && tc_nt_supported(s.H, P2);
-    p.splits = p.tc ? tc_nt_splits((int)BT, s.H, P2) : gemm_nt_splits((int)BT);
+    p.planes = !p.tc && s.io_dtype == SSM_F32 && planes_supported(s);
+    p.splits = p.tc ? tc_nt_splits((int)BT, s.H, P2) : (p.planes ? tc_nt_multi_splits((int)BT, s.H, P2) : gemm_nt_splits((int)BT));
     p.hdr = take(off, sizeof(WsHeader));
     p.Abar = take(off, (size_t)s.P * 8);
     p.Alo = take(off, (size_t)s.P * 8);
@@ -46,13 +64,21 @@ LayerPlan plan_layer(const ssm_shape& s, bool allow_tc = true) {
         p.xs = take(off, BT * s.P * 8);       // x as two bf16 planes (hi, lo)
         p.gs = take(off, BT * s.P * 8);       // s as two bf16 planes (hi, lo)
     } else {
-        p.W0 = take(off, 2 * PH * 4);   // Bp [2P, H]
-        p.W1 = take(off, 2 * PH * 4);   // Cq [2P, H]
-        p.W2 = take(off, 2 * PH * 4);   // Cp [H, 2P]
-        p.W3 = take(off, 2 * PH * 4);   // Bq [H, 2P]
+        // CUDA-core path: fp32 operands.  Plane path: three bf16 planes of each (6 PH values, 2 bytes each).
+        p.W0 = take(off, p.planes ? 6 * PH * 2 : 2 * PH * 4);   // Bp [2P, H]   | Wb3 [2P, 3H]
+        p.W1 = take(off, p.planes ? 6 * PH * 2 : 2 * PH * 4);   // Cq [2P, H]   | Cq3 [2P, 3H]
+        p.W2 = take(off, p.planes ? 6 * PH * 2 : 2 * PH * 4);   // Cp [H, 2P]   | Cp3 [H, 3 * 2P]
+        p.W3 = take(off, p.planes ? 6 * PH * 2 : 2 * PH * 4);   // Bq [H, 2P]   | Bq3 [H, 3 * 2P]
         p.f32buf = off;                 // unused
         p.xs = take(off, BT * s.P * 8); // Bu, overwritten in place by x
         p.gs = take(off, BT * s.P * 8); // g_x, overwritten in place by s
+        if (p.planes) {
+            p.u3 = take(off, BT * 3 * s.H * 2);
+            p.gy3 = take(off, BT * 3 * s.H * 2);
+            p.x3 = take(off, BT * 6 * s.P * 2);
+            p.s3 = take(off, BT * 6 * s.P * 2);
+            p.acc = take(off, BT * s.H * 4);
+        }
     }
     p.gAbar = take(off, (size_t)s.P * 8);
     p.gBbar = take(off, PH * 8);
@@ -190,6 +216,12 @@ static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
                                   at<void>(ws, p.W3), st);
         return;
     }
+    if (p.planes) {
+        launch_discretize_pack_planes(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, (const float2*)Cc,
+                                      at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar),
+                                      at<void>(ws, p.W0), at<void>(ws, p.W1), at<void>(ws, p.W2), at<void>(ws, p.W3), st);
+        return;
+    }
     launch_discretize(s.H, s.P, (const float2*)Lambda, Delta, (const float2*)Bc, at<float2>(ws, p.Abar),
                       at<float2>(ws, p.Alo), at<float2>(ws, p.Bbar), st);
     launch_pack_operands(s.H, s.P, false, at<float2>(ws, p.Bbar), (const float2*)Cc, at<void>(ws, p.W0),
@@ -244,6 +276,39 @@ static int layer_fwd_run(const ssm_shape& s, const LayerPlan& p, const LayerIo& 
             StageTimer tm("gemm_y", st);
             GemmTcTN g{at<void>(ws, p.xs), at<void>(ws, p.W2), BT, s.H, P2, false, false, y, D, u, hdr};
             if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+    } else if (p.planes) {
+        {   // Bu = u Bbar^T as a sum of plane products (u: three planes of an fp32 input, or the bf16 input itself)
+            StageTimer tm("gemm_Bu", st);
+            if (!io.u_bf16) launch_split_planes((const float*)u, (size_t)BT, s.H, at<void>(ws, p.u3), st);
+            GemmTcTN g{io.u_bf16 ? u : at<void>(ws, p.u3), at<void>(ws, p.W0), BT, P2, s.H, false, true, at<void>(ws, p.xs),
+                       nullptr, nullptr, hdr};
+            g.n_products = io.u_bf16 ? 3 : 6;
+            g.planes_a = io.u_bf16 ? 1 : 3;
+            g.planes_w = 3;
+            g.prod_a = io.u_bf16 ? kProd3A : kProd6A;
+            g.prod_w = io.u_bf16 ? kProd3B : kProd6B;
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+        {
+            StageTimer tm("scan_fwd", st);
+            rc = launch_scan_fwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), at<float2>(ws, p.xs), done,
+                                 (const float2*)x0, at<void>(ws, p.xs), false, (float2*)xT, hdr,
+                                 at<char>(ws, p.scan), st);
+            if (rc) return rc;
+        }
+        {   // y = x Cp^T + D u: planes of x, six products, then the skip term
+            StageTimer tm("gemm_y", st);
+            launch_split_planes(at<float>(ws, p.xs), (size_t)BT, P2, at<void>(ws, p.x3), st);
+            GemmTcTN g{at<void>(ws, p.x3), at<void>(ws, p.W2), BT, s.H, P2, false, true, at<void>(ws, p.acc), nullptr,
+                       nullptr, hdr};
+            g.n_products = 6;
+            g.planes_a = 3;
+            g.planes_w = 3;
+            g.prod_a = kProd6A;
+            g.prod_w = kProd6B;
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+            launch_diag_skip(at<float>(ws, p.acc), D, u, io.u_bf16, nullptr, (size_t)BT, s.H, y, io.y_bf16, st);
         }
     } else {
         {
@@ -535,6 +600,61 @@ static int layer_bwd_impl(const ssm_shape& s, const LayerPlan& p, const LayerIo&
         {   // dC[h,p] = sum_m gy[m,h] conj(x[m,p])
             StageTimer tm("gemm_gC", st);
             GemmTcNT g{gy, s.H, at<void>(ws, p.xs), at<void>(ws, p.xs + plane), P2, BT, p.splits, part_c, hdr};
+            if ((rc = launch_gemm_tc_nt(g, st))) return rc;
+        }
+    } else if (p.planes) {
+        const bool gyb = io.gy_bf16, ub = io.u_bf16;
+        {   // g_x = gy conj(C)
+            StageTimer tm("gemm_gx", st);
+            if (!gyb) launch_split_planes((const float*)gy, (size_t)BT, s.H, at<void>(ws, p.gy3), st);
+            GemmTcTN g{gyb ? gy : at<void>(ws, p.gy3), at<void>(ws, p.W1), BT, P2, s.H, false, true, at<void>(ws, p.gs),
+                       nullptr, nullptr, hdr};
+            g.n_products = gyb ? 3 : 6;
+            g.planes_a = gyb ? 1 : 3;
+            g.planes_w = 3;
+            g.prod_a = gyb ? kProd3A : kProd6A;
+            g.prod_w = gyb ? kProd3B : kProd6B;
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+        }
+        {
+            StageTimer tm("scan_bwd", st);
+            rc = launch_scan_bwd(s.B, s.T, s.P, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo), done, (const float2*)x0,
+                                 at<void>(ws, p.xs), false, at<float2>(ws, p.gs), (const float2*)gxT,
+                                 at<void>(ws, p.gs), false, at<float2>(ws, p.gAbar), (float2*)dx0, hdr,
+                                 at<char>(ws, p.scan), st, &gA_part, &gA_rows);
+            if (rc) return rc;
+        }
+        {   // du = s Bq^T + D gy (+ the residual branch's gradient)
+            StageTimer tm("gemm_du", st);
+            launch_split_planes(at<float>(ws, p.gs), (size_t)BT, P2, at<void>(ws, p.s3), st);
+            GemmTcTN g{at<void>(ws, p.s3), at<void>(ws, p.W3), BT, s.H, P2, false, true, at<void>(ws, p.acc), nullptr,
+                       nullptr, hdr};
+            g.n_products = 6;
+            g.planes_a = 3;
+            g.planes_w = 3;
+            g.prod_a = kProd6A;
+            g.prod_w = kProd6B;
+            if ((rc = launch_gemm_tc_tn(g, st))) return rc;
+            launch_diag_skip(at<float>(ws, p.acc), D, gy, gyb, du_add, (size_t)BT, s.H, du, io.du_bf16, st);
+        }
+        {   // gBbar = s^T u
+            StageTimer tm("gemm_gBbar", st);
+            GemmTcNT g{ub ? u : at<void>(ws, p.u3), s.H, at<void>(ws, p.s3), nullptr, P2, BT, p.splits, part, hdr};
+            g.n_products = ub ? 3 : 6;
+            g.planes_a = ub ? 1 : 3;
+            g.planes_b = 3;
+            g.prod_a = ub ? kProd3A : kProd6A;
+            g.prod_b = ub ? kProd3B : kProd6B;
+            if ((rc = launch_gemm_tc_nt(g, st))) return rc;
+        }
+        {   // dC = gy^T conj(x)
+            StageTimer tm("gemm_gC", st);
+            GemmTcNT g{gyb ? gy : at<void>(ws, p.gy3), s.H, at<void>(ws, p.x3), nullptr, P2, BT, p.splits, part_c, hdr};
+            g.n_products = gyb ? 3 : 6;
+            g.planes_a = gyb ? 1 : 3;
+            g.planes_b = 3;
+            g.prod_a = gyb ? kProd3A : kProd6A;
+            g.prod_b = gyb ? kProd3B : kProd6B;
             if ((rc = launch_gemm_tc_nt(g, st))) return rc;
         }
     } else {

@@ -242,6 +242,62 @@ discretize_pack_tc_kernel(int H, int P, bool pair_cols, bool pair_cols_C, const 
     }
 }
 
+// The same for the projections that run as sums of bf16 plane products (fp32 inputs and outputs): every
+// operand as three planes side by side along its K.
+//   Wb3[2p+c, a H + h] = plane a of (c ? Im : Re) Bbar[p,h]       [2P, 3H]   (Bu = u Wb3^T)
+//   Cq3[2p+c, a H + h] = plane a of (c ? -Im : Re) C[h,p]         [2P, 3H]   (g_x = gy Cq3^T)
+//   Cp3[h, a 2P + 2p+c] = plane a of (c ? -Im : Re) C[h,p]        [H, 3 2P]  (y = x Cp3^T)
+//   Bq3[h, a 2P + 2p+c] = plane a of (c ? Im : Re) Bbar[p,h]      [H, 3 2P]  (du = s Bq3^T)
+__device__ __forceinline__ void store3(__nv_bfloat16* base, size_t plane_stride, float v) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    base[0] = hi;
+    base[plane_stride] = mid;
+    base[2 * plane_stride] = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+}
+
+__global__ void __launch_bounds__(128)
+discretize_pack_planes_kernel(int H, int P, const float2* __restrict__ Lambda, const float* __restrict__ Delta,
+                              const float2* __restrict__ Bc, const float2* __restrict__ Cc, float2* __restrict__ Abar,
+                              float2* __restrict__ Abar_lo, float2* __restrict__ Bbar, __nv_bfloat16* __restrict__ Wb3,
+                              __nv_bfloat16* __restrict__ Cq3, __nv_bfloat16* __restrict__ Cp3,
+                              __nv_bfloat16* __restrict__ Bq3) {
+    __shared__ float2 gamma_s;
+    const int p = blockIdx.x;
+    if (threadIdx.x == 0) {
+        ZohTerms z = zoh_terms(Lambda[p], Delta[p]);
+        const float2 ah = make_float2((float)z.ar, (float)z.ai);
+        Abar[p] = ah;
+        if (Abar_lo) Abar_lo[p] = make_float2((float)(z.ar - (double)ah.x), (float)(z.ai - (double)ah.y));
+        gamma_s = make_float2((float)z.gr, (float)z.gi);
+    }
+    __syncthreads();
+    const float2 g = gamma_s;
+    const size_t H3 = 3 * (size_t)H, P6 = 6 * (size_t)P;
+    for (int h = threadIdx.x; h < H; h += blockDim.x) {
+        const float2 v = cmul(g, Bc[(size_t)p * H + h]);
+        Bbar[(size_t)p * H + h] = v;
+        store3(Wb3 + (size_t)(2 * p) * H3 + h, H, v.x);
+        store3(Wb3 + (size_t)(2 * p + 1) * H3 + h, H, v.y);
+        store3(Bq3 + (size_t)h * P6 + 2 * p, 2 * (size_t)P, v.x);
+        store3(Bq3 + (size_t)h * P6 + 2 * p + 1, 2 * (size_t)P, v.y);
+        const float2 c = Cc[(size_t)h * P + p];
+        store3(Cq3 + (size_t)(2 * p) * H3 + h, H, c.x);
+        store3(Cq3 + (size_t)(2 * p + 1) * H3 + h, H, -c.y);
+        store3(Cp3 + (size_t)h * P6 + 2 * p, 2 * (size_t)P, c.x);
+        store3(Cp3 + (size_t)h * P6 + 2 * p + 1, 2 * (size_t)P, -c.y);
+    }
+}
+
+void launch_discretize_pack_planes(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
+                                   const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar, void* Wb3, void* Cq3,
+                                   void* Cp3, void* Bq3, cudaStream_t st) {
+    count_launch();
+    discretize_pack_planes_kernel<<<P, 128, 0, st>>>(H, P, Lambda, Delta, Bc, Cc, Abar, Abar_lo, Bbar, (__nv_bfloat16*)Wb3,
+                                                     (__nv_bfloat16*)Cq3, (__nv_bfloat16*)Cp3, (__nv_bfloat16*)Bq3);
+}
+
 void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
                                const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
                                void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st) {

@@ -264,6 +264,21 @@ struct TnParams {
     const char* a_base;   // A as bytes; rows are K * 2 bytes apart and contiguous
     int a_row_bytes;
     float* dot_part;      // epilogue 3: [CTAs, ldo] column sums of skip * dot, one row per CTA
+    // Sum of several products in one accumulator (operands split into bf16 planes laid side by side along K:
+    // plane a of A in columns [a Kp, (a + 1) Kp), likewise W): k-block kb belongs to product kb / kpp, which
+    // takes plane (pa >> 4 j) & 15 of A and plane (pb >> 4 j) & 15 of W.  kpp = 0: one product, planes 0.
+    int kpp;              // k-blocks per product (Kp / BK)
+    uint32_t pa, pb;
+    __device__ __forceinline__ int a_col(int kb) const {
+        if (kpp == 0) return kb * BK;
+        const int j = kb / kpp;
+        return (int)((pa >> (4 * j)) & 15u) * kpp * BK + (kb - j * kpp) * BK;
+    }
+    __device__ __forceinline__ int w_col(int kb) const {
+        if (kpp == 0) return kb * BK;
+        const int j = kb / kpp;
+        return (int)((pb >> (4 * j)) & 15u) * kpp * BK + (kb - j * kpp) * BK;
+    }
 };
 
 // One epilogue warp's share of a finished accumulator tile: rows m0 + 32 (warp % 4) .. + 31, one half
@@ -506,8 +521,8 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
                     mbar_expect_tx(s.full(stage), kStageBytes);
                     const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
-                    tma_load_2d(a_dst, &tmA, s.full(stage), kb * BK, m0);
-                    tma_load_2d(a_dst + kABytes, &tmW, s.full(stage), kb * BK, n0);
+                    tma_load_2d(a_dst, &tmA, s.full(stage), p.a_col(kb), m0);
+                    tma_load_2d(a_dst + kABytes, &tmW, s.full(stage), p.w_col(kb), n0);
                     if (++stage == kTnStages) {
                         stage = 0;
                         phase ^= 1u;
@@ -656,8 +671,8 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                     if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
                     if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kPairStageBytes);
                     const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
-                    tma_load_2d_pair(a_dst, &tmA, leader_full0 + 8u * stage, kb * BK, m0);
-                    tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full0 + 8u * stage, kb * BK, n0);
+                    tma_load_2d_pair(a_dst, &tmA, leader_full0 + 8u * stage, p.a_col(kb), m0);
+                    tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full0 + 8u * stage, p.w_col(kb), n0);
                     if (++stage == kSt) {
                         stage = 0;
                         phase ^= 1u;
@@ -1557,8 +1572,15 @@ struct NtParams {
     int blocks_per_split;  // k-blocks (of BK rows) per slice
     float* part;        // [splits, I, J]
     WsHeader* hdr;
+    // kMulti: n_prod products of bf16 planes in one accumulator; product j takes plane (pa >> 4 j) & 15 of A
+    // (columns [a I, (a + 1) I) of its matrix) and plane (pb >> 4 j) & 15 of Bm (columns [b J, (b + 1) J)).
+    int n_prod;
+    uint32_t pa, pb;
 };
 
+// kMulti = false: the 256 accumulator columns are 128 output columns times the two planes (hi, lo) of Bm, added
+// in the epilogue.  kMulti = true: 256 output columns, every product of the schedule accumulated in place.
+template <bool kMulti>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBhi,
                   const __grid_constant__ CUtensorMap tmBlo, NtParams p) {
@@ -1567,7 +1589,7 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t tmem_base = prologue(s, warp, lane, 128);
     const int tile = blockIdx.x, split = blockIdx.y;
-    constexpr int kOutCols = BN / 2;   // accumulator columns [0,128): hi plane, [128,256): lo plane
+    constexpr int kOutCols = kMulti ? BN : BN / 2;   // (not kMulti) accumulator columns [0,128): hi plane, [128,256): lo plane
     const int i0 = (tile / p.j_tiles) * BM, j0 = (tile % p.j_tiles) * kOutCols;
     const int total_blocks = (p.K + BK - 1) / BK;
     const int kb0 = split * p.blocks_per_split;
@@ -1581,18 +1603,26 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             prefetch_tmap(&tmBlo);
             int stage = 0;
             uint32_t phase = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int kq = 0; kq < (kMulti ? p.n_prod : 1) * nkb; ++kq) {
                 if (!mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag)) break;
                 mbar_expect_tx(s.full(stage), kStageBytes);
                 const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageBytes);
+                const int j = kq / max(nkb, 1), kb = kq - j * nkb;   // product of the schedule, k-block of the slice
                 const int row = (kb0 + kb) * BK;
+                const int ia = kMulti ? (int)((p.pa >> (4 * j)) & 15u) * p.I + i0 : i0;
+                const int jb = kMulti ? (int)((p.pb >> (4 * j)) & 15u) * p.J + j0 : j0;
 #pragma unroll
-                for (int h = 0; h < BM / 64; ++h) tma_load_2d(a_dst + h * (BK * 128), &tmA, s.full(stage), i0 + 64 * h, row);
+                for (int h = 0; h < BM / 64; ++h) tma_load_2d(a_dst + h * (BK * 128), &tmA, s.full(stage), ia + 64 * h, row);
+                if (kMulti) {
 #pragma unroll
-                for (int h = 0; h < kOutCols / 64; ++h) {
-                    tma_load_2d(a_dst + kABytes + h * (BK * 128), &tmBhi, s.full(stage), j0 + 64 * h, row);
-                    tma_load_2d(a_dst + kABytes + (kOutCols / 64 + h) * (BK * 128), &tmBlo, s.full(stage),
-                                j0 + 64 * h, row);
+                    for (int h = 0; h < BN / 64; ++h)
+                        tma_load_2d(a_dst + kABytes + h * (BK * 128), &tmBhi, s.full(stage), jb + 64 * h, row);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < BN / 128; ++h) {
+                        tma_load_2d(a_dst + kABytes + h * (BK * 128), &tmBhi, s.full(stage), j0 + 64 * h, row);
+                        tma_load_2d(a_dst + kABytes + (BN / 128 + h) * (BK * 128), &tmBlo, s.full(stage), j0 + 64 * h, row);
+                    }
                 }
                 if (++stage == kStages) {
                     stage = 0;
@@ -1606,7 +1636,7 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int kb = 0; kb < (kMulti ? p.n_prod : 1) * nkb; ++kb) {
                 if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                 tc_fence_after();
                 const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageBytes);
@@ -1646,10 +1676,12 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    tmem_ld32(t_row + (uint32_t)(kOutCols + c), r);
-                    tmem_ld_wait();
+                    if (!kMulti) {
+                        tmem_ld32(t_row + (uint32_t)(kOutCols + c), r);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r[i]);
+                        for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r[i]);
+                    }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = 0.f;
@@ -1722,6 +1754,8 @@ static bool set_smem(K kernel, size_t bytes) {
 
 }  // namespace tc
 
+int tc_max_n() { return tc::kMaxDiag; }
+
 bool tc_tn_supported(int M, int N_out, int K, bool split_w) {
     const int out_cols = split_w ? tc::BN / 2 : tc::BN;
     return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % out_cols) == 0 && N_out <= tc::kMaxDiag;
@@ -1749,7 +1783,12 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     if (epi == 3 && (!g.dot_part || !g.dot_rows || !tc_tn_dot_supported(g.M, g.N_out, g.K))) return SSM_ERR_SHAPE;
     if (epi == 2 && (!g.split_w || !g.store_f32 || !g.skip || !tc_tn_gate_supported(g.M, g.N_out, g.K))) return SSM_ERR_SHAPE;
     CUtensorMap ma, mw, mo, ms, mg;
-    if (!make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, BK, BM)) return SSM_ERR_CUDA;
+    // with a product schedule the operands are planes_a / planes_w bf16 planes of K columns each, side by side
+    const int n_prod = g.n_products > 0 ? g.n_products : 1;
+    const uint64_t a_cols = (uint64_t)g.K * (g.n_products > 0 ? g.planes_a : 1);
+    const uint64_t w_cols = (uint64_t)g.K * (g.n_products > 0 ? g.planes_w : 1);
+    if (g.n_products > 8) return SSM_ERR_SHAPE;
+    if (!make_map(&ma, g.A, (uint64_t)g.M, a_cols, BK, BM)) return SSM_ERR_CUDA;
     if (g.store_f32) {   // fp32 result, stored by the TMA unit in boxes of 32 rows x 32 columns
         if (!make_map(&mo, g.out, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, true)) return SSM_ERR_CUDA;
     } else {             // bf16 result: 32 x 32 boxes, 64-byte rows
@@ -1763,12 +1802,13 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
         return SSM_ERR_CUDA;
     if (epi == 3 && !make_map(&mg, g.dot, (uint64_t)g.M, (uint64_t)g.N_out, 32, 32, false, CU_TENSOR_MAP_SWIZZLE_64B))
         return SSM_ERR_CUDA;   // (the dot operand travels in the map slot of the gated result)
-    TnParams p{g.M, n_tiles, g.K / BK, g.N_out, g.diag, g.hdr, (const char*)g.A, g.K * 2, g.dot_part};
+    TnParams p{g.M, n_tiles, n_prod * (g.K / BK), g.N_out, g.diag, g.hdr, (const char*)g.A, (int)a_cols * 2, g.dot_part,
+               g.n_products > 0 ? g.K / BK : 0, g.prod_a, g.prod_w};
     const int m_tiles = (g.M + BM - 1) / BM;
     const int pair_tiles = pair_tiles_of(g.M, n_tiles);
     bool ok = true;
     if (pair_tiles >= sm_count() / 2) {   // enough 256-row tiles to give every CTA pair one
-        if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN / 2)) return SSM_ERR_CUDA;
+        if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, w_cols, BK, BN / 2)) return SSM_ERR_CUDA;
         count_launch();
         // The kernel is persistent: its grid is the number of CTA pairs the device can hold at once
         // (not every SM has a partner that a cluster may use).
@@ -1790,7 +1830,7 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
 #undef SSM_LAUNCH_PAIR
         return ok ? SSM_OK : SSM_ERR_CUDA;
     }
-    if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, (uint64_t)g.K, BK, BN)) return SSM_ERR_CUDA;
+    if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, w_cols, BK, BN)) return SSM_ERR_CUDA;
     const int grid = min(sm_count(), m_tiles * n_tiles);
     count_launch();
 #define SSM_LAUNCH_TN(EPI, SPLIT)                                                                          \
@@ -1895,19 +1935,42 @@ int tc_nt_splits(int K, int I, int J) {
 int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
     using namespace tc;
     CUtensorMap ma, mbh, mbl;
+    const int blocks = (g.K + BK - 1) / BK;
+    const int bps = (blocks + g.splits - 1) / g.splits;
+    if (g.n_products > 0) {   // planes side by side: A [K, planes_a * I], Bm [K, planes_b * J]
+        if (g.n_products > 8 || g.J % BN != 0) return SSM_ERR_SHAPE;
+        if (!make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.I * g.planes_a, 64, BK)) return SSM_ERR_CUDA;
+        if (!make_map(&mbh, g.Bm_hi, (uint64_t)g.K, (uint64_t)g.J * g.planes_b, 64, BK)) return SSM_ERR_CUDA;
+        const int j_tiles = g.J / BN;
+        NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr, g.n_products, g.prod_a, g.prod_b};
+        dim3 grid((g.I / BM) * j_tiles, g.splits);
+        count_launch();
+        const bool ok = set_smem(gemm_tc_nt_kernel<true>, kNtSmemBytes);
+        gemm_tc_nt_kernel<true><<<grid, kThreads, kNtSmemBytes, st>>>(ma, mbh, mbh, p);
+        return ok ? SSM_OK : SSM_ERR_CUDA;
+    }
     if (!make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.I, 64, BK, false, CU_TENSOR_MAP_SWIZZLE_128B, (uint64_t)g.lda))
         return SSM_ERR_CUDA;
     if (!make_map(&mbh, g.Bm_hi, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
     if (!make_map(&mbl, g.Bm_lo, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
-    const int blocks = (g.K + BK - 1) / BK;
-    const int bps = (blocks + g.splits - 1) / g.splits;
     const int j_tiles = g.J / (BN / 2);
-    NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr};
+    NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr, 0, 0u, 0u};
     dim3 grid((g.I / BM) * j_tiles, g.splits);
     count_launch();
-    const bool ok = set_smem(gemm_tc_nt_kernel, kNtSmemBytes);
-    gemm_tc_nt_kernel<<<grid, kThreads, kNtSmemBytes, st>>>(ma, mbh, mbl, p);
+    const bool ok = set_smem(gemm_tc_nt_kernel<false>, kNtSmemBytes);
+    gemm_tc_nt_kernel<false><<<grid, kThreads, kNtSmemBytes, st>>>(ma, mbh, mbl, p);
     return ok ? SSM_OK : SSM_ERR_CUDA;
+}
+
+// Split-K factor of the product-schedule variant (tiles of 128 x 256 outputs).
+int tc_nt_multi_splits(int K, int I, int J) {
+    const int tiles = (I / tc::BM) * (J / tc::BN);
+    const int blocks = (K + tc::BK - 1) / tc::BK;
+    int s = tc::sm_count() / (tiles > 0 ? tiles : 1);
+    if (s < 1) s = 1;
+    if (s > blocks) s = blocks;
+    if (s > 64) s = 64;
+    return s;
 }
 
 }  // namespace ssm

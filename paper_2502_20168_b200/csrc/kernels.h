@@ -115,8 +115,14 @@ struct GemmTcTN {
     const void* dot = nullptr;
     float* dot_part = nullptr;
     int* dot_rows = nullptr;
+    // Sum of n_products products in one accumulator (fp32-accurate results from bf16 tensor-core products):
+    // A is planes_a bf16 planes of K columns side by side ([M, planes_a * K]), W likewise ([N_out, planes_w * K]);
+    // product j multiplies plane (prod_a >> 4 j) & 15 of A by plane (prod_w >> 4 j) & 15 of W.  fp32 result only.
+    int n_products = 0, planes_a = 1, planes_w = 1;
+    uint32_t prod_a = 0, prod_w = 0;
 };
 bool tc_tn_supported(int M, int N_out, int K, bool split_w);
+int tc_max_n();   // widest output of the tensor-core projections
 bool tc_tn_dot_supported(int M, int N_out, int K);
 int tc_tn_dot_max_rows();
 bool tc_tn_gate_supported(int M, int N_out, int K);
@@ -171,7 +177,12 @@ struct GemmTcNT {
     float* part;
     WsHeader* hdr;
     int lda = 0;   // elements between rows of A when A is a column block of a wider matrix (0: I)
+    // Product schedule (see GemmTcTN): A = planes_a planes of I columns, Bm_hi = planes_b planes of J columns
+    // (Bm_lo unused), J a multiple of 256; splits from tc_nt_multi_splits.
+    int n_products = 0, planes_a = 1, planes_b = 1;
+    uint32_t prod_a = 0, prod_b = 0;
 };
+int tc_nt_multi_splits(int K, int I, int J);
 bool tc_nt_supported(int I, int J);
 int tc_nt_splits(int K, int I, int J);
 int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
@@ -184,6 +195,17 @@ void launch_pack_operands_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, c
 void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
                                const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
                                void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st);
+
+// planes.cu / discretize.cu: fp32 tensors as three bf16 planes side by side ([M, K] -> [M, 3K]) so that a
+// projection with fp32 inputs runs on the bf16 tensor cores as a sum of plane products (GemmTcTN / GemmTcNT
+// with a product schedule), and what follows such a projection: out = acc + diag * skip (+ add).
+void launch_split_planes(const float* in, size_t M, int K, void* out, cudaStream_t st);
+void launch_diag_skip(const float* acc, const float* diag, const void* skip, bool skip_bf16, const float* add, size_t M,
+                      int N, void* out, bool out_bf16, cudaStream_t st);
+// Discretisation and the four projection operands as planes: Wb3, Cq3 [2P, 3H]; Cp3, Bq3 [H, 3 * 2P].
+void launch_discretize_pack_planes(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc,
+                                   const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar, void* Wb3, void* Cq3,
+                                   void* Cp3, void* Bq3, cudaStream_t st);
 
 // glu.cu: what surrounds the GEMMs of the half-GLU gate out = v * sigmoid(GELU(v) W).
 // Tensor-core path (may be NULL): Wt2 [2H, 2H], the hi/lo stacked operand of z = [x1_hi | x1_lo] W, and

@@ -59,6 +59,15 @@ def test_tensor_core_path_shapes_bf16(B, T, H, P):
     run(w, with_x0=True, with_gxT=True)
 
 
+@pytest.mark.parametrize("B,T,H,P", [(1, 1, 256, 128), (2, 100, 256, 128), (3, 333, 512, 128), (5, 77, 256, 384),
+                                     (300, 66, 256, 128)])
+def test_plane_path_shapes_fp32(B, T, H, P):
+    # fp32 I/O with tile-sized H and P: the projections run on the tensor cores as sums of products of bf16
+    # planes (three planes per fp32 value); B*T is ragged against the 128-row tiles.  fp32 tolerance.
+    w = I.Workload("planes", B=B, T=T, H=H, P=P, io_dtype="f32", p_done=0.02, seed=B + T)
+    run(w, with_x0=True, with_gxT=True)
+
+
 @pytest.mark.parametrize("B,T,H,P", [(81, 128, 256, 128), (150, 256, 256, 64), (76, 384, 512, 128),
                                      (301, 64, 256, 128), (601, 32, 256, 128), (2403, 16, 256, 64)])
 def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
