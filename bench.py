@@ -337,6 +337,64 @@ def replay_ms(buf, torch, stream, reps=20):
     return round(g0.elapsed_time(g1) / reps, 5)
 
 
+def time_paper_block(w, n_blocks, torch, sb, harness, steps=20):
+    """The paper's sequence block (SSM layer, then the half-GLU gate on its output; Appendix "S5 Sequence
+    Layer") n_blocks times in a row, forward + backward, at a workload's sizes: CUDA-event time per step,
+    eager and replayed from a CUDA graph."""
+    shape = sb.make_shape(w.B, w.T, w.H, w.P, w.io_dtype)
+    layers = [harness.LayerBuffers(harness.device_drawn(I.small_variant(w, seed=w.seed + l)), w.io_dtype) for l in range(n_blocks)]
+    g = torch.Generator(device="cuda")
+    g.manual_seed(w.seed)
+    Ws = [(torch.randn((w.H, w.H), device="cuda", generator=g) / w.H ** 0.5).contiguous() for _ in range(n_blocks)]
+    dWs = [torch.empty_like(W) for W in Ws]
+    gws = [sb.alloc_workspace(sb.ssm_glu_workspace_bytes(shape)) for _ in range(n_blocks)]
+    outs = [torch.empty_like(layers[0].y) for _ in range(n_blocks)]
+    gout = layers[0].gy.clone()
+    for l, L in enumerate(layers):
+        L.gy = torch.empty_like(L.y)
+        if l > 0:
+            L.u = outs[l - 1]
+
+    def step(stream):
+        for l, L in enumerate(layers):
+            L.forward(stream)
+            sb.ssm_glu_fwd(shape, Ws[l], L.y, outs[l], gws[l], stream)
+        gr = gout
+        for l in range(n_blocks - 1, -1, -1):
+            L = layers[l]
+            sb.ssm_glu_bwd(shape, Ws[l], L.y, gr, gws[l], L.gy, dWs[l], stream)
+            L.backward(stream)
+            gr = L.du
+
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        step(stream)
+    torch.cuda.synchronize()
+    n0 = sb.ssm_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step(stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    launches = (sb.ssm_launch_count() - n0) / steps
+
+    class _Both:      # forward + backward of the chain, in the shape replay_ms wants
+        def forward(self, s):
+            step(s)
+
+        def backward(self, s):
+            pass
+
+    out = {"blocks": n_blocks, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
+           "ms_per_step": round(ms, 5), "timesteps_per_sec": w.timesteps / (ms * 1e-3), "launches_per_step": launches,
+           "graph_ms_per_step": replay_ms(_Both(), torch, stream)}
+    for L in layers:
+        sb.ssm_check(L.ws)
+    return out
+
+
 def scan_stage_summary(r, peaks):
     """The two scan stages of a timed layer step (fused with their projections, or apart) as
     algorithmic GB/s and as fractions of the measured copy rate and of the nominal 8 TB/s."""
@@ -619,6 +677,9 @@ def main():
             torch.cuda.empty_cache()
             line["configs"] = {c.name: time_workload(c, torch, sb, harness, steps=20, graph=True)
                                for c in (I.C0, I.C1, I.C2, I.C3, I.PAPER_STATE, I.PAPER_VISION)}
+            # the paper's own blocks (layer + half-GLU gate): one at the state task's sizes, two at the vision task's
+            line["paper_block"] = {"state": time_paper_block(I.PAPER_STATE, 1, torch, sb, harness),
+                                   "vision": time_paper_block(I.PAPER_VISION, 2, torch, sb, harness)}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, I.draw_layer(I.small_variant(w, B=min(w.B, max(1, 262144 // w.T)))))
         print(json.dumps(line))
