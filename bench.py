@@ -489,15 +489,15 @@ def main():
     stream = torch.cuda.current_stream()
 
     exchange = args.allreduce_grads and world > 1 and not stacked
-    pending = []
+    xchg = harness.GradExchange(buf) if exchange else None
 
     def step():
         buf.forward(stream)
-        if pending:                      # last step's gradient sum has to be out of the bucket before it is rewritten
-            pending.pop().wait()
+        if xchg:                         # last step's gradient sum has to be out of the bucket before it is rewritten
+            xchg.finish()
         buf.backward(stream)
-        if exchange:
-            pending.append(harness.allreduce_param_grads(buf, async_op=True))
+        if xchg:
+            xchg.start()
 
     def barrier():
         if world > 1:
@@ -518,8 +518,8 @@ def main():
     ev0.record(stream)
     for _ in range(args.steps):
         step()
-    while pending:                       # the last step's exchange belongs to the timed region
-        pending.pop().wait()
+    if xchg:                             # the last step's exchange belongs to the timed region
+        xchg.finish()
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)

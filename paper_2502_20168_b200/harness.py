@@ -56,6 +56,32 @@ def allreduce_param_grads(buf, group=None, async_op=False):
     return dist.all_reduce(buf.grad_bucket, op=dist.ReduceOp.SUM, group=group, async_op=async_op)
 
 
+class GradExchange:
+    """Order of the gradient exchange in a batch-sharded training loop.  The layer's backward pass finishes all
+    five parameter gradients in its last two kernels (the split-K sums and the adjoint of the discretisation),
+    so there is no tail of the backward pass left to hide the exchange under: it is started right after the
+    backward call and runs under the next step's forward pass; before the next backward call rewrites the bucket
+    the exchange has to be done.  `start()` issues the one all-reduce of the bucket asynchronously; `finish()`
+    waits for it (a no-op when none is pending) and must be called before the next backward; a second `start()`
+    without `finish()` in between is an error, since the bucket would have been rewritten under the collective."""
+
+    def __init__(self, buf, group=None):
+        self.buf, self.group, self.pending = buf, group, None
+        self.started = self.finished = 0
+
+    def start(self):
+        if self.pending is not None:
+            raise RuntimeError("gradient bucket rewritten while its all-reduce was in flight: call finish() first")
+        self.pending = allreduce_param_grads(self.buf, group=self.group, async_op=True)
+        self.started += 1
+
+    def finish(self):
+        if self.pending is not None:
+            self.pending.wait()
+            self.pending = None
+            self.finished += 1
+
+
 class LayerBuffers:
     """Device copies of one layer's inputs plus preallocated outputs and workspace."""
 

@@ -64,6 +64,51 @@ def _bucket_rank_main(rank, world, port, out):
     dist.destroy_process_group()
 
 
+def _exchange_order_rank_main(rank, world, port, out):
+    """Three steps of a training loop's gradient exchange: backward writes the bucket, start(), the next forward
+    runs, finish() before the next backward."""
+    import types
+    from paper_2502_20168_b200 import harness
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    bucket, _ = harness.grad_bucket(W.P, W.H, "cpu")
+    x = harness.GradExchange(types.SimpleNamespace(grad_bucket=bucket))
+    sums, refused = [], False
+    for step in range(3):
+        x.finish()                                   # before the backward pass rewrites the bucket
+        bucket.fill_(float(10 * step + rank + 1))    # "backward": this rank's gradients of this step
+        x.start()
+        if step == 1:
+            try:
+                x.start()                            # a rewrite + restart without finish() must be refused
+            except RuntimeError:
+                refused = True
+        # (the next step's forward pass would run here, under the exchange)
+        x.finish()
+        sums.append(float(bucket[0]))
+        assert torch.all(bucket == bucket[0])
+    out.put((rank, sums, refused, x.started, x.finished))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_gradient_exchange_is_finished_before_the_bucket_is_rewritten():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_exchange_order_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = [q.get(timeout=120) for _ in procs]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, sums, refused, started, finished in got:
+        assert sums == [3.0, 23.0, 43.0]             # (10 s + 1) + (10 s + 2) per step s, never a mix of two steps
+        assert refused and started == finished == 3
+
+
 def test_parameter_gradients_summed_over_two_ranks_by_one_bucket_allreduce():
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
