@@ -1166,13 +1166,16 @@ struct FbParams {
     int B, T, P;
     int n_tiles;      // 2P / 128
     int k_blocks;     // H / 64
-    int tblocks;      // T / 128
-    int nchains;      // n_tiles * ceil(B / 2)
+    int tblocks;      // tiles per chain: T / 128, or 1
+    int unit_rows;    // rows of a chain: T, or 128 when T < 128 (a tile then holds 128 / T whole sequences)
+    int n_units;      // chains per 64 states: B, or ceil(B * T / 128)
+    int gps;          // row groups per sequence inside a tile: 8, or T / 16
+    int nchains;      // n_tiles * ceil(n_units / 2)
     const float2* Abar;
     const uint8_t* done;
     const float2* x0;     // [B, P] or NULL
     const float2* gxT;    // [B, P] or NULL
-    float2* gA_part;      // [B, P]
+    float2* gA_part;      // [n_units, P]: one row of sums per chain
     float2* gx0;          // [B, P] or NULL
     WsHeader* hdr;
 };
@@ -1214,7 +1217,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     auto seq_of = [&](int chain) { return 2 * (chain / p.n_tiles) + (int)rank; };
     auto row_of = [&](int chain, int tb) {
         const int b = seq_of(chain);
-        return b < p.B ? b * p.T + tb * BM : M;   // no sequence (odd B): rows past the end read as zero
+        return b < p.n_units ? b * p.unit_rows + tb * BM : M;   // nothing for this CTA: rows past the end read as zero
     };
 
     if (warp == 0) {
@@ -1283,7 +1286,10 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
         const int sp = te & 31, sl = te >> 5;       // scan role: pair of states of the tile, group of its rows
         const int prow = q * 32 + lane;             // drain role: row of the tile
-        const bool from_carry = sl == nsl - 1;      // the last rows come first
+        const bool short_seq = p.T < BM;            // then a chain is one tile of 128 / T whole sequences
+        const int g0 = sl - sl % p.gps;             // first and last row group of this group's sequence in the tile
+        const int gl = g0 + p.gps - 1;
+        const bool from_carry = sl == gl;           // the last rows come first
         float4* T4 = reinterpret_cast<float4*>(s.staging);
         uint8_t* warp_buf = s.staging + sl * (2 * R * 256);   // this warp's rows of the tile; later x_{t-1}, then s
         uint2* xs = reinterpret_cast<uint2*>(warp_buf) + sp;
@@ -1295,7 +1301,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         bool ok = true;
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
-            const bool has_seq = b < p.B;
+            const bool has_seq = b < p.n_units;
             const int pg = n_tile * 64 + 2 * sp;    // the first of this thread's two states
             const float2 a0 = cconj(p.Abar[pg]), a1 = cconj(p.Abar[pg + 1]);
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
@@ -1315,7 +1321,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             C2 g = zero;        // this thread's part of the chain's sums s_t conj(x_{t-1})
             f32x2 gim_neg = 0ull;   // the part of Im g that enters with a minus sign, summed apart
             C2 xinit = zero;    // x0: what stands before the sequence's first row
-            if (sl == 0 && p.x0 && has_seq) {
+            if (!short_seq && sl == 0 && p.x0 && has_seq) {
                 const float2 c0 = p.x0[(size_t)b * p.P + pg], c1 = p.x0[(size_t)b * p.P + pg + 1];
                 xinit.re = pack2(c0.x, c1.x);
                 xinit.im = pack2(c0.y, c1.y);
@@ -1324,8 +1330,10 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             for (int tb = p.tblocks - 1; tb >= 0; --tb) {
                 const int m0 = row_of(chain, tb);
                 if (p.done && te < BM) {
-                    const bool f0 = has_seq && p.done[(size_t)m0 + te] != 0;
-                    const bool f1 = has_seq && tb * BM + te + 1 < p.T && p.done[(size_t)m0 + te + 1] != 0;
+                    // a row's own flag, and the flag of the row after it if that row belongs to the same sequence
+                    const bool next_in_seq = short_seq ? ((te + 1) % p.T != 0 && m0 + te + 1 < M) : (tb * BM + te + 1 < p.T);
+                    const bool f0 = has_seq && m0 + te < M && p.done[(size_t)m0 + te] != 0;
+                    const bool f1 = has_seq && next_in_seq && p.done[(size_t)m0 + te + 1] != 0;
                     const uint32_t mk0 = __ballot_sync(0xffffffffu, f0), mk1 = __ballot_sync(0xffffffffu, f1);
                     if (lane == 0) {
                         masks[te >> 5] = mk1;
@@ -1373,6 +1381,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 epi_sync();
                 // (2) this thread's two states over its R rows, last row first
                 const int r0 = sl * R;
+                const bool grp_valid = has_seq && m0 + r0 < M;           // (short sequences: the last tile may be ragged)
+                const int b_grp = short_seq ? (m0 + r0) / p.T : b;      // this group's sequence
                 uint32_t gflags = 0;   // bit g: a reset acts inside or right after row group g
                 uint32_t mask = 0u, mask0 = 0u;
                 if (p.done) {
@@ -1394,8 +1404,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     v[i].re = pack2(t.x, t.y);
                     v[i].im = pack2(t.z, t.w);
                 }
-                if (from_carry && tb == p.tblocks - 1 && p.gxT && has_seq) {   // the gradient of the final state
-                    const float2 c0 = p.gxT[(size_t)b * p.P + pg], c1 = p.gxT[(size_t)b * p.P + pg + 1];
+                if (from_carry && tb == p.tblocks - 1 && p.gxT && grp_valid) {   // the gradient of the final state
+                    const float2 c0 = p.gxT[(size_t)b_grp * p.P + pg], c1 = p.gxT[(size_t)b_grp * p.P + pg + 1];
                     float v0, v1, v2, v3;
                     unpack2(v[R - 1].re, v0, v1);
                     unpack2(v[R - 1].im, v2, v3);
@@ -1412,8 +1422,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (tb > 0) tma_prefetch_3d(&tmX, n_tile * 64, m0 - BM + r0 - 1, 0);
                 }
                 C2 e = zero;
-                if (from_carry) {   // from the carried value: these results are final
-                    const float4 c = carry_s[sp];
+                if (from_carry) {   // from the carried value (nothing, for a sequence inside the tile): these results are final
+                    const float4 c = short_seq ? make_float4(0.f, 0.f, 0.f, 0.f) : carry_s[sp];
                     C2 x = {pack2(c.x, c.y), pack2(c.z, c.w)};
                     if (mask == 0u) {
 #pragma unroll
@@ -1446,13 +1456,13 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 C2 x = e;
                 if (!from_carry) {   // s of the row after this group's last
                     {
-                        const float4 c = agg_e[(nsl - 1) * 32 + sp];
+                        const float4 c = agg_e[gl * 32 + sp];
                         x.re = pack2(c.x, c.y);
                         x.im = pack2(c.z, c.w);
                     }
 #pragma unroll
                     for (int gq = nsl - 2; gq >= 1; --gq) {
-                        if (gq > sl) {
+                        if (gq > sl && gq < gl) {
                             const float4 c = agg_e[gq * 32 + sp];
                             const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
                             x = ((gflags >> gq) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
@@ -1464,7 +1474,15 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     // (the wait gave up: the flag is set, everybody leaves at the next barrier)
                 }
                 xphase ^= 1u;
-                const bool seq_start = tb == 0 && sl == 0;   // row 0 of this group is the sequence's first row
+                const bool seq_start = tb == 0 && sl == g0;   // row 0 of this group is the sequence's first row
+                if (short_seq && seq_start) {                // the state before that row: this sequence's x0
+                    xinit = zero;
+                    if (p.x0 && grp_valid) {
+                        const float2 c0 = p.x0[(size_t)b_grp * p.P + pg], c1 = p.x0[(size_t)b_grp * p.P + pg + 1];
+                        xinit.re = pack2(c0.x, c1.x);
+                        xinit.im = pack2(c0.y, c1.y);
+                    }
+                }
                 // A tile without flags (the common case) takes the loop without the per-row tests.
                 auto fold_rows = [&](auto with_flags) {
                     constexpr bool kFlags = decltype(with_flags)::value;
@@ -1512,21 +1530,21 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     fold_rows(std::true_type{});
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0 && has_seq) {
+                if (lane == 0 && grp_valid) {
                     tma_store_3d_nocommit(&tmS, smem_u32(warp_buf), n_tile * 64, m0 + r0, 0);
                     tma_commit_group();
                 }
-                if (sl == 0) {   // x is s of the tile's first row
+                if (sl == g0) {   // x is s of the first row of the tile (of the sequence, when it lies inside the tile)
                     float x0r, x1r, x0i, x1i;
                     unpack2(x.re, x0r, x1r);
                     unpack2(x.im, x0i, x1i);
                     if (tb > 0) {
                         carry_s[sp] = make_float4(x0r, x1r, x0i, x1i);
-                    } else if (p.gx0 && has_seq) {   // what reaches the initial state: keep_0 conj(Abar) s_0
+                    } else if (p.gx0 && grp_valid) {   // what reaches the initial state: keep_0 conj(Abar) s_0
                         const bool cut = (mask0 & 1u) != 0u;
                         const float2 z = make_float2(0.f, 0.f);
-                        p.gx0[(size_t)b * p.P + pg] = cut ? z : cfma(a0, make_float2(x0r, x0i), z);
-                        p.gx0[(size_t)b * p.P + pg + 1] = cut ? z : cfma(a1, make_float2(x1r, x1i), z);
+                        p.gx0[(size_t)b_grp * p.P + pg] = cut ? z : cfma(a0, make_float2(x0r, x0i), z);
+                        p.gx0[(size_t)b_grp * p.P + pg + 1] = cut ? z : cfma(a1, make_float2(x1r, x1i), z);
                     }
                 }
             }
@@ -1897,9 +1915,13 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
 }
 
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) {
-    if (T % tc::BM != 0 || H % tc::BK != 0 || P % 64 != 0) return false;
-    return (2 * P / 128) * ((B + 1) / 2) >= fused_min_pairs();
+    const bool t_ok = T % tc::BM == 0 || T == 16 || T == 32 || T == 64;
+    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return false;
+    return (2 * P / 128) * ((fs_units(B, T) + 1) / 2) >= fused_min_pairs();
 }
+
+// Rows of gA_part that launch_gemm_scan_bwd writes: one per chain of 64 states.
+int tc_gemm_scan_bwd_part_rows(int B, int T) { return fs_units(B, T); }
 
 int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {
     using namespace tc;
@@ -1909,7 +1931,9 @@ int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {
     if (!make_map(&ma, g.gy, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
     if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
     if (!make_plane_map(&mx, g.x_planes, M, g.P) || !make_plane_map(&ms, g.s_planes, M, g.P)) return SSM_ERR_CUDA;
-    FbParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T / BM, (P2 / 128) * ((g.B + 1) / 2),
+    const int units = fs_units(g.B, g.T);
+    FbParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
+               g.T >= BM ? BM / kFsRows : g.T / kFsRows, (P2 / 128) * ((units + 1) / 2),
                g.Abar, g.done, g.x0, g.gxT, g.gA_part, g.gx0, g.hdr};
     count_launch();
     auto kern = gemm_scan_bwd_kernel;

@@ -147,7 +147,8 @@ int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st);
 
 // g_x projection and reverse scan fused (gemm_tc.cu): s = reverse scan(gy conj(C)) written as the two
 // bf16 planes of s, the sums s_t conj(x_{t-1}) per (sequence, state) in gA_part; g_x never reaches
-// memory.  T must be a multiple of 128, with enough chains (tc_gemm_scan_bwd_supported).
+// memory.  T must be a multiple of 128, or 16, 32 or 64 (a 128-row tile then holds whole sequences), with
+// enough chains (tc_gemm_scan_bwd_supported).
 struct GemmScanBwd {
     const void* gy;         // bf16 [B*T, H]
     const void* Wsplit;     // hi/lo stacked conj(C) operand [4P, H], rows in the pair_cols order
@@ -158,11 +159,12 @@ struct GemmScanBwd {
     const float2* gxT;      // [B, P] or NULL
     const void* x_planes;   // bf16 hi plane [B*T, 2P], then the lo plane
     void* s_planes;         // out: the same layout
-    float2* gA_part;        // out [B, P]
+    float2* gA_part;        // out [tc_gemm_scan_bwd_part_rows(B, T), P]
     float2* gx0;            // out [B, P] or NULL
     WsHeader* hdr;
 };
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P);
+int tc_gemm_scan_bwd_part_rows(int B, int T);   // rows of gA_part the kernel writes (one per chain of 64 states)
 int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st);
 // scan.cu: the same with gA_part placed in `scratch` (as for launch_scan_bwd) and brought down to
 // *gA_rows <= kMaxPartialRows rows at *gA_part_out; the caller sums those.

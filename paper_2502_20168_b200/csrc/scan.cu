@@ -371,7 +371,8 @@ int launch_gemm_scan_bwd_part(GemmScanBwd g, void* scratch, const float2** gA_pa
     float* tmp = reinterpret_cast<float*>(base + s.off_tmp);
     g.gA_part = reinterpret_cast<float2*>(part);
     if (int rc = launch_gemm_scan_bwd(g, st)) return rc;
-    *gA_part_out = reinterpret_cast<const float2*>(launch_reduce_rows(part, g.B, 2 * g.P, tmp, kMaxPartialRows, gA_rows, st));
+    *gA_part_out = reinterpret_cast<const float2*>(
+        launch_reduce_rows(part, tc_gemm_scan_bwd_part_rows(g.B, g.T), 2 * g.P, tmp, kMaxPartialRows, gA_rows, st));
     return SSM_OK;
 }
 
