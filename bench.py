@@ -455,6 +455,11 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="run the workload with this many sequences instead of its own B (cut-down cases for profiler "
+                         "captures; the line says so and is not a headline number)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="stop after the device-resident timed steps and print their stage times only (profiler captures)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the extra measurements reported beside the headline (sweep, scans alone, other configs)")
     ap.add_argument("--allreduce-grads", action="store_true",
@@ -482,6 +487,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     w = I.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = I.small_variant(w, B=args.batch)
     wr = I.small_variant(w, seed=w.seed + 1000 * rank)
     d = I.draw_layer(wr)
     stacked = w.n_layers > 1
@@ -527,6 +534,14 @@ def main():
     launches = sb.ssm_launch_count() - launches0
     clocks = sampler.stop() if sampler else None
     sb.ssm_check(buf.ws)
+    if args.kernels_only:
+        if rank == 0:
+            print(json.dumps({"kernels_only": True, "workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P,
+                              "steps": args.steps, "ms_per_step": ms / args.steps, "gpu_launches": int(launches),
+                              "stage_ms_per_step": {k: round(v[1] / args.steps, 4) for k, v in stages.items()}}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end to end: pinned host inputs in, results out, every step ----
     in_names = ("u", "gout") if stacked else ("u", "gy")
@@ -641,7 +656,7 @@ def main():
             "dtype": "bf16-io/bf16-hi+lo-mma/f32-acc+state" if w.io_dtype == "bf16" and not stacked else "f32",
             "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "T": w.T, "H": w.H, "P": w.P, "io_dtype": w.io_dtype,
-                       "p_done": w.p_done, "n_layers": w.n_layers, "l2": "inputs larger than L2 (no flush)"
+                       "p_done": w.p_done, "n_layers": w.n_layers, "batch_override": args.batch > 0, "l2": "inputs larger than L2 (no flush)"
                        if w.timesteps * w.H * s_io > 126e6 else "inputs fit in L2", "parallelism": f"batch-sharded x{world}" + (" + gradient all-reduce" if exchange else "")},
             "e2e": {"value": total_ts * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "mode": e2e_mode},
