@@ -50,21 +50,22 @@ STAGE_MODEL = {
 }
 
 
-# DRAM bytes per launch seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum, summaries under
-# profiles/) on c4_sweep_T1024_bf16, per timestep (B*T = 262144 rows).  They hold for H = 512,
-# P = 256, bf16 I/O at T = 1024 (the scans choose other tile shapes at other T); an entry is None
-# once its kernel has changed since the counters were taken.
+# DRAM bytes per timestep seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum, or dram__bytes.sum.per_second x
+# duration; summaries under profiles/), captured on c4_sweep_T1024_bf16 cut down to B = 128 (131072 rows) and divided
+# by those rows: every kernel's traffic is proportional to the rows it processes, so a launch of the full workload
+# moves this figure times its timesteps.  They hold for H = 512, P = 256, bf16 I/O, T = 1024; an entry is None where
+# no capture of the kernel as it stands exists.
 NCU_TRAFFIC_PER_TIMESTEP = {
-    "gemm_Bu_scan_fwd": 777.8e6 / 262144,
-    "gemm_gx_scan_bwd": 1327.6e6 / 262144,
-    "scan_fwd": 1021.7e6 / 262144,
-    "scan_bwd": 1579.9e6 / 262144,
-    "gemm_Bu": 763.6e6 / 262144,
-    "gemm_gx": 763.6e6 / 262144,
-    "gemm_y": None,      # (proxy fences added to the bf16 epilogue since the capture: 793.0 MB before)
-    "gemm_du": None,
-    "gemm_gBbar": 813.4e6 / 262144,
-    "gemm_gC": 813.4e6 / 262144,
+    "gemm_Bu_scan_fwd": 359.1e6 / 131072,
+    "gemm_gx_scan_bwd": 646.8e6 / 131072,
+    "gemm_y": 375.5e6 / 131072,
+    "gemm_du": 538.5e6 / 131072,
+    "gemm_gBbar": 406.5e6 / 131072,
+    "gemm_gC": 406.7e6 / 131072,
+    "scan_fwd": None,
+    "scan_bwd": None,
+    "gemm_Bu": None,
+    "gemm_gx": None,
 }
 
 
@@ -458,6 +459,9 @@ def main():
     ap.add_argument("--batch", type=int, default=0,
                     help="run the workload with this many sequences instead of its own B (cut-down cases for profiler "
                          "captures; the line says so and is not a headline number)")
+    ap.add_argument("--scans-alone", type=int, default=0, metavar="T",
+                    help="time only ssm_scan_fwd / ssm_scan_bwd at sequence length T (B*T = 262144 rows, or --batch "
+                         "sequences) and print that (profiler captures of the stand-alone scan kernels)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="stop after the device-resident timed steps and print their stage times only (profiler captures)")
     ap.add_argument("--no-extras", action="store_true",
@@ -486,6 +490,12 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
+    if args.scans_alone > 0:
+        peaks, _ = load_peaks()
+        T = args.scans_alone
+        rows = args.batch * T if args.batch > 0 else 262144
+        print(json.dumps({"scans_alone": time_scans_alone(T, torch, sb, peaks, rows=rows, steps=max(1, args.steps))}))
+        return
     w = I.WORKLOADS[args.workload]
     if args.batch > 0:
         w = I.small_variant(w, B=args.batch)
