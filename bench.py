@@ -83,11 +83,13 @@ class ClockSampler:
     while the timed region runs; falls back to one nvidia-smi query loop if NVML is missing."""
 
     REASONS = (("hw_slowdown", 0x8), ("sw_thermal_slowdown", 0x20), ("hw_thermal_slowdown", 0x40),
-               ("sw_power_cap", 0x4))
+               ("sw_power_cap", 0x4), ("applications_clocks_setting", 0x2), ("sync_boost", 0x10),
+               ("hw_power_brake_slowdown", 0x80), ("display_clock_setting", 0x100))
 
     def __init__(self, gpu_uuid: str, period_s: float = 0.002):
         import threading
         self.sm, self.bits, self.mx, self.err = [], 0, None, None
+        self.power_w = []
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -107,6 +109,7 @@ class ClockSampler:
                     try:
                         self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
                         self.bits |= int(reasons(h))
+                        self.power_w.append(pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0)
                     except Exception as e:      # keep what was sampled
                         self.err = repr(e)
                         return
@@ -123,8 +126,9 @@ class ClockSampler:
             self._thread.join(timeout=5)
         if not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": self.mx, "reasons": ["no samples: " + str(self.err)]}
-        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.mx,
-                "reasons": [n for n, bit in self.REASONS if self.bits & bit], "samples": len(self.sm)}
+        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.mx, "sm_mhz_min": min(self.sm),
+                "reasons": [n for n, bit in self.REASONS if self.bits & bit], "reasons_mask": hex(self.bits),
+                "power_w_max": max(self.power_w) if self.power_w else None, "samples": len(self.sm)}
 
 
 def oracle_sample_run(d, n_seq):
@@ -451,7 +455,7 @@ def time_scans_alone(T, torch, sb, peaks, P=256, rows=262144, steps=10):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
