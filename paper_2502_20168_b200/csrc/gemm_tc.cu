@@ -333,7 +333,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
             }
             fence_async_smem();
             __syncwarp();
-            if (lane == 0 && row0 < p.M) tma_store_2d(tmOut, smem_u32(stg), n_out0 + c, row0);
+            if (lane == 0 && row0 < p.M && n_out0 + c < p.ldo) tma_store_2d(tmOut, smem_u32(stg), n_out0 + c, row0);
         }
         return true;
     }
@@ -402,7 +402,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
             }
             fence_async_smem();
             __syncwarp();
-            if (lane == 0 && row0 < p.M) {
+            if (lane == 0 && row0 < p.M && n_out0 + c < p.ldo) {
                 tma_store_2d(tmOut, smem_u32(stg), n_out0 + c, row0);
                 tma_store_2d(tmGate, smem_u32(ob), n_out0 + c, row0);
             }
@@ -467,7 +467,7 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(ob + lane * 64 + ((j ^ swz) << 4)) = o[j];
         fence_async_smem();
         __syncwarp();
-        if (lane == 0 && row0 < p.M) tma_store_2d(tmOut, smem_u32(ob), n_out0 + c, row0);
+        if (lane == 0 && row0 < p.M && n_out0 + c < p.ldo) tma_store_2d(tmOut, smem_u32(ob), n_out0 + c, row0);
         if (kDot) {
             // Column sums over the warp's 32 rows: at every halving step a lane keeps the half of its values
             // that its lane bit selects and adds the other lane's; lane l ends with the sum of column l.
@@ -501,8 +501,8 @@ gemm_tc_tn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, kTnStages, tn_staging_bytes(kEpi), tn_diag_bytes(kEpi), kStageBytes, tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (kEpi == 1)
-        for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
+    if (kEpi == 1)   // (zero where the last tile reaches past the output's columns)
+        for (int i = threadIdx.x; i < p.n_tiles * BN; i += kTnThreads) s.diag[i] = i < p.ldo ? p.diag[i] : 0.f;
     const uint32_t tmem_base = prologue(s, warp, lane, 32 * kTnEpiWarps);
     const int m_tiles = (p.M + BM - 1) / BM;
     const int total = m_tiles * p.n_tiles;
@@ -614,8 +614,8 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                               tn_skip_bytes(kEpi));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
-    if (kEpi == 1 || kEpi == 3)
-        for (int i = threadIdx.x; i < p.ldo; i += kTnThreads) s.diag[i] = p.diag[i];
+    if (kEpi == 1 || kEpi == 3)   // (zero where the last tile reaches past the output's columns)
+        for (int i = threadIdx.x; i < p.n_tiles * BN; i += kTnThreads) s.diag[i] = i < p.ldo ? p.diag[i] : 0.f;
     if (kEpi == 3)   // the epilogue warps' column sums start at zero
         for (int i = threadIdx.x; i < kTnEpiWarps * (kDotMaxN / 2); i += kTnThreads) s.diag[kDotMaxN + i] = 0.f;
     // barriers and tensor memory (both CTAs), then the whole pair meets
@@ -1776,7 +1776,10 @@ int tc_max_n() { return tc::kMaxDiag; }
 
 bool tc_tn_supported(int M, int N_out, int K, bool split_w) {
     const int out_cols = split_w ? tc::BN / 2 : tc::BN;
-    return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % out_cols) == 0 && N_out <= tc::kMaxDiag;
+    // Outputs are a multiple of 128 columns wide; a last tile of the 256-column kind may be half empty (its
+    // weight rows past N_out read as zero and its results past N_out are clipped by the TMA stores).
+    (void)out_cols;
+    return M >= 1 && K >= tc::BK && (K % tc::BK) == 0 && (N_out % (tc::BN / 2)) == 0 && N_out <= tc::kMaxDiag;
 }
 
 static int pair_tiles_of(int M, int n_tiles) { return ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * n_tiles; }
@@ -1784,7 +1787,7 @@ static int pair_tiles_of(int M, int n_tiles) { return ((M + 2 * tc::BM - 1) / (2
 // The bf16 epilogue can also sum skip * dot over the rows (one partial row per CTA) where the pair kernel
 // runs and the output is at most kDotMaxN wide.
 bool tc_tn_dot_supported(int M, int N_out, int K) {
-    return tc_tn_supported(M, N_out, K, false) && N_out <= tc::kDotMaxN && pair_tiles_of(M, N_out / tc::BN) >= tc::sm_count() / 2;
+    return tc_tn_supported(M, N_out, K, false) && N_out <= tc::kDotMaxN && pair_tiles_of(M, (N_out + tc::BN - 1) / tc::BN) >= tc::sm_count() / 2;
 }
 int tc_tn_dot_max_rows() { return 2 * tc::sm_count(); }
 
@@ -1795,7 +1798,7 @@ bool tc_tn_gate_supported(int M, int N_out, int K) {
 int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     using namespace tc;
     const int out_cols = g.split_w ? BN / 2 : BN;
-    const int n_tiles = g.N_out / out_cols;
+    const int n_tiles = (g.N_out + out_cols - 1) / out_cols;
     const int epi = g.gate_out ? 2 : (g.store_f32 ? 0 : (g.dot ? 3 : 1));
     if ((epi == 1 || epi == 3) && (g.split_w || !g.diag || !g.skip)) return SSM_ERR_SHAPE;
     if (epi == 3 && (!g.dot_part || !g.dot_rows || !tc_tn_dot_supported(g.M, g.N_out, g.K))) return SSM_ERR_SHAPE;
@@ -1824,9 +1827,11 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
                g.n_products > 0 ? g.K / BK : 0, g.prod_a, g.prod_w};
     const int m_tiles = (g.M + BM - 1) / BM;
     const int pair_tiles = pair_tiles_of(g.M, n_tiles);
+    // rows of the packed weight matrix that exist (tiles may reach past them: those rows read as zero)
+    const uint64_t w_rows = g.split_w ? (uint64_t)2 * g.N_out : (uint64_t)g.N_out;
     bool ok = true;
     if (pair_tiles >= sm_count() / 2) {   // enough 256-row tiles to give every CTA pair one
-        if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, w_cols, BK, BN / 2)) return SSM_ERR_CUDA;
+        if (!make_map(&mw, g.W, w_rows, w_cols, BK, BN / 2)) return SSM_ERR_CUDA;
         count_launch();
         // The kernel is persistent: its grid is the number of CTA pairs the device can hold at once
         // (not every SM has a partner that a cluster may use).
@@ -1848,7 +1853,7 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
 #undef SSM_LAUNCH_PAIR
         return ok ? SSM_OK : SSM_ERR_CUDA;
     }
-    if (!make_map(&mw, g.W, (uint64_t)n_tiles * BN, w_cols, BK, BN)) return SSM_ERR_CUDA;
+    if (!make_map(&mw, g.W, w_rows, w_cols, BK, BN)) return SSM_ERR_CUDA;
     const int grid = min(sm_count(), m_tiles * n_tiles);
     count_launch();
 #define SSM_LAUNCH_TN(EPI, SPLIT)                                                                          \
