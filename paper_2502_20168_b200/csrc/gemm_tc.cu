@@ -1716,6 +1716,143 @@ gemm_tc_nt_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 }
 
 // ---------------------------------------------------------------------------------------------
+// NT kernel on CTA pairs
+// ---------------------------------------------------------------------------------------------
+// The same product on clusters of two CTAs: one MMA spans a 256 x 256 accumulator tile, CTA r holding
+// output rows i0 + 128 r .. (its 128 columns of A) and one plane of Bm (r = 0: the high halves, r = 1: the low
+// halves; the MMA takes half of its B columns from each CTA).  Every CTA then brings in 32 KB per k-block
+// instead of 48 KB for the same tensor-core cycles, which is what bounds the single-CTA kernel (96 KB through
+// shared memory per 512 tensor-core cycles).  Barriers as in the TN pair kernel: the leader's `full` barriers
+// count both CTAs' bytes, its commits arrive in both CTAs.  One tile and one slice of the rows per pair.
+constexpr int kNtPairStages = 6;
+constexpr int kNtPairStageBytes = kABytes + kBBytes / 2;   // 32 KB
+constexpr size_t kNtPairSmemBytes = (size_t)kNtPairStages * kNtPairStageBytes + 1024 + 256;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc_nt_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBhi,
+                       const __grid_constant__ CUtensorMap tmBlo, NtParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, kNtPairStages, 0, 0, kNtPairStageBytes, 0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    // barriers of the ring: more stages than the common layout has slots for, so they take the skip slots
+    auto rfull = [&](int i) { return s.skip_full(i); };
+    auto rempty = [&](int i) { return s.skip_full(kNtPairStages + i); };
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kNtPairStages; ++i) {
+            mbar_init(rfull(i), 1);
+            mbar_init(rempty(i), 1);
+        }
+        mbar_init(s.tmem_full(0), 1);
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == 1) tmem_alloc_pair(s.tmem_slot, BN);
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *s.tmem_slot_ptr;
+
+    const int tile = blockIdx.x >> 1, split = blockIdx.y;
+    constexpr int kOutCols = BN / 2;
+    const int i0 = (tile / p.j_tiles) * (2 * BM) + (int)rank * BM, j0 = (tile % p.j_tiles) * kOutCols;
+    const int total_blocks = (p.K + BK - 1) / BK;
+    const int kb0 = split * p.blocks_per_split;
+    const int nkb = max(0, min(total_blocks, kb0 + p.blocks_per_split) - kb0);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(rank == 0 ? &tmBhi : &tmBlo);
+            const CUtensorMap* tmB = rank == 0 ? &tmBhi : &tmBlo;
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!mbar_wait(rempty(stage), phase ^ 1u, s.abort_flag)) break;
+                const uint32_t leader_full = map_to_cta(rfull(stage), 0);
+                if (rank == 0) mbar_expect_tx(rfull(stage), 2 * kNtPairStageBytes);
+                const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kNtPairStageBytes);
+                const int row = (kb0 + kb) * BK;
+#pragma unroll
+                for (int h = 0; h < BM / 64; ++h) tma_load_2d_pair(a_dst + h * (BK * 128), &tmA, leader_full, i0 + 64 * h, row);
+#pragma unroll
+                for (int h = 0; h < kOutCols / 64; ++h)
+                    tma_load_2d_pair(a_dst + kABytes + h * (BK * 128), tmB, leader_full, j0 + 64 * h, row);
+                if (++stage == kNtPairStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0 && nkb > 0) {
+            constexpr uint32_t idesc = instr_desc(2 * BM, BN, 1, 1);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!(ok = mbar_wait(rfull(stage), phase, s.abort_flag))) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kNtPairStageBytes);
+                const uint64_t adesc = smem_desc_mnmajor(a_addr);
+                const uint64_t bdesc = smem_desc_mnmajor(a_addr + kABytes);
+#pragma unroll
+                for (int k = 0; k < BK / UK; ++k)
+                    umma_bf16_pair(tmem_base, adesc + (uint64_t)(128 * k), bdesc + (uint64_t)(128 * k), idesc,
+                                   (uint32_t)((kb | k) != 0));
+                umma_commit_pair(rempty(stage));
+                if (++stage == kNtPairStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+            if (ok) umma_commit_pair(s.tmem_full(0));
+        }
+    } else {
+        const int q = warp & 3;
+        const int row = i0 + q * 32 + lane;
+        float* dst_row = p.part + ((size_t)split * p.I + row) * p.J + j0;
+        bool ok = true;
+        if (nkb > 0) {
+            ok = mbar_wait(s.tmem_full(0), 0, s.abort_flag);
+            tc_fence_after();
+        }
+        if (ok) {
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < kOutCols; c += 32) {
+                float v[32];
+                if (nkb > 0) {
+                    uint32_t r[32], r2[32];
+                    tmem_ld32(t_row + (uint32_t)c, r);
+                    tmem_ld32(t_row + (uint32_t)(kOutCols + c), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) + __uint_as_float(r2[i]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0.f;
+                }
+                if (row < p.I) {
+                    float4* dst = reinterpret_cast<float4*>(dst_row + c);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+            }
+        }
+    }
+    // nobody leaves (or frees tensor memory) while the other CTA may still signal or compute
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync_all();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc_pair(tmem_base, BN);
+    if (threadIdx.x == 0 && *s.abort_flag && p.hdr) p.hdr->status = SSM_ERR_TIMEOUT;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
 // Row-major bf16 matrix [rows, cols] (cols contiguous), boxes of box_cols x box_rows, 128-byte swizzle.
@@ -1961,6 +2098,9 @@ int tc_nt_splits(int K, int I, int J) {
     return s;
 }
 
+#ifndef SSM_NT_PAIRS
+#define SSM_NT_PAIRS 1   // weight-gradient products on CTA pairs where the output has a multiple of 256 rows
+#endif
 int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
     using namespace tc;
     CUtensorMap ma, mbh, mbl;
@@ -1984,6 +2124,13 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
     if (!make_map(&mbl, g.Bm_lo, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
     const int j_tiles = g.J / (BN / 2);
     NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr, 0, 0u, 0u};
+    if (SSM_NT_PAIRS && g.I % (2 * BM) == 0 && g.lda == 0) {   // 256 x 256 tiles on CTA pairs
+        dim3 grid(2 * (g.I / (2 * BM)) * j_tiles, g.splits);
+        count_launch();
+        const bool ok = set_smem(gemm_tc_nt_pair_kernel, kNtPairSmemBytes);
+        gemm_tc_nt_pair_kernel<<<grid, kThreads, kNtPairSmemBytes, st>>>(ma, mbh, mbl, p);
+        return ok ? SSM_OK : SSM_ERR_CUDA;
+    }
     dim3 grid((g.I / BM) * j_tiles, g.splits);
     count_launch();
     const bool ok = set_smem(gemm_tc_nt_kernel<false>, kNtSmemBytes);
