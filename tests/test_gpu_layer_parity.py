@@ -133,6 +133,13 @@ def test_every_step_flagged_and_no_flags(io):
     run(I.small_variant(w, p_done=0.0), with_gxT=True)
 
 
+def test_very_many_short_sequences_fp32():
+    # more than 512 * 64 sequences: the per-sequence partial sums of gAbar take two passes of the row reduction
+    # (alternating between its two buffers) before the last kernel of the backward pass adds what is left
+    w = I.Workload("many", B=33000, T=2, H=8, P=8, io_dtype="f32", p_done=0.1, seed=78)
+    run(w, with_x0=True, with_gxT=True)
+
+
 def test_long_sequence_small_batch_fp32():
     # long enough that a sequence is many tiles, with the state carried from tile to tile
     w = I.Workload("long", B=2, T=2500, H=16, P=24, io_dtype="f32", p_done=0.003, seed=77)
