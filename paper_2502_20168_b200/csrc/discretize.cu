@@ -181,32 +181,6 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* W, int H, int n, int 
 // neighbouring states come out as (re, re, im, im): the kernel that scans the accumulators in its
 // epilogue advances two states per packed instruction.  State p, component c -> row
 // (p / 64) * 128 + 4 * ((p % 64) / 2) + 2 * c + p % 2 of the [2P, H] operand.
-__global__ void pack_operands_tc_kernel(int H, int P, bool pair_cols, bool pair_cols_C, const float2* __restrict__ Bbar, const float2* __restrict__ Cc,
-                                        __nv_bfloat16* __restrict__ WsB, __nv_bfloat16* __restrict__ WsC,
-                                        __nv_bfloat16* __restrict__ Cp, __nv_bfloat16* __restrict__ Bq) {
-    const size_t n = (size_t)P * H;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        {   // i indexes Bbar[p, h]
-            const int p = (int)(i / H), h = (int)(i % H);
-            const float2 v = Bbar[i];
-            const int n = pair_cols ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
-            store_split(WsB, H, n, h, v.x);
-            store_split(WsB, H, n + (pair_cols ? 2 : 1), h, v.y);
-            Bq[(size_t)h * 2 * P + 2 * p] = __float2bfloat16_rn(v.x);
-            Bq[(size_t)h * 2 * P + 2 * p + 1] = __float2bfloat16_rn(v.y);
-        }
-        {   // i indexes C[h, p]
-            const int h = (int)(i / P), p = (int)(i % P);
-            const float2 v = Cc[i];
-            Cp[(size_t)h * 2 * P + 2 * p] = __float2bfloat16_rn(v.x);
-            Cp[(size_t)h * 2 * P + 2 * p + 1] = __float2bfloat16_rn(-v.y);
-            const int n = pair_cols_C ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
-            store_split(WsC, H, n, h, v.x);
-            store_split(WsC, H, n + (pair_cols_C ? 2 : 1), h, -v.y);
-        }
-    }
-}
-
 // Discretisation and operand packing of the tensor-core path in one kernel: block p computes Abar_p and
 // gamma_p (double precision, one thread), then the row p of Bbar with its packed forms and the packed forms
 // of column p of C.
@@ -305,16 +279,6 @@ void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C,
     discretize_pack_tc_kernel<<<P, 128, 0, st>>>(H, P, pair_cols_B, pair_cols_C, Lambda, Delta, Bc, Cc, Abar, Abar_lo, Bbar,
                                                  (__nv_bfloat16*)Wsplit_B, (__nv_bfloat16*)Wsplit_C, (__nv_bfloat16*)Cp,
                                                  (__nv_bfloat16*)Bq);
-}
-
-void launch_pack_operands_tc(int H, int P, bool pair_cols, bool pair_cols_C, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
-                             void* Cp, void* Bq, cudaStream_t st) {
-    const int threads = 256;
-    const int blocks = (int)(((size_t)P * H + threads - 1) / threads);
-    count_launch();
-    pack_operands_tc_kernel<<<blocks, threads, 0, st>>>(H, P, pair_cols, pair_cols_C, Bbar, Cc, (__nv_bfloat16*)Wsplit_B,
-                                                        (__nv_bfloat16*)Wsplit_C, (__nv_bfloat16*)Cp,
-                                                        (__nv_bfloat16*)Bq);
 }
 
 void launch_discretize(int H, int P, const float2* Lambda, const float* Delta, const float2* Bc, float2* Abar,

@@ -182,22 +182,10 @@ void launch_gemm_nt(const GemmNT& g, cudaStream_t st) {
         gemm_nt_kernel<float, float><<<grid, kGemmThreads, 0, st>>>((const float*)g.A, g.I, (const float*)g.Bm, g.J, g.K, kps, g.part);
 }
 
-__global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits, int I, int J, int mode,
-                                     float* __restrict__ out) {
-    const size_t n = (size_t)I * J;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        float acc = 0.f;
-        for (int s = 0; s < splits; ++s) acc += part[(size_t)s * n + e];
-        const int i = (int)(e / J), j = (int)(e % J);
-        if (mode == 0)
-            out[((size_t)(j >> 1) * I + i) * 2 + (j & 1)] = acc;
-        else
-            out[((size_t)i * (J >> 1) + (j >> 1)) * 2 + (j & 1)] = (j & 1) ? -acc : acc;
-    }
-}
-
 // Both weight-gradient reductions of a layer in one launch: blockIdx.y = 0 sums part0 into out0 in mode 0,
 // blockIdx.y = 1 sums part1 into out1 in mode 1.
+// mode 0: complex out[J/2, I]: out[j/2, i].(re if j even else im) = sum_s part[s,i,j]
+// mode 1: complex out[I, J/2]: out[i, j/2] likewise, with the imaginary part negated
 __global__ void splitk_reduce2_kernel(const float* __restrict__ part0, const float* __restrict__ part1, int splits,
                                       int I, int J, float* __restrict__ out0, float* __restrict__ out1) {
     const size_t n = (size_t)I * J;
@@ -221,13 +209,6 @@ void launch_splitk_reduce2(const float* part0, const float* part1, int splits, i
     const int blocks = (int)(((size_t)I * J + threads - 1) / threads);
     count_launch();
     splitk_reduce2_kernel<<<dim3(blocks, 2), threads, 0, st>>>(part0, part1, splits, I, J, (float*)out0, (float*)out1);
-}
-
-void launch_splitk_reduce(const float* part, int splits, int I, int J, int mode, float2* out, cudaStream_t st) {
-    const int threads = 256;
-    const int blocks = (int)(((size_t)I * J + threads - 1) / threads);
-    count_launch();
-    splitk_reduce_kernel<<<blocks, threads, 0, st>>>(part, splits, I, J, mode, (float*)out);
 }
 
 }  // namespace ssm

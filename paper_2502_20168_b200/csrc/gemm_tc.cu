@@ -1,19 +1,25 @@
 #include <type_traits>
 // bf16 projections on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
-// memory, operands staged in shared memory by TMA).  Two kernels:
+// memory, operands staged in shared memory by TMA).  The kernels:
 //
-//  * gemm_tc_tn_kernel: out[m, n] = sum_k A[m, k] * W[n, k]  (both operands K-contiguous).
-//    Persistent, one CTA per SM walking 128 x 256 accumulator tiles.  A = activations or states
-//    [B*T, K]; W = packed parameters.  With kSplitW the 256 accumulator columns of a tile hold
-//    the products with the high and the low bf16 halves of 128 weight rows, summed in the
-//    epilogue (weights then carry ~16 mantissa bits; see pack_operands_tc_kernel).
-//  * gemm_tc_nt_kernel: part[s, i, j] = sum_{m in slice s} A[m, i] * Bm[m, j]  (both operands
-//    contiguous in the output index, i.e. MN-major), split over the B*T rows.
+//  * gemm_tc_tn_kernel / gemm_tc_tn_pair_kernel: out[m, n] = sum_k A[m, k] * W[n, k]  (both operands
+//    K-contiguous).  Persistent; one CTA per SM walking 128 x 256 accumulator tiles, or clusters of two
+//    CTAs on 256 x 256 tiles.  A = activations or states [B*T, K]; W = packed parameters.  With kSplitW
+//    the 256 accumulator columns of a tile hold the products with the high and the low bf16 halves of 128
+//    weight rows, summed in the epilogue (weights then carry ~16 mantissa bits; see
+//    discretize_pack_tc_kernel).  With a product schedule the accumulator sums several products of bf16
+//    planes of both operands (fp32-accurate results, see planes.cu).  Epilogues: fp32 store; bf16
+//    acc + diag * skip; the same with column sums of skip * dot; fp32 store with a gated bf16 result.
+//  * gemm_scan_fwd_kernel / gemm_scan_bwd_kernel: the pair kernel with the scan of Sec. III-B (and its
+//    adjoint) in the epilogue, so that Bu and g_x never reach memory.
+//  * gemm_tc_nt_kernel / gemm_tc_nt_pair_kernel: part[s, i, j] = sum_{m in slice s} A[m, i] * Bm[m, j]
+//    (both operands contiguous in the output index, i.e. MN-major), split over the B*T rows: the weight
+//    gradients.
 //
-// Warp roles in both: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
-// warps 2..5 drain accumulators (one TMEM lane quarter each).  Every mbarrier wait is bounded;
-// a wait that gives up raises a CTA-wide abort flag, the status word of the workspace header
-// is set, tensor memory is released and the kernel returns.
+// Warp roles in all: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs, the other
+// warps drain accumulators (each may read one TMEM lane quarter).  Every mbarrier wait is bounded; a wait
+// that gives up raises a CTA-wide abort flag, the status word of the workspace header is set, tensor
+// memory is released and the kernel returns.
 #include <map>
 #include <mutex>
 #include <utility>
@@ -2124,7 +2130,7 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st) {
     if (!make_map(&mbl, g.Bm_lo, (uint64_t)g.K, (uint64_t)g.J, 64, BK)) return SSM_ERR_CUDA;
     const int j_tiles = g.J / (BN / 2);
     NtParams p{g.K, g.J, g.I, j_tiles, bps, g.part, g.hdr, 0, 0u, 0u};
-    if (SSM_NT_PAIRS && g.I % (2 * BM) == 0 && g.lda == 0) {   // 256 x 256 tiles on CTA pairs
+    if (SSM_NT_PAIRS && g.I % (2 * BM) == 0) {   // 256 x 256 tiles on CTA pairs
         dim3 grid(2 * (g.I / (2 * BM)) * j_tiles, g.splits);
         count_launch();
         const bool ok = set_smem(gemm_tc_nt_pair_kernel, kNtPairSmemBytes);

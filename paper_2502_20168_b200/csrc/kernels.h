@@ -55,9 +55,7 @@ size_t colsum_tmp_floats(int R, int C);
 // Reduces [R, C] partial sums to at most `limit` rows (groups of rows summed in a fixed order; `in` and `tmp`,
 // colsum_tmp_floats(R, C) floats, are both overwritten); returns where the rows are, *rows_out how many.
 const float* launch_reduce_rows(float* in, int R, int C, float* tmp, int limit, int* rows_out, cudaStream_t st);
-// out[c] = sum_m a[m,c]*b[m,c]; a and b each fp32 or bf16.
-void launch_dot_columns(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* out, float* tmp,
-                        cudaStream_t st);
+// part[g, c] = sum over the rows m of group g of a[m,c]*b[m,c]; a and b each fp32 or bf16.
 size_t dot_columns_tmp_floats(int M, int C);
 // The group sums only: tmp[g, c] for g < the returned number of groups.
 int launch_dot_columns_partial(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* tmp,
@@ -87,16 +85,13 @@ struct GemmNT {
 };
 int gemm_nt_splits(int K);
 void launch_gemm_nt(const GemmNT& g, cudaStream_t st);
-// mode 0: complex out[J/2, I]: out[j/2, i].(re if j even else im) = sum_s part[s,i,j]
-// mode 1: complex out[I, J/2]: out[i, j/2] likewise, with the imaginary part negated
-void launch_splitk_reduce(const float* part, int splits, int I, int J, int mode, float2* out, cudaStream_t st);
 // part0 in mode 0 into out0 and part1 in mode 1 into out1, one launch
 void launch_splitk_reduce2(const float* part0, const float* part1, int splits, int I, int J, float2* out0, float2* out1,
                            cudaStream_t st);
 
 // gemm_tc.cu: bf16 projections on tcgen05 tensor cores (operands by TMA, accumulators in TMEM).
 struct GemmTcTN {
-    // out[m, n] = sum_k A[m, k] * W[n, k];  A bf16 [M, K];  W bf16 packed by pack_operands_tc:
+    // out[m, n] = sum_k A[m, k] * W[n, k];  A bf16 [M, K];  W bf16 packed by discretize_pack_tc_kernel:
     // [N_out, K], or with split_w [2 * N_out, K] where each group of 256 rows holds the high
     // halves of 128 output columns followed by their low halves.
     const void* A; const void* W;
@@ -191,9 +186,7 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 
 // discretize.cu: operands of the tensor-core path (bf16).  Wsplit_B / Wsplit_C: [4P, H] hi/lo
 // stacked forms of Bp / Cq (see GemmTcTN);  Cp, Bq: [H, 2P] single bf16.
-void launch_pack_operands_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Bbar, const float2* Cc, void* Wsplit_B, void* Wsplit_C,
-                             void* Cp, void* Bq, cudaStream_t st);
-// launch_discretize and launch_pack_operands_tc in one kernel.
+// Discretisation and packing of the four bf16 operands in one kernel.
 void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
                                const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
                                void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st);

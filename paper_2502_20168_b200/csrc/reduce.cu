@@ -119,24 +119,7 @@ size_t dot_columns_tmp_floats(int M, int C) {
     return (size_t)g * C + colsum_tmp_floats(g, C);
 }
 
-void launch_dot_columns(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* out, float* tmp,
-                        cudaStream_t st) {
-    using bf = __nv_bfloat16;
-    const int g = dot_groups(M);
-    dim3 blk(32, 8), grid(g, (C + 127) / 128);   // row groups along x: no 65535 limit there
-    count_launch();
-    if (a_bf16 && b_bf16)
-        dot_columns_kernel<bf, bf><<<grid, blk, 0, st>>>((const bf*)a, (const bf*)b, M, C, tmp);
-    else if (a_bf16)
-        dot_columns_kernel<bf, float><<<grid, blk, 0, st>>>((const bf*)a, (const float*)b, M, C, tmp);
-    else if (b_bf16)
-        dot_columns_kernel<float, bf><<<grid, blk, 0, st>>>((const float*)a, (const bf*)b, M, C, tmp);
-    else
-        dot_columns_kernel<float, float><<<grid, blk, 0, st>>>((const float*)a, (const float*)b, M, C, tmp);
-    launch_colsum(tmp, g, C, out, tmp + (size_t)g * C, st);
-}
-
-// The same without the final sum: the group sums stay in tmp[0 .. groups * C); returns the number of groups.
+// The group sums stay in tmp[0 .. groups * C) (the caller adds them); returns the number of groups.
 int launch_dot_columns_partial(bool a_bf16, const void* a, bool b_bf16, const void* b, int M, int C, float* tmp,
                                cudaStream_t st) {
     using bf = __nv_bfloat16;
