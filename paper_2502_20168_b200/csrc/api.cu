@@ -209,8 +209,8 @@ static void layer_prepare(const ssm_shape& s, const LayerPlan& p, const ssm_c64*
     StageTimer tm("discretize_pack", st);
     if (p.tc) {
         // one kernel (the kernels that scan in the epilogue of a projection want their own column order)
-        launch_discretize_pack_tc(s.H, s.P, tc_gemm_scan_fwd_supported(s.B, s.T, s.H, s.P),
-                                  tc_gemm_scan_bwd_supported(s.B, s.T, s.H, s.P), (const float2*)Lambda, Delta,
+        const int group = tc_gemm_scan_group(s.B, s.T, s.H, s.P);
+        launch_discretize_pack_tc(s.H, s.P, group, group, (const float2*)Lambda, Delta,
                                   (const float2*)Bc, (const float2*)Cc, at<float2>(ws, p.Abar), at<float2>(ws, p.Alo),
                                   at<float2>(ws, p.Bbar), at<void>(ws, p.W0), at<void>(ws, p.W1), at<void>(ws, p.W2),
                                   at<void>(ws, p.W3), st);

@@ -169,23 +169,20 @@ __global__ void pack_operands_kernel(int H, int P, const float2* __restrict__ Bb
 // in the two projections that feed the states (Bu and g_x), so that the states see ~16
 // mantissa bits of the parameters.  Logical row n of the [2P, H] operand goes to rows
 // (n/128)*256 + n%128 (hi) and (n/128)*256 + 128 + n%128 (lo) of the stacked [4P, H] matrix.
-__device__ __forceinline__ void store_split(__nv_bfloat16* W, int H, int n, int h, float w) {
+// `stack`: rows per hi (and per lo) block, 128 for the plain projections, twice the states per chain otherwise.
+__device__ __forceinline__ void store_split(__nv_bfloat16* W, int H, int n, int h, float w, int stack = 128) {
     const __nv_bfloat16 hi = __float2bfloat16_rn(w);
     const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
-    const size_t r = (size_t)(n >> 7) * 256 + (n & 127);
+    const size_t r = (size_t)(n / stack) * (2 * stack) + (n % stack);
     W[r * H + h] = hi;
-    W[(r + 128) * H + h] = lo;
+    W[(r + stack) * H + h] = lo;
 }
 
-// pair_cols (Bbar operand), pair_cols_C (conj(C) operand): the rows of the operand are ordered so that the accumulator columns of two
-// neighbouring states come out as (re, re, im, im): the kernel that scans the accumulators in its
-// epilogue advances two states per packed instruction.  State p, component c -> row
-// (p / 64) * 128 + 4 * ((p % 64) / 2) + 2 * c + p % 2 of the [2P, H] operand.
 // Discretisation and operand packing of the tensor-core path in one kernel: block p computes Abar_p and
 // gamma_p (double precision, one thread), then the row p of Bbar with its packed forms and the packed forms
 // of column p of C.
 __global__ void __launch_bounds__(128)
-discretize_pack_tc_kernel(int H, int P, bool pair_cols, bool pair_cols_C, const float2* __restrict__ Lambda,
+discretize_pack_tc_kernel(int H, int P, int group_B, int group_C, const float2* __restrict__ Lambda,
                           const float* __restrict__ Delta, const float2* __restrict__ Bc, const float2* __restrict__ Cc,
                           float2* __restrict__ Abar, float2* __restrict__ Abar_lo, float2* __restrict__ Bbar,
                           __nv_bfloat16* __restrict__ WsB, __nv_bfloat16* __restrict__ WsC,
@@ -201,18 +198,20 @@ discretize_pack_tc_kernel(int H, int P, bool pair_cols, bool pair_cols_C, const 
     }
     __syncthreads();
     const float2 g = gamma_s;
-    const int nB = pair_cols ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
-    const int nC = pair_cols_C ? (p >> 6) * 128 + 4 * ((p & 63) >> 1) + (p & 1) : 2 * p;
+    // state p, component c -> row (p / G) 2G + 4 ((p % G) / 2) + 2 c + p % 2 inside groups of G states
+    auto row_of = [&](int G) { return G ? (p / G) * 2 * G + 4 * ((p % G) >> 1) + (p & 1) : 2 * p; };
+    const int nB = row_of(group_B), nC = row_of(group_C);
+    const int sB = group_B ? 2 * group_B : 128, sC = group_C ? 2 * group_C : 128;
     for (int h = threadIdx.x; h < H; h += blockDim.x) {
         const float2 v = cmul(g, Bc[(size_t)p * H + h]);
         Bbar[(size_t)p * H + h] = v;
-        store_split(WsB, H, nB, h, v.x);
-        store_split(WsB, H, nB + (pair_cols ? 2 : 1), h, v.y);
+        store_split(WsB, H, nB, h, v.x, sB);
+        store_split(WsB, H, nB + (group_B ? 2 : 1), h, v.y, sB);
         *reinterpret_cast<__nv_bfloat162*>(Bq + (size_t)h * 2 * P + 2 * p) = __floats2bfloat162_rn(v.x, v.y);
         const float2 c = Cc[(size_t)h * P + p];
         *reinterpret_cast<__nv_bfloat162*>(Cp + (size_t)h * 2 * P + 2 * p) = __floats2bfloat162_rn(c.x, -c.y);
-        store_split(WsC, H, nC, h, c.x);
-        store_split(WsC, H, nC + (pair_cols_C ? 2 : 1), h, -c.y);
+        store_split(WsC, H, nC, h, c.x, sC);
+        store_split(WsC, H, nC + (group_C ? 2 : 1), h, -c.y, sC);
     }
 }
 
@@ -272,11 +271,11 @@ void launch_discretize_pack_planes(int H, int P, const float2* Lambda, const flo
                                                      (__nv_bfloat16*)Cq3, (__nv_bfloat16*)Cp3, (__nv_bfloat16*)Bq3);
 }
 
-void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
+void launch_discretize_pack_tc(int H, int P, int group_B, int group_C, const float2* Lambda, const float* Delta,
                                const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
                                void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st) {
     count_launch();
-    discretize_pack_tc_kernel<<<P, 128, 0, st>>>(H, P, pair_cols_B, pair_cols_C, Lambda, Delta, Bc, Cc, Abar, Abar_lo, Bbar,
+    discretize_pack_tc_kernel<<<P, 128, 0, st>>>(H, P, group_B, group_C, Lambda, Delta, Bc, Cc, Abar, Abar_lo, Bbar,
                                                  (__nv_bfloat16*)Wsplit_B, (__nv_bfloat16*)Wsplit_C, (__nv_bfloat16*)Cp,
                                                  (__nv_bfloat16*)Bq);
 }

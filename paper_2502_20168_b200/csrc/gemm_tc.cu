@@ -775,11 +775,11 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // tile, and every row group that begins a sequence starts from that sequence's initial state.
 struct FsParams {
     int B, T, P;
-    int n_tiles;      // 2P / 128
+    int n_tiles;      // state groups: P / kS
     int k_blocks;     // H / 64
     int tblocks;      // tiles per chain: T / 128, or 1
     int unit_rows;    // rows of a chain: T, or 128 when T < 128
-    int n_units;      // chains per 64 states: B, or ceil(B * T / 128)
+    int n_units;      // chains per state group: B, or ceil(B * T / 128)
     int gps;          // row groups per sequence inside a tile: 8, or T / 16
     int nchains;      // n_tiles * ceil(n_units / 2)
     const float2* Abar;
@@ -791,13 +791,27 @@ struct FsParams {
     WsHeader* hdr;
 };
 
-constexpr int kFsTileBytes = BM * 128 * 4;   // 128 rows x 128 fp32
-constexpr size_t kFsSmemBytes = (size_t)kPairStages * kPairStageBytes + kFsTileBytes + 1024 + 256;
-
-constexpr int kFsEpiWarps = 8;               // two per TMEM lane quarter (16 measured slower: 0.34 against 0.31 ms)
-constexpr int kFsEpiThreads = 32 * kFsEpiWarps;
-constexpr int kFsThreads = 64 + kFsEpiThreads;
-constexpr int kFsRows = BM * 32 / kFsEpiThreads;   // rows per scanning thread: 32 pairs of states x (128 / kFsRows) groups
+// Sizes of the kernels that scan in their epilogue, for chains of kS states (64, or 32 where 64-state
+// chains would leave CTA pairs without work): the MMA tile is 256 rows x 4 kS columns (re / im of kS states,
+// hi | lo weight halves), a CTA holds 2 kS weight rows, the fp32 tile it scans is 128 rows x 2 kS columns,
+// and kS / 2 scanning threads (two states each) share a group of 16 rows.
+constexpr int kFsRows = 16;                  // rows per scanning thread; 8 row groups per tile
+template <int kS>
+struct FsCfg {
+    static_assert(kS == 64 || kS == 32, "chains of 64 or 32 states");
+    static constexpr int kPairs = kS / 2;              // state pairs of a tile = scanning threads per row group
+    static constexpr int kN = 4 * kS;                  // accumulator columns of a tile
+    static constexpr int kCols = 2 * kS;               // fp32 columns after hi + lo
+    static constexpr int kChunks = kCols / 4;          // 16-byte chunks per row of the fp32 tile
+    static constexpr int kWRows = 2 * kS;              // weight rows per CTA
+    static constexpr int kEpiWarps = kS / 8;           // 8 (two per TMEM lane quarter; 16 measured slower) or 4
+    static constexpr int kEpiThreads = 32 * kEpiWarps;
+    static constexpr int kThreads = 64 + kEpiThreads;
+    static constexpr int kTileBytes = BM * kCols * 4;
+    static constexpr int kStageBytes = kABytes + kWRows * BK * 2;
+    static constexpr int kGroupBytes = 2 * kFsRows * kPairs * 8;   // both planes of one row group's results
+    static constexpr size_t kSmemBytes = (size_t)kPairStages * kStageBytes + kTileBytes + 1024 + 256;
+};
 
 // Two fp32 values in one 64-bit register pair, and the packed multiply-add on them: the scan of
 // the epilogue advances two states per instruction.
@@ -836,15 +850,21 @@ __device__ __forceinline__ C2 cstep2(f32x2 ar, f32x2 ai, f32x2 nai, C2 x, C2 b) 
     return r;
 }
 
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kFsEpiThreads) : "memory"); }
+template <int kThreadsN>
+__device__ __forceinline__ void epi_sync_n() { asm volatile("bar.sync 1, %0;" ::"n"(kThreadsN) : "memory"); }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFsThreads, 1)
+template <int kS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FsCfg<kS>::kThreads, 1)
 gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
                      const __grid_constant__ CUtensorMap tmX, FsParams p) {
+    using Cfg = FsCfg<kS>;
+    constexpr int kPairs = Cfg::kPairs, kChunks = Cfg::kChunks, kFsEpiThreads = Cfg::kEpiThreads, kFsEpiWarps = Cfg::kEpiWarps;
+    constexpr int kStageB = Cfg::kStageBytes;
+    auto epi_sync = [] { epi_sync_n<Cfg::kEpiThreads>(); };
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float4 agg_e[kFsEpiThreads], carry_s[32];   // (re, re, im, im) of two neighbouring states
+    __shared__ float4 agg_e[kFsEpiThreads], carry_s[kPairs];   // (re, re, im, im) of two neighbouring states
     __shared__ uint32_t masks[4];
-    const Smem s = carve_smem(smem_raw, kPairStages, kFsTileBytes, 0, kPairStageBytes, 0);
+    const Smem s = carve_smem(smem_raw, kPairStages, Cfg::kTileBytes, 0, kStageB, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     if (threadIdx.x == 0) {
@@ -885,15 +905,15 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             uint32_t phase = 0;
             bool ok = true;
             for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
-                const int n0 = (chain % p.n_tiles) * BN + (int)rank * (BN / 2);
+                const int n0 = (chain % p.n_tiles) * Cfg::kN + (int)rank * Cfg::kWRows;
                 for (int tb = 0; tb < p.tblocks && ok; ++tb) {
                     const int m0 = row_of(chain, tb);
                     // (no L2 prefetch of the next tile's rows here: with it the kernel ran 7 % slower)
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
                         if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
                         const uint32_t leader_full = map_to_cta(s.full(stage), 0);
-                        if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kPairStageBytes);
-                        const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kStageB);
+                        const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageB);
                         tma_load_2d_pair(a_dst, &tmA, leader_full, kb * BK, m0);
                         tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full, kb * BK, n0);
                         if (++stage == kPairStages) {
@@ -906,7 +926,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = instr_desc(2 * BM, BN, 0, 0);
+            constexpr uint32_t idesc = instr_desc(2 * BM, Cfg::kN, 0, 0);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -914,11 +934,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 for (int tb = 0; tb < p.tblocks && ok; ++tb) {
                     if (!(ok = mbar_wait(s.tmem_empty(acc), acc_phase ^ 1u, s.abort_flag))) break;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * Cfg::kN);
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
                         if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                         tc_fence_after();
-                        const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageB);
                         const uint64_t adesc = smem_desc_kmajor(a_addr);
                         const uint64_t bdesc = smem_desc_kmajor(a_addr + kABytes);
 #pragma unroll
@@ -942,7 +962,8 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
         const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
         const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
-        const int sp = te & 31, sl = te >> 5;       // scan role: pair of states of the tile, group of its rows
+        const int sp = te % kPairs, sl = te / kPairs;   // scan role: pair of states of the tile, group of its rows
+        const bool group_leader = lane % kPairs == 0;   // the lane that talks to the TMA unit for its row group
         const int prow = q * 32 + lane;             // drain role: row of the tile
         float4* T4 = reinterpret_cast<float4*>(s.staging);
         const C2 zero = {0ull, 0ull};
@@ -955,7 +976,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const bool short_seq = p.T < BM;        // then b counts tiles of rows, not sequences
             const int g0 = sl - sl % p.gps;         // the first row group of this group's sequence in the tile
             const bool from_carry = sl == g0;
-            const int pg = n_tile * 64 + 2 * sp;    // the first of this thread's two states
+            const int pg = n_tile * kS + 2 * sp;    // the first of this thread's two states
             const float2 a0 = p.Abar[pg], a1 = p.Abar[pg + 1];
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
             f32x2 pr, pi, npi;   // Abar^R by squaring in fp32 (a few 1e-7 relative: the results leave as bf16 pairs)
@@ -987,7 +1008,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (lane == 0) masks[te >> 5] = mk;
                 }
                 (void)mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag);
-                if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
+                if (group_leader) tma_store_wait_read();   // this row group's results of the previous tile have left shared memory
                 epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
                               // the 256 threads leave together or not at all
                 if (*s.abort_flag) {
@@ -996,16 +1017,16 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 tc_fence_after();
                 // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7)
-                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * Cfg::kN);
 #pragma unroll
-                for (int g = grp; g < 4; g += kFsEpiWarps / 4) {   // 32 columns = one 128-byte group of the row
+                for (int g = grp; g < Cfg::kCols / 32; g += kFsEpiWarps / 4) {   // 32 columns = one 128-byte group of the row
                     uint32_t r[32], r2[32];
                     tmem_ld32(t_row + (uint32_t)(g * 32), r);
-                    tmem_ld32(t_row + (uint32_t)(BN / 2 + g * 32), r2);
+                    tmem_ld32(t_row + (uint32_t)(Cfg::kCols + g * 32), r2);
                     tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        T4[prow * 32 + g * 8 + (j ^ (prow & 7))] =
+                        T4[prow * kChunks + g * 8 + (j ^ (prow & 7))] =
                             make_float4(__uint_as_float(r[4 * j]) + __uint_as_float(r2[4 * j]),
                                         __uint_as_float(r[4 * j + 1]) + __uint_as_float(r2[4 * j + 1]),
                                         __uint_as_float(r[4 * j + 2]) + __uint_as_float(r2[4 * j + 2]),
@@ -1035,7 +1056,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
                 for (int i = 0; i < R; ++i) {
                     const int row = r0 + i;
-                    const float4 t = T4[row * 32 + ((sp & ~7) | ((sp & 7) ^ (row & 7)))];   // (re, re, im, im)
+                    const float4 t = T4[row * kChunks + ((sp & ~7) | ((sp & 7) ^ (row & 7)))];   // (re, re, im, im)
                     v[i].re = pack2(t.x, t.y);
                     v[i].im = pack2(t.z, t.w);
                 }
@@ -1082,14 +1103,14 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 C2 x = e;
                 if (!from_carry) {   // state before this group's first row
                     {
-                        const float4 c = agg_e[g0 * 32 + sp];
+                        const float4 c = agg_e[g0 * kPairs + sp];
                         x.re = pack2(c.x, c.y);
                         x.im = pack2(c.z, c.w);
                     }
 #pragma unroll
                     for (int g = 1; g < nsl - 1; ++g) {
                         if (g > g0 && g < sl) {
-                            const float4 c = agg_e[g * 32 + sp];
+                            const float4 c = agg_e[g * kPairs + sp];
                             const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
                             x = ((gflags >> g) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
                         }
@@ -1097,7 +1118,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 // (3) fold again; results as hi / lo bf16 halves into this warp's part of the tile (everybody
                 // has its rows in registers by now): [plane][row][64 states], which the warp hands to the TMA unit
-                uint8_t* warp_out = s.staging + sl * (2 * R * 256);
+                uint8_t* warp_out = s.staging + sl * Cfg::kGroupBytes;
                 uint2* out = reinterpret_cast<uint2*>(warp_out) + sp;
                 auto emit = [&](int i, C2 xv) {
                     float re0, re1, im0, im1;
@@ -1107,8 +1128,8 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
                     const __nv_bfloat162 l0 = __floats2bfloat162_rn(re0 - f0.x, im0 - f0.y);
                     const __nv_bfloat162 l1 = __floats2bfloat162_rn(re1 - f1.x, im1 - f1.y);
-                    out[i * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-                    out[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+                    out[i * kPairs] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                    out[(R + i) * kPairs] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
                 };
                 if (from_carry) {
 #pragma unroll
@@ -1125,8 +1146,8 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0 && grp_valid) {
-                    tma_store_3d_nocommit(&tmX, smem_u32(warp_out), n_tile * 64, m0 + r0, 0);
+                if (group_leader && grp_valid) {
+                    tma_store_3d_nocommit(&tmX, smem_u32(warp_out), n_tile * kS, m0 + r0, 0);
                     tma_commit_group();
                 }
                 if (short_seq ? (sl - g0 == p.gps - 1) : (sl == nsl - 1)) {   // the group that ends a sequence or the tile
@@ -1143,7 +1164,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
             }
         }
-        if (lane == 0) tma_store_wait_all();
+        if (group_leader) tma_store_wait_all();
     }
     tc_fence_before();
     __syncwarp();
@@ -1170,11 +1191,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 // state), each written once.  T must be a multiple of 128.
 struct FbParams {
     int B, T, P;
-    int n_tiles;      // 2P / 128
+    int n_tiles;      // state groups: P / kS
     int k_blocks;     // H / 64
     int tblocks;      // tiles per chain: T / 128, or 1
     int unit_rows;    // rows of a chain: T, or 128 when T < 128 (a tile then holds 128 / T whole sequences)
-    int n_units;      // chains per 64 states: B, or ceil(B * T / 128)
+    int n_units;      // chains per state group: B, or ceil(B * T / 128)
     int gps;          // row groups per sequence inside a tile: 8, or T / 16
     int nchains;      // n_tiles * ceil(n_units / 2)
     const float2* Abar;
@@ -1186,14 +1207,19 @@ struct FbParams {
     WsHeader* hdr;
 };
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFsThreads, 1)
+template <int kS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FsCfg<kS>::kThreads, 1)
 gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
                      const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmS, FbParams p) {
+    using Cfg = FsCfg<kS>;
+    constexpr int kPairs = Cfg::kPairs, kChunks = Cfg::kChunks, kFsEpiThreads = Cfg::kEpiThreads, kFsEpiWarps = Cfg::kEpiWarps;
+    constexpr int kStageB = Cfg::kStageBytes;
+    auto epi_sync = [] { epi_sync_n<Cfg::kEpiThreads>(); };
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float4 agg_e[kFsEpiThreads], carry_s[32];   // (re, re, im, im) of two neighbouring states
+    __shared__ float4 agg_e[kFsEpiThreads], carry_s[kPairs];   // (re, re, im, im) of two neighbouring states
     __shared__ uint32_t masks[8];   // [0, 4): flags of the rows one later (the resets of the reverse scan); [4, 8): of the rows
-    __shared__ __align__(8) uint64_t xbar[kFsEpiWarps];   // one per warp: its rows of x have arrived
-    const Smem s = carve_smem(smem_raw, kPairStages, kFsTileBytes, 0, kPairStageBytes, 0);
+    __shared__ __align__(8) uint64_t xbar[BM / kFsRows];   // one per row group: its rows of x have arrived
+    const Smem s = carve_smem(smem_raw, kPairStages, Cfg::kTileBytes, 0, kStageB, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     if (threadIdx.x == 0) {
@@ -1205,7 +1231,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             mbar_init(s.tmem_full(i), 1);
             mbar_init(s.tmem_empty(i), 2 * kFsEpiThreads);
         }
-        for (int i = 0; i < kFsEpiWarps; ++i) mbar_init(smem_u32(&xbar[i]), 1);
+        for (int i = 0; i < BM / kFsRows; ++i) mbar_init(smem_u32(&xbar[i]), 1);
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1234,14 +1260,14 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             uint32_t phase = 0;
             bool ok = true;
             for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
-                const int n0 = (chain % p.n_tiles) * BN + (int)rank * (BN / 2);
+                const int n0 = (chain % p.n_tiles) * Cfg::kN + (int)rank * Cfg::kWRows;
                 for (int tb = p.tblocks - 1; tb >= 0 && ok; --tb) {
                     const int m0 = row_of(chain, tb);
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
                         if (!(ok = mbar_wait(s.empty(stage), phase ^ 1u, s.abort_flag))) break;
                         const uint32_t leader_full = map_to_cta(s.full(stage), 0);
-                        if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kPairStageBytes);
-                        const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        if (rank == 0) mbar_expect_tx(s.full(stage), 2 * kStageB);
+                        const uint32_t a_dst = smem_u32(s.tiles + (size_t)stage * kStageB);
                         tma_load_2d_pair(a_dst, &tmA, leader_full, kb * BK, m0);
                         tma_load_2d_pair(a_dst + kABytes, &tmWh, leader_full, kb * BK, n0);
                         if (++stage == kPairStages) {
@@ -1254,7 +1280,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = instr_desc(2 * BM, BN, 0, 0);
+            constexpr uint32_t idesc = instr_desc(2 * BM, Cfg::kN, 0, 0);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -1262,11 +1288,11 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 for (int tb = 0; tb < p.tblocks && ok; ++tb) {
                     if (!(ok = mbar_wait(s.tmem_empty(acc), acc_phase ^ 1u, s.abort_flag))) break;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * Cfg::kN);
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
                         if (!(ok = mbar_wait(s.full(stage), phase, s.abort_flag))) break;
                         tc_fence_after();
-                        const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kPairStageBytes);
+                        const uint32_t a_addr = smem_u32(s.tiles + (size_t)stage * kStageB);
                         const uint64_t adesc = smem_desc_kmajor(a_addr);
                         const uint64_t bdesc = smem_desc_kmajor(a_addr + kABytes);
 #pragma unroll
@@ -1290,14 +1316,15 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         constexpr int R = kFsRows, nsl = BM / kFsRows;   // rows per thread; groups of rows
         const int te = threadIdx.x - 64;            // 0 .. kFsEpiThreads - 1
         const int q = warp & 3, grp = (warp - 2) >> 2;   // drain role: TMEM lane quarter, 32-column group
-        const int sp = te & 31, sl = te >> 5;       // scan role: pair of states of the tile, group of its rows
+        const int sp = te % kPairs, sl = te / kPairs;   // scan role: pair of states of the tile, group of its rows
+        const bool group_leader = lane % kPairs == 0;   // the lane that talks to the TMA unit for its row group
         const int prow = q * 32 + lane;             // drain role: row of the tile
         const bool short_seq = p.T < BM;            // then a chain is one tile of 128 / T whole sequences
         const int g0 = sl - sl % p.gps;             // first and last row group of this group's sequence in the tile
         const int gl = g0 + p.gps - 1;
         const bool from_carry = sl == gl;           // the last rows come first
         float4* T4 = reinterpret_cast<float4*>(s.staging);
-        uint8_t* warp_buf = s.staging + sl * (2 * R * 256);   // this warp's rows of the tile; later x_{t-1}, then s
+        uint8_t* warp_buf = s.staging + sl * Cfg::kGroupBytes;   // this row group's rows of the tile; later x_{t-1}, then s
         uint2* xs = reinterpret_cast<uint2*>(warp_buf) + sp;
         const uint32_t xb = smem_u32(&xbar[sl]);
         uint32_t xphase = 0;
@@ -1308,7 +1335,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
             const bool has_seq = b < p.n_units;
-            const int pg = n_tile * 64 + 2 * sp;    // the first of this thread's two states
+            const int pg = n_tile * kS + 2 * sp;    // the first of this thread's two states
             const float2 a0 = cconj(p.Abar[pg]), a1 = cconj(p.Abar[pg + 1]);
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
             f32x2 pr, pi, npi;   // conj(Abar)^R by squaring in fp32
@@ -1351,12 +1378,13 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 // (1) accumulators -> shared-memory tile: 16-byte chunk j of a 128-byte group sits at j ^ (row & 7).
                 // A warp drains two groups of 32 columns (hi + lo halves each): the first group's loads are in
                 // flight while it waits for the tile to be free, the second group's while it stores the first.
-                static_assert(kFsEpiWarps == 8, "two 32-column groups per warp");
-                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+                constexpr int kGrpStep = kFsEpiWarps / 4;   // a warp drains the 32-column groups grp and grp + kGrpStep
+                static_assert(Cfg::kCols / 32 == 2 * kGrpStep, "two 32-column groups per warp");
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * Cfg::kN);
                 uint32_t ra[32], ra2[32], rb[32], rb2[32];
                 tmem_ld32(t_row + (uint32_t)(grp * 32), ra);
-                tmem_ld32(t_row + (uint32_t)(BN / 2 + grp * 32), ra2);
-                if (lane == 0) tma_store_wait_read();   // this warp's results of the previous tile have left shared memory
+                tmem_ld32(t_row + (uint32_t)(Cfg::kCols + grp * 32), ra2);
+                if (group_leader) tma_store_wait_read();   // this row group's results of the previous tile have left shared memory
                 epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
                               // the 256 threads leave together or not at all
                 tmem_ld_wait();
@@ -1364,11 +1392,11 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     ok = false;
                     break;
                 }
-                tmem_ld32(t_row + (uint32_t)((grp + 2) * 32), rb);
-                tmem_ld32(t_row + (uint32_t)(BN / 2 + (grp + 2) * 32), rb2);
+                tmem_ld32(t_row + (uint32_t)((grp + kGrpStep) * 32), rb);
+                tmem_ld32(t_row + (uint32_t)(Cfg::kCols + (grp + kGrpStep) * 32), rb2);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    T4[prow * 32 + grp * 8 + (j ^ (prow & 7))] =
+                    T4[prow * kChunks + grp * 8 + (j ^ (prow & 7))] =
                         make_float4(__uint_as_float(ra[4 * j]) + __uint_as_float(ra2[4 * j]),
                                     __uint_as_float(ra[4 * j + 1]) + __uint_as_float(ra2[4 * j + 1]),
                                     __uint_as_float(ra[4 * j + 2]) + __uint_as_float(ra2[4 * j + 2]),
@@ -1376,7 +1404,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    T4[prow * 32 + (grp + 2) * 8 + (j ^ (prow & 7))] =
+                    T4[prow * kChunks + (grp + kGrpStep) * 8 + (j ^ (prow & 7))] =
                         make_float4(__uint_as_float(rb[4 * j]) + __uint_as_float(rb2[4 * j]),
                                     __uint_as_float(rb[4 * j + 1]) + __uint_as_float(rb2[4 * j + 1]),
                                     __uint_as_float(rb[4 * j + 2]) + __uint_as_float(rb2[4 * j + 2]),
@@ -1406,7 +1434,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
                 for (int i = 0; i < R; ++i) {
                     const int row = r0 + i;
-                    const float4 t = T4[row * 32 + ((sp & ~7) | ((sp & 7) ^ (row & 7)))];   // (re, re, im, im)
+                    const float4 t = T4[row * kChunks + ((sp & ~7) | ((sp & 7) ^ (row & 7)))];   // (re, re, im, im)
                     v[i].re = pack2(t.x, t.y);
                     v[i].im = pack2(t.z, t.w);
                 }
@@ -1421,11 +1449,11 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 // the warp has its rows: rows m - 1 ... m + R - 2 of x (both planes) into its part of the tile
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_expect_tx(xb, 2 * R * 256);
-                    tma_load_3d(smem_u32(warp_buf), &tmX, xb, n_tile * 64, m0 + r0 - 1, 0);
+                if (group_leader) {
+                    mbar_expect_tx(xb, Cfg::kGroupBytes);
+                    tma_load_3d(smem_u32(warp_buf), &tmX, xb, n_tile * kS, m0 + r0 - 1, 0);
                     // and the same rows of the tile before this one into L2, where the next load will find them
-                    if (tb > 0) tma_prefetch_3d(&tmX, n_tile * 64, m0 - BM + r0 - 1, 0);
+                    if (tb > 0) tma_prefetch_3d(&tmX, n_tile * kS, m0 - BM + r0 - 1, 0);
                 }
                 C2 e = zero;
                 if (from_carry) {   // from the carried value (nothing, for a sequence inside the tile): these results are final
@@ -1462,14 +1490,14 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 C2 x = e;
                 if (!from_carry) {   // s of the row after this group's last
                     {
-                        const float4 c = agg_e[gl * 32 + sp];
+                        const float4 c = agg_e[gl * kPairs + sp];
                         x.re = pack2(c.x, c.y);
                         x.im = pack2(c.z, c.w);
                     }
 #pragma unroll
                     for (int gq = nsl - 2; gq >= 1; --gq) {
                         if (gq > sl && gq < gl) {
-                            const float4 c = agg_e[gq * 32 + sp];
+                            const float4 c = agg_e[gq * kPairs + sp];
                             const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
                             x = ((gflags >> gq) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
                         }
@@ -1504,7 +1532,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             if (seq_start && i == 0) {
                                 xp = xinit;
                             } else {
-                                const uint2 xh = xs[i * 32], xl = xs[(R + i) * 32];
+                                const uint2 xh = xs[i * kPairs], xl = xs[(R + i) * kPairs];
                                 xp.re = add2(pack2(__uint_as_float(xh.x << 16), __uint_as_float(xh.y << 16)),
                                              pack2(__uint_as_float(xl.x << 16), __uint_as_float(xl.y << 16)));
                                 xp.im = add2(pack2(__uint_as_float(xh.x & 0xffff0000u), __uint_as_float(xh.y & 0xffff0000u)),
@@ -1526,8 +1554,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         unpack2(lre, lr0, lr1);
                         unpack2(lim, li0, li1);
                         const __nv_bfloat162 l0 = __floats2bfloat162_rn(lr0, li0), l1 = __floats2bfloat162_rn(lr1, li1);
-                        xs[i * 32] = make_uint2(hb0, hb1);
-                        xs[(R + i) * 32] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+                        xs[i * kPairs] = make_uint2(hb0, hb1);
+                        xs[(R + i) * kPairs] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
                     }
                 };
                 if ((mask | mask0) == 0u)
@@ -1536,8 +1564,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     fold_rows(std::true_type{});
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0 && grp_valid) {
-                    tma_store_3d_nocommit(&tmS, smem_u32(warp_buf), n_tile * 64, m0 + r0, 0);
+                if (group_leader && grp_valid) {
+                    tma_store_3d_nocommit(&tmS, smem_u32(warp_buf), n_tile * kS, m0 + r0, 0);
                     tma_commit_group();
                 }
                 if (sl == g0) {   // x is s of the first row of the tile (of the sequence, when it lies inside the tile)
@@ -1568,14 +1596,14 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 float4 sum = agg_e[sp];
 #pragma unroll
                 for (int gq = 1; gq < nsl; ++gq) {
-                    const float4 c = agg_e[gq * 32 + sp];
+                    const float4 c = agg_e[gq * kPairs + sp];
                     sum.x += c.x, sum.y += c.y, sum.z += c.z, sum.w += c.w;
                 }
                 p.gA_part[(size_t)b * p.P + pg] = make_float2(sum.x, sum.z);
                 p.gA_part[(size_t)b * p.P + pg + 1] = make_float2(sum.y, sum.w);
             }
         }
-        if (lane == 0) tma_store_wait_all();
+        if (group_leader) tma_store_wait_all();
     }
     tc_fence_before();
     __syncwarp();
@@ -2012,84 +2040,108 @@ int launch_gemm_tc_tn(const GemmTcTN& g, cudaStream_t st) {
     return ok ? SSM_OK : SSM_ERR_CUDA;
 }
 
-// The two bf16 planes of a state tensor as [2, B*T, P] 32-bit words, in boxes of 64 states x kFsRows rows x both planes.
-static bool make_plane_map(CUtensorMap* map, const void* planes, int M, int P) {
+// The two bf16 planes of a state tensor as [2, B*T, P] 32-bit words, in boxes of `states` states x kFsRows rows x both planes.
+static bool make_plane_map(CUtensorMap* map, const void* planes, int M, int P, int states) {
     PFN_cuTensorMapEncodeTiled fn = tc::encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)M, 2};
     cuuint64_t strides[2] = {(cuuint64_t)P * 4, (cuuint64_t)M * P * 4};
-    cuuint32_t box[3] = {64, (cuuint32_t)tc::kFsRows, 2};
+    cuuint32_t box[3] = {(cuuint32_t)states, (cuuint32_t)tc::kFsRows, 2};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(planes), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Fewest (sequence, 64 states) chain pairs for which the kernels that scan in the epilogue of a projection
+// Fewest (sequence, state group) chain pairs for which the kernels that scan in the epilogue of a projection
 // are taken: below it too many CTA pairs would idle while a few walk their chains tile by tile.
 #ifndef SSM_FUSED_MIN_PAIRS
 #define SSM_FUSED_MIN_PAIRS 32   // measured: 32 pairs (16 sequences of 256 states) still beat the separate kernels
 #endif
-static int fused_min_pairs() { return SSM_FUSED_MIN_PAIRS; }
+#ifndef SSM_FUSED_NARROW_BELOW
+#define SSM_FUSED_NARROW_BELOW 0   // 0: chains of 32 states where chains of 64 would occupy at most half of the CTA pairs
+#endif
 
-// Chains per 64 states: the sequences, or, when a 128-row tile holds several whole sequences, the tiles.
+// Chains per state group: the sequences, or, when a 128-row tile holds several whole sequences, the tiles.
 static int fs_units(int B, int T) { return T >= tc::BM ? B : (B * T + tc::BM - 1) / tc::BM; }
 
-bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) {
+// States per chain of the kernels that scan in their epilogue for this problem: 64, 32 (few sequences: twice the
+// chains, half the tile), or 0 where those kernels are not taken.
+int tc_gemm_scan_group(int B, int T, int H, int P) {
     const bool t_ok = T % tc::BM == 0 || T == 16 || T == 32 || T == 64;
-    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return false;
-    return (2 * P / 128) * ((fs_units(B, T) + 1) / 2) >= fused_min_pairs();
+    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return 0;
+    const int pairs64 = (P / 64) * ((fs_units(B, T) + 1) / 2);
+    if (pairs64 < SSM_FUSED_MIN_PAIRS) return 0;
+    // A tile of 32 states takes about 0.8 of the time of a tile of 64 (measured), so halving the chains pays only
+    // where the second half of the CTA pairs would otherwise idle: 16 x 16384 at P = 256 1.88 -> 1.78 ms per step,
+    // 16 x 1024 0.242 -> 0.229; with 64 of 74 pairs busy (32 sequences) it costs 30 - 50 % in these kernels.
+    const int narrow_below = SSM_FUSED_NARROW_BELOW > 0 ? SSM_FUSED_NARROW_BELOW : tc::sm_count() / 4 + 1;
+    return pairs64 < narrow_below ? 32 : 64;
+}
+bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) { return tc_gemm_scan_group(B, T, H, P) != 0; }
+bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) { return tc_gemm_scan_group(B, T, H, P) != 0; }
+
+template <int kS>
+static int launch_gemm_scan_fwd_s(const GemmScanFwd& g, cudaStream_t st) {
+    using namespace tc;
+    using Cfg = FsCfg<kS>;
+    const int M = g.B * g.T;
+    CUtensorMap ma, mw, mx;
+    if (!make_map(&ma, g.u, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
+    if (!make_map(&mw, g.Wsplit, (uint64_t)4 * g.P, (uint64_t)g.H, BK, Cfg::kWRows)) return SSM_ERR_CUDA;
+    if (!make_plane_map(&mx, g.x_planes, M, g.P, kS)) return SSM_ERR_CUDA;
+    const int units = fs_units(g.B, g.T), n_tiles = g.P / kS;
+    FsParams p{g.B, g.T, g.P, n_tiles, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
+               g.T >= BM ? BM / kFsRows : g.T / kFsRows, n_tiles * ((units + 1) / 2),
+               g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr};
+    count_launch();
+    auto kern = gemm_scan_fwd_kernel<kS>;
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SSM_ERR_CUDA;
+    const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes, Cfg::kThreads);
+    if (pairs <= 0) return SSM_ERR_CUDA;
+    kern<<<2 * min(pairs, p.nchains), Cfg::kThreads, Cfg::kSmemBytes, st>>>(ma, mw, mx, p);
+    return SSM_OK;
 }
 
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
-    using namespace tc;
-    if (!tc_gemm_scan_fwd_supported(g.B, g.T, g.H, g.P)) return SSM_ERR_SHAPE;
-    const int M = g.B * g.T, P2 = 2 * g.P;
-    CUtensorMap ma, mw, mx;
-    if (!make_map(&ma, g.u, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
-    if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
-    if (!make_plane_map(&mx, g.x_planes, M, g.P)) return SSM_ERR_CUDA;
-    const int units = fs_units(g.B, g.T);
-    FsParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
-               g.T >= BM ? BM / kFsRows : g.T / kFsRows, (P2 / 128) * ((units + 1) / 2),
-               g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr};
-    count_launch();
-    auto kern = gemm_scan_fwd_kernel;
-    if (!set_smem(kern, kFsSmemBytes)) return SSM_ERR_CUDA;
-    const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), kFsSmemBytes, kFsThreads);
-    if (pairs <= 0) return SSM_ERR_CUDA;
-    kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, mx, p);
-    return SSM_OK;
+    switch (tc_gemm_scan_group(g.B, g.T, g.H, g.P)) {
+        case 64: return launch_gemm_scan_fwd_s<64>(g, st);
+        case 32: return launch_gemm_scan_fwd_s<32>(g, st);
+        default: return SSM_ERR_SHAPE;
+    }
 }
 
-bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) {
-    const bool t_ok = T % tc::BM == 0 || T == 16 || T == 32 || T == 64;
-    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return false;
-    return (2 * P / 128) * ((fs_units(B, T) + 1) / 2) >= fused_min_pairs();
-}
-
-// Rows of gA_part that launch_gemm_scan_bwd writes: one per chain of 64 states.
+// Rows of gA_part that launch_gemm_scan_bwd writes: one per chain of a state group.
 int tc_gemm_scan_bwd_part_rows(int B, int T) { return fs_units(B, T); }
 
-int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {
+template <int kS>
+static int launch_gemm_scan_bwd_s(const GemmScanBwd& g, cudaStream_t st) {
     using namespace tc;
-    if (!tc_gemm_scan_bwd_supported(g.B, g.T, g.H, g.P)) return SSM_ERR_SHAPE;
-    const int M = g.B * g.T, P2 = 2 * g.P;
+    using Cfg = FsCfg<kS>;
+    const int M = g.B * g.T;
     CUtensorMap ma, mw, mx, ms;
     if (!make_map(&ma, g.gy, (uint64_t)M, (uint64_t)g.H, BK, BM)) return SSM_ERR_CUDA;
-    if (!make_map(&mw, g.Wsplit, (uint64_t)(P2 / 128) * BN, (uint64_t)g.H, BK, BN / 2)) return SSM_ERR_CUDA;
-    if (!make_plane_map(&mx, g.x_planes, M, g.P) || !make_plane_map(&ms, g.s_planes, M, g.P)) return SSM_ERR_CUDA;
-    const int units = fs_units(g.B, g.T);
-    FbParams p{g.B, g.T, g.P, P2 / 128, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
-               g.T >= BM ? BM / kFsRows : g.T / kFsRows, (P2 / 128) * ((units + 1) / 2),
+    if (!make_map(&mw, g.Wsplit, (uint64_t)4 * g.P, (uint64_t)g.H, BK, Cfg::kWRows)) return SSM_ERR_CUDA;
+    if (!make_plane_map(&mx, g.x_planes, M, g.P, kS) || !make_plane_map(&ms, g.s_planes, M, g.P, kS)) return SSM_ERR_CUDA;
+    const int units = fs_units(g.B, g.T), n_tiles = g.P / kS;
+    FbParams p{g.B, g.T, g.P, n_tiles, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
+               g.T >= BM ? BM / kFsRows : g.T / kFsRows, n_tiles * ((units + 1) / 2),
                g.Abar, g.done, g.x0, g.gxT, g.gA_part, g.gx0, g.hdr};
     count_launch();
-    auto kern = gemm_scan_bwd_kernel;
-    if (!set_smem(kern, kFsSmemBytes)) return SSM_ERR_CUDA;
-    const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), kFsSmemBytes, kFsThreads);
+    auto kern = gemm_scan_bwd_kernel<kS>;
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SSM_ERR_CUDA;
+    const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes, Cfg::kThreads);
     if (pairs <= 0) return SSM_ERR_CUDA;
-    kern<<<2 * min(pairs, p.nchains), kFsThreads, kFsSmemBytes, st>>>(ma, mw, mx, ms, p);
+    kern<<<2 * min(pairs, p.nchains), Cfg::kThreads, Cfg::kSmemBytes, st>>>(ma, mw, mx, ms, p);
     return SSM_OK;
+}
+
+int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {
+    switch (tc_gemm_scan_group(g.B, g.T, g.H, g.P)) {
+        case 64: return launch_gemm_scan_bwd_s<64>(g, st);
+        case 32: return launch_gemm_scan_bwd_s<32>(g, st);
+        default: return SSM_ERR_SHAPE;
+    }
 }
 
 bool tc_nt_supported(int I, int J) { return (I % tc::BM) == 0 && (J % (tc::BN / 2)) == 0; }

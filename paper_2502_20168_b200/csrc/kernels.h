@@ -138,6 +138,9 @@ struct GemmScanFwd {
     WsHeader* hdr;
 };
 bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P);
+// States per chain these kernels (forward and backward alike) use for a problem: 64 or 32; 0: not taken.  The
+// hi/lo stacked operands they read are packed for that group size (launch_discretize_pack_tc).
+int tc_gemm_scan_group(int B, int T, int H, int P);
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st);
 
 // g_x projection and reverse scan fused (gemm_tc.cu): s = reverse scan(gy conj(C)) written as the two
@@ -187,7 +190,10 @@ int launch_gemm_tc_nt(const GemmTcNT& g, cudaStream_t st);
 // discretize.cu: operands of the tensor-core path (bf16).  Wsplit_B / Wsplit_C: [4P, H] hi/lo
 // stacked forms of Bp / Cq (see GemmTcTN);  Cp, Bq: [H, 2P] single bf16.
 // Discretisation and packing of the four bf16 operands in one kernel.
-void launch_discretize_pack_tc(int H, int P, bool pair_cols_B, bool pair_cols_C, const float2* Lambda, const float* Delta,
+// group_B / group_C: 0 = rows in the plain order (2p + c, hi/lo stacked per 128 rows: GemmTcTN with split_w), or the
+// states per chain (64, 32) of the kernels that scan in their epilogue: rows of two neighbouring states interleaved
+// as (re, re, im, im) inside groups of that many states, hi/lo stacked per group.
+void launch_discretize_pack_tc(int H, int P, int group_B, int group_C, const float2* Lambda, const float* Delta,
                                const float2* Bc, const float2* Cc, float2* Abar, float2* Abar_lo, float2* Bbar,
                                void* Wsplit_B, void* Wsplit_C, void* Cp, void* Bq, cudaStream_t st);
 

@@ -71,7 +71,9 @@ def test_plane_path_shapes_fp32(B, T, H, P):
 
 
 @pytest.mark.parametrize("B,T,H,P", [(81, 128, 256, 128), (150, 256, 256, 64), (76, 384, 512, 128),
-                                     (301, 64, 256, 128), (601, 32, 256, 128), (2403, 16, 256, 64)])
+                                     (301, 64, 256, 128), (601, 32, 256, 128), (2403, 16, 256, 64),
+                                     # chains of 64 states would occupy at most half of the CTA pairs: chains of 32 states
+                                     (17, 256, 256, 256), (33, 64, 256, 256), (130, 16, 256, 256), (33, 128, 512, 128)])
 def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
     # Enough (sequence, 64 states) chains and T a multiple of 128, or T = 16, 32, 64 (a 128-row tile
     # then holds whole sequences; odd B leaves the last tile ragged): the input projection and the
