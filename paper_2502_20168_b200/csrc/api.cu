@@ -82,7 +82,7 @@ LayerPlan plan_layer(const ssm_shape& s, bool allow_tc = true) {
     }
     p.gAbar = take(off, (size_t)s.P * 8);
     p.gBbar = take(off, PH * 8);
-    p.scan = take(off, scan_scratch_bytes(s.B, s.T, s.P));
+    p.scan = take(off, scan_scratch_bytes(s.B, s.T, s.P, 2));
     p.part = take(off, (size_t)2 * p.splits * 2 * PH * 4);   // split-K partials of gBbar, then those of dC
     {   // dD: partial column sums of gy * u, from the stand-alone kernel or from the epilogue of the du projection
         const size_t rows = (size_t)tc_tn_dot_max_rows();

@@ -110,6 +110,34 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// For data handed from one CTA of the cluster to the other through shared memory: the sender stores into the
+// peer's memory and arrives (release, cluster scope) on the peer's barrier, the receiver waits with acquire.
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_acquire_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_acquire_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait_acquire_cluster(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void st_cluster_f4(uint32_t cluster_addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -853,7 +881,7 @@ __device__ __forceinline__ C2 cstep2(f32x2 ar, f32x2 ai, f32x2 nai, C2 x, C2 b) 
 template <int kThreadsN>
 __device__ __forceinline__ void epi_sync_n() { asm volatile("bar.sync 1, %0;" ::"n"(kThreadsN) : "memory"); }
 
-template <int kS>
+template <int kS, bool kTPair>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FsCfg<kS>::kThreads, 1)
 gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
                      const __grid_constant__ CUtensorMap tmX, FsParams p) {
@@ -864,6 +892,9 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     __shared__ float4 agg_e[kFsEpiThreads], carry_s[kPairs];   // (re, re, im, im) of two neighbouring states
     __shared__ uint32_t masks[4];
+    __shared__ float4 carry_ring[2][kTPair ? kPairs : 1];   // kTPair: the state handed over by the peer CTA, two slots in turn
+    __shared__ __align__(8) uint64_t carry_bar[2];           // kTPair: slot i has arrived (one arrival per sending thread)
+    static_assert(!kTPair || kPairs == 32, "the last row group of a tile is one warp");
     const Smem s = carve_smem(smem_raw, kPairStages, Cfg::kTileBytes, 0, kStageB, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -875,6 +906,7 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int i = 0; i < 2; ++i) {
             mbar_init(s.tmem_full(i), 1);
             mbar_init(s.tmem_empty(i), 2 * kFsEpiThreads);
+            mbar_init(smem_u32(&carry_bar[i]), kPairs);
         }
         *s.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -891,9 +923,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int M = p.B * p.T;
     // chain -> (64 states, this CTA's sequence or, for short sequences, tile of rows); tile tb of a chain -> first row
-    auto seq_of = [&](int chain) { return 2 * (chain / p.n_tiles) + (int)rank; };
+    // kTPair: both CTAs of the pair walk ONE sequence, tile 2 tb on CTA 0 and tile 2 tb + 1 on CTA 1.
+    auto seq_of = [&](int chain) { return kTPair ? chain / p.n_tiles : 2 * (chain / p.n_tiles) + (int)rank; };
     auto row_of = [&](int chain, int tb) {
         const int b = seq_of(chain);
+        if (kTPair) return b * p.unit_rows + (2 * tb + (int)rank) * BM;
         return b < p.n_units ? b * p.unit_rows + tb * BM : M;   // nothing left for this CTA: rows past the end read as zero
     };
 
@@ -969,17 +1003,21 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const C2 zero = {0ull, 0ull};
         int acc = 0;
         uint32_t acc_phase = 0;
+        uint32_t n_recv = 0, n_send = 0;            // kTPair: states received from / handed to the peer so far
+        const uint32_t peer_ring = map_to_cta(smem_u32(&carry_ring[0][0]), rank ^ 1u);
+        const uint32_t peer_bar = map_to_cta(smem_u32(&carry_bar[0]), rank ^ 1u);
         bool ok = true;
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
             const bool has_seq = b < p.n_units;
-            const bool short_seq = p.T < BM;        // then b counts tiles of rows, not sequences
+            const bool short_seq = !kTPair && p.T < BM;        // then b counts tiles of rows, not sequences
             const int g0 = sl - sl % p.gps;         // the first row group of this group's sequence in the tile
-            const bool from_carry = sl == g0;
+            const bool from_carry = !kTPair && sl == g0;   // (kTPair: the carried state arrives late; every group joins)
             const int pg = n_tile * kS + 2 * sp;    // the first of this thread's two states
             const float2 a0 = p.Abar[pg], a1 = p.Abar[pg + 1];
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
             f32x2 pr, pi, npi;   // Abar^R by squaring in fp32 (a few 1e-7 relative: the results leave as bf16 pairs)
+            f32x2 tr = 0ull, ti = 0ull, nti = 0ull;
             {
                 float re0 = a0.x, im0 = a0.y, re1 = a1.x, im1 = a1.y;
 #pragma unroll
@@ -991,8 +1029,25 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 pr = pack2(re0, re1);
                 pi = pack2(im0, im1);
                 npi = pack2(-im0, -im1);
+                if (kTPair) {   // Abar^128: what a tile without flags does to the state that enters it
+#pragma unroll
+                    for (int n = R; n < BM; n *= 2) {
+                        const float r0 = fmaf(re0, re0, -im0 * im0), i0 = 2.f * re0 * im0;
+                        const float r1 = fmaf(re1, re1, -im1 * im1), i1 = 2.f * re1 * im1;
+                        re0 = r0, im0 = i0, re1 = r1, im1 = i1;
+                    }
+                    tr = pack2(re0, re1);
+                    ti = pack2(im0, im1);
+                    nti = pack2(-im0, -im1);
+                }
             }
-            if (sl == 0 && !short_seq) {   // the carried state, as (re, re, im, im) of the two states
+            C2 cin = zero;      // kTPair: the state that enters this CTA's tile
+            if (kTPair && rank == 0 && p.x0) {
+                const float2 c0 = p.x0[(size_t)b * p.P + pg], c1 = p.x0[(size_t)b * p.P + pg + 1];
+                cin.re = pack2(c0.x, c1.x);
+                cin.im = pack2(c0.y, c1.y);
+            }
+            if (sl == 0 && !short_seq && !kTPair) {   // the carried state, as (re, re, im, im) of the two states
                 float2 c0 = make_float2(0.f, 0.f), c1 = c0;
                 if (p.x0 && has_seq) {
                     c0 = p.x0[(size_t)b * p.P + pg];
@@ -1101,7 +1156,48 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 epi_sync();   // group results visible; every thread has its rows in registers
                 C2 x = e;
-                if (!from_carry) {   // state before this group's first row
+                if (kTPair) {
+                    // The state that enters the tile comes from the peer CTA (the tile before this one), except for
+                    // the sequence's first tile.  The last row group passes the tile's end state on as soon as it
+                    // can: the tile's own contribution (the groups' results joined from zero) is ready before the
+                    // peer's state arrives, so the hand-over costs one multiply-add per tile and CTA.
+                    const bool first = rank == 0 && tb == 0, last = rank == 1 && tb == p.tblocks - 1;
+                    C2 tile = zero;
+                    if (sl == nsl - 1 && !last) {
+#pragma unroll
+                        for (int g = 0; g < nsl - 1; ++g) {
+                            const float4 c = agg_e[g * kPairs + sp];
+                            const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                            tile = (g == 0 || ((gflags >> g) & 1u)) ? eg : cstep2(pr, pi, npi, tile, eg);
+                        }
+                        tile = ((gflags >> (nsl - 1)) & 1u) ? e : cstep2(pr, pi, npi, tile, e);
+                    }
+                    if (!first) {
+                        (void)mbar_wait_acquire_cluster(smem_u32(&carry_bar[n_recv & 1u]), (n_recv >> 1) & 1u, s.abort_flag);
+                        const float4 c = carry_ring[n_recv & 1u][sp];
+                        cin.re = pack2(c.x, c.y);
+                        cin.im = pack2(c.z, c.w);
+                        ++n_recv;
+                    }
+                    if (sl == nsl - 1 && !last) {
+                        const C2 out = gflags == 0u ? cstep2(tr, ti, nti, cin, tile) : tile;
+                        float o0, o1, o2, o3;
+                        unpack2(out.re, o0, o1);
+                        unpack2(out.im, o2, o3);
+                        st_cluster_f4(peer_ring + (uint32_t)(((n_send & 1u) * kPairs + sp) * sizeof(float4)), make_float4(o0, o1, o2, o3));
+                        mbar_arrive_release_cluster(peer_bar + 8u * (n_send & 1u));
+                        ++n_send;
+                    }
+                    x = cin;
+#pragma unroll
+                    for (int g = 0; g < nsl - 1; ++g) {
+                        if (g < sl) {
+                            const float4 c = agg_e[g * kPairs + sp];
+                            const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                            x = ((gflags >> g) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
+                        }
+                    }
+                } else if (!from_carry) {   // state before this group's first row
                     {
                         const float4 c = agg_e[g0 * kPairs + sp];
                         x.re = pack2(c.x, c.y);
@@ -1155,7 +1251,12 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     unpack2(x.re, x0r, x1r);
                     unpack2(x.im, x0i, x1i);
                     // (not after the chain's last tile: by then the first group may already have set up the next chain)
-                    if (!short_seq && tb < p.tblocks - 1) {
+                    if (kTPair) {
+                        if (rank == 1 && tb == p.tblocks - 1 && p.xT) {
+                            p.xT[(size_t)b * p.P + pg] = make_float2(x0r, x0i);
+                            p.xT[(size_t)b * p.P + pg + 1] = make_float2(x1r, x1i);
+                        }
+                    } else if (!short_seq && tb < p.tblocks - 1) {
                         carry_s[sp] = make_float4(x0r, x1r, x0i, x1i);
                     } else if (p.xT && grp_valid) {
                         p.xT[(size_t)b_grp * p.P + pg] = make_float2(x0r, x0i);
@@ -1207,7 +1308,7 @@ struct FbParams {
     WsHeader* hdr;
 };
 
-template <int kS>
+template <int kS, bool kTPair>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FsCfg<kS>::kThreads, 1)
 gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
                      const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmS, FbParams p) {
@@ -1219,6 +1320,9 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     __shared__ float4 agg_e[kFsEpiThreads], carry_s[kPairs];   // (re, re, im, im) of two neighbouring states
     __shared__ uint32_t masks[8];   // [0, 4): flags of the rows one later (the resets of the reverse scan); [4, 8): of the rows
     __shared__ __align__(8) uint64_t xbar[BM / kFsRows];   // one per row group: its rows of x have arrived
+    __shared__ float4 carry_ring[2][kTPair ? kPairs : 1];   // kTPair: the value handed over by the peer CTA, two slots in turn
+    __shared__ __align__(8) uint64_t carry_bar[2];           // kTPair: slot i has arrived (one arrival per sending thread)
+    static_assert(!kTPair || kPairs == 32, "the first row group of a tile is one warp");
     const Smem s = carve_smem(smem_raw, kPairStages, Cfg::kTileBytes, 0, kStageB, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -1230,6 +1334,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int i = 0; i < 2; ++i) {
             mbar_init(s.tmem_full(i), 1);
             mbar_init(s.tmem_empty(i), 2 * kFsEpiThreads);
+            mbar_init(smem_u32(&carry_bar[i]), kPairs);
         }
         for (int i = 0; i < BM / kFsRows; ++i) mbar_init(smem_u32(&xbar[i]), 1);
         *s.abort_flag = 0;
@@ -1246,9 +1351,11 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int M = p.B * p.T;
-    auto seq_of = [&](int chain) { return 2 * (chain / p.n_tiles) + (int)rank; };
+    // kTPair: both CTAs of the pair walk ONE sequence, tile 2 tb on CTA 0 and tile 2 tb + 1 on CTA 1.
+    auto seq_of = [&](int chain) { return kTPair ? chain / p.n_tiles : 2 * (chain / p.n_tiles) + (int)rank; };
     auto row_of = [&](int chain, int tb) {
         const int b = seq_of(chain);
+        if (kTPair) return b * p.unit_rows + (2 * tb + (int)rank) * BM;
         return b < p.n_units ? b * p.unit_rows + tb * BM : M;   // nothing for this CTA: rows past the end read as zero
     };
 
@@ -1319,10 +1426,13 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const int sp = te % kPairs, sl = te / kPairs;   // scan role: pair of states of the tile, group of its rows
         const bool group_leader = lane % kPairs == 0;   // the lane that talks to the TMA unit for its row group
         const int prow = q * 32 + lane;             // drain role: row of the tile
-        const bool short_seq = p.T < BM;            // then a chain is one tile of 128 / T whole sequences
+        const bool short_seq = !kTPair && p.T < BM;            // then a chain is one tile of 128 / T whole sequences
         const int g0 = sl - sl % p.gps;             // first and last row group of this group's sequence in the tile
         const int gl = g0 + p.gps - 1;
-        const bool from_carry = sl == gl;           // the last rows come first
+        const bool from_carry = !kTPair && sl == gl;           // the last rows come first (kTPair: the carried value arrives late; every group joins)
+        uint32_t n_recv = 0, n_send = 0;            // kTPair: values received from / handed to the peer so far
+        const uint32_t peer_ring = map_to_cta(smem_u32(&carry_ring[0][0]), rank ^ 1u);
+        const uint32_t peer_bar = map_to_cta(smem_u32(&carry_bar[0]), rank ^ 1u);
         float4* T4 = reinterpret_cast<float4*>(s.staging);
         uint8_t* warp_buf = s.staging + sl * Cfg::kGroupBytes;   // this row group's rows of the tile; later x_{t-1}, then s
         uint2* xs = reinterpret_cast<uint2*>(warp_buf) + sp;
@@ -1339,6 +1449,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const float2 a0 = cconj(p.Abar[pg]), a1 = cconj(p.Abar[pg + 1]);
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
             f32x2 pr, pi, npi;   // conj(Abar)^R by squaring in fp32
+            f32x2 tr = 0ull, ti = 0ull, nti = 0ull;
             {
                 float re0 = a0.x, im0 = a0.y, re1 = a1.x, im1 = a1.y;
 #pragma unroll
@@ -1350,11 +1461,23 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 pr = pack2(re0, re1);
                 pi = pack2(im0, im1);
                 npi = pack2(-im0, -im1);
+                if (kTPair) {   // conj(Abar)^128: what a tile without flags does to the value that enters it
+#pragma unroll
+                    for (int n = R; n < BM; n *= 2) {
+                        const float r0 = fmaf(re0, re0, -im0 * im0), i0 = 2.f * re0 * im0;
+                        const float r1 = fmaf(re1, re1, -im1 * im1), i1 = 2.f * re1 * im1;
+                        re0 = r0, im0 = i0, re1 = r1, im1 = i1;
+                    }
+                    tr = pack2(re0, re1);
+                    ti = pack2(im0, im1);
+                    nti = pack2(-im0, -im1);
+                }
             }
+            C2 cin = zero;      // kTPair: s of the row after this CTA's tile (nothing after the sequence's last row)
             C2 g = zero;        // this thread's part of the chain's sums s_t conj(x_{t-1})
             f32x2 gim_neg = 0ull;   // the part of Im g that enters with a minus sign, summed apart
             C2 xinit = zero;    // x0: what stands before the sequence's first row
-            if (!short_seq && sl == 0 && p.x0 && has_seq) {
+            if (!short_seq && sl == 0 && p.x0 && has_seq && (!kTPair || rank == 0)) {
                 const float2 c0 = p.x0[(size_t)b * p.P + pg], c1 = p.x0[(size_t)b * p.P + pg + 1];
                 xinit.re = pack2(c0.x, c1.x);
                 xinit.im = pack2(c0.y, c1.y);
@@ -1364,7 +1487,8 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 const int m0 = row_of(chain, tb);
                 if (p.done && te < BM) {
                     // a row's own flag, and the flag of the row after it if that row belongs to the same sequence
-                    const bool next_in_seq = short_seq ? ((te + 1) % p.T != 0 && m0 + te + 1 < M) : (tb * BM + te + 1 < p.T);
+                    const int tix = kTPair ? 2 * tb + (int)rank : tb;   // this tile's place in its sequence
+                    const bool next_in_seq = short_seq ? ((te + 1) % p.T != 0 && m0 + te + 1 < M) : (tix * BM + te + 1 < p.T);
                     const bool f0 = has_seq && m0 + te < M && p.done[(size_t)m0 + te] != 0;
                     const bool f1 = has_seq && next_in_seq && p.done[(size_t)m0 + te + 1] != 0;
                     const uint32_t mk0 = __ballot_sync(0xffffffffu, f0), mk1 = __ballot_sync(0xffffffffu, f1);
@@ -1438,7 +1562,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     v[i].re = pack2(t.x, t.y);
                     v[i].im = pack2(t.z, t.w);
                 }
-                if (from_carry && tb == p.tblocks - 1 && p.gxT && grp_valid) {   // the gradient of the final state
+                if (sl == gl && tb == p.tblocks - 1 && (!kTPair || rank == 1) && p.gxT && grp_valid) {   // the gradient of the final state
                     const float2 c0 = p.gxT[(size_t)b_grp * p.P + pg], c1 = p.gxT[(size_t)b_grp * p.P + pg + 1];
                     float v0, v1, v2, v3;
                     unpack2(v[R - 1].re, v0, v1);
@@ -1453,7 +1577,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     mbar_expect_tx(xb, Cfg::kGroupBytes);
                     tma_load_3d(smem_u32(warp_buf), &tmX, xb, n_tile * kS, m0 + r0 - 1, 0);
                     // and the same rows of the tile before this one into L2, where the next load will find them
-                    if (tb > 0) tma_prefetch_3d(&tmX, n_tile * kS, m0 - BM + r0 - 1, 0);
+                    if (tb > 0) tma_prefetch_3d(&tmX, n_tile * kS, m0 - (kTPair ? 2 : 1) * BM + r0 - 1, 0);
                 }
                 C2 e = zero;
                 if (from_carry) {   // from the carried value (nothing, for a sequence inside the tile): these results are final
@@ -1488,7 +1612,50 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 epi_sync();   // group results visible
                 C2 x = e;
-                if (!from_carry) {   // s of the row after this group's last
+                if (kTPair) {
+                    // The value that enters the tile (s of the row after it) comes from the peer CTA, which holds the
+                    // tile after this one, except for the sequence's last tile.  The first row group passes s of the
+                    // tile's first row on as soon as it can: the tile's own contribution (the groups' results joined
+                    // from zero) is ready before the peer's value arrives.
+                    const bool first = rank == 1 && tb == p.tblocks - 1, last = rank == 0 && tb == 0;
+                    C2 tile = zero;
+                    if (sl == 0 && !last) {
+#pragma unroll
+                        for (int gq = nsl - 1; gq >= 1; --gq) {
+                            const float4 c = agg_e[gq * kPairs + sp];
+                            const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                            tile = (gq == nsl - 1 || ((gflags >> gq) & 1u)) ? eg : cstep2(pr, pi, npi, tile, eg);
+                        }
+                        tile = (gflags & 1u) ? e : cstep2(pr, pi, npi, tile, e);
+                    }
+                    if (!first) {
+                        (void)mbar_wait_acquire_cluster(smem_u32(&carry_bar[n_recv & 1u]), (n_recv >> 1) & 1u, s.abort_flag);
+                        const float4 c = carry_ring[n_recv & 1u][sp];
+                        cin.re = pack2(c.x, c.y);
+                        cin.im = pack2(c.z, c.w);
+                        ++n_recv;
+                    } else {
+                        cin = zero;
+                    }
+                    if (sl == 0 && !last) {
+                        const C2 out = gflags == 0u ? cstep2(tr, ti, nti, cin, tile) : tile;
+                        float o0, o1, o2, o3;
+                        unpack2(out.re, o0, o1);
+                        unpack2(out.im, o2, o3);
+                        st_cluster_f4(peer_ring + (uint32_t)(((n_send & 1u) * kPairs + sp) * sizeof(float4)), make_float4(o0, o1, o2, o3));
+                        mbar_arrive_release_cluster(peer_bar + 8u * (n_send & 1u));
+                        ++n_send;
+                    }
+                    x = cin;
+#pragma unroll
+                    for (int gq = nsl - 1; gq >= 1; --gq) {
+                        if (gq > sl) {
+                            const float4 c = agg_e[gq * kPairs + sp];
+                            const C2 eg = {pack2(c.x, c.y), pack2(c.z, c.w)};
+                            x = ((gflags >> gq) & 1u) ? eg : cstep2(pr, pi, npi, x, eg);
+                        }
+                    }
+                } else if (!from_carry) {   // s of the row after this group's last
                     {
                         const float4 c = agg_e[gl * kPairs + sp];
                         x.re = pack2(c.x, c.y);
@@ -1508,7 +1675,7 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     // (the wait gave up: the flag is set, everybody leaves at the next barrier)
                 }
                 xphase ^= 1u;
-                const bool seq_start = tb == 0 && sl == g0;   // row 0 of this group is the sequence's first row
+                const bool seq_start = tb == 0 && sl == g0 && (!kTPair || rank == 0);   // row 0 of this group is the sequence's first row
                 if (short_seq && seq_start) {                // the state before that row: this sequence's x0
                     xinit = zero;
                     if (p.x0 && grp_valid) {
@@ -1572,7 +1739,9 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     float x0r, x1r, x0i, x1i;
                     unpack2(x.re, x0r, x1r);
                     unpack2(x.im, x0i, x1i);
-                    if (tb > 0) {
+                    if (kTPair && !(rank == 0 && tb == 0)) {
+                        // (handed to the peer above)
+                    } else if (tb > 0) {
                         carry_s[sp] = make_float4(x0r, x1r, x0i, x1i);
                     } else if (p.gx0 && grp_valid) {   // what reaches the initial state: keep_0 conj(Abar) s_0
                         const bool cut = (mask0 & 1u) != 0u;
@@ -1599,8 +1768,9 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const float4 c = agg_e[gq * kPairs + sp];
                     sum.x += c.x, sum.y += c.y, sum.z += c.z, sum.w += c.w;
                 }
-                p.gA_part[(size_t)b * p.P + pg] = make_float2(sum.x, sum.z);
-                p.gA_part[(size_t)b * p.P + pg + 1] = make_float2(sum.y, sum.w);
+                const size_t part_row = kTPair ? 2 * (size_t)b + rank : (size_t)b;   // kTPair: each CTA has half of the sequence's rows
+                p.gA_part[part_row * p.P + pg] = make_float2(sum.x, sum.z);
+                p.gA_part[part_row * p.P + pg + 1] = make_float2(sum.y, sum.w);
             }
         }
         if (group_leader) tma_store_wait_all();
@@ -2065,23 +2235,36 @@ static bool make_plane_map(CUtensorMap* map, const void* planes, int M, int P, i
 // Chains per state group: the sequences, or, when a 128-row tile holds several whole sequences, the tiles.
 static int fs_units(int B, int T) { return T >= tc::BM ? B : (B * T + tc::BM - 1) / tc::BM; }
 
-// States per chain of the kernels that scan in their epilogue for this problem: 64, 32 (few sequences: twice the
-// chains, half the tile), or 0 where those kernels are not taken.
-int tc_gemm_scan_group(int B, int T, int H, int P) {
+// How the kernels that scan in their epilogue take a problem: chains of 64 states, of 32 (few sequences: twice
+// the chains, half the tile), or not at all (group 0); and, for few long sequences, both CTAs of a pair on one
+// sequence (time pairs: CTA 0 has the even tiles, CTA 1 the odd ones, the state passes from one to the other
+// through shared memory), which doubles the chains without halving the tile.
+#ifndef SSM_FUSED_TIME_PAIRS
+#define SSM_FUSED_TIME_PAIRS 1
+#endif
+struct FusedMode {
+    int group;
+    bool time_pairs;
+};
+static FusedMode fused_mode(int B, int T, int H, int P) {
     const bool t_ok = T % tc::BM == 0 || T == 16 || T == 32 || T == 64;
-    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return 0;
+    if (!t_ok || H % tc::BK != 0 || P % 64 != 0) return {0, false};
     const int pairs64 = (P / 64) * ((fs_units(B, T) + 1) / 2);
-    if (pairs64 < SSM_FUSED_MIN_PAIRS) return 0;
     // A tile of 32 states takes about 0.8 of the time of a tile of 64 (measured), so halving the chains pays only
     // where the second half of the CTA pairs would otherwise idle: 16 x 16384 at P = 256 1.88 -> 1.78 ms per step,
     // 16 x 1024 0.242 -> 0.229; with 64 of 74 pairs busy (32 sequences) it costs 30 - 50 % in these kernels.
+    // Time pairs double the chains at the full tile: 16 x 16384 1.76 -> 1.48 ms, 16 x 1024 0.228 -> 0.212.
     const int narrow_below = SSM_FUSED_NARROW_BELOW > 0 ? SSM_FUSED_NARROW_BELOW : tc::sm_count() / 4 + 1;
-    return pairs64 < narrow_below ? 32 : 64;
+    if (pairs64 >= narrow_below) return {64, false};
+    if (SSM_FUSED_TIME_PAIRS && T % (2 * tc::BM) == 0 && (P / 64) * B >= SSM_FUSED_MIN_PAIRS) return {64, true};
+    if (pairs64 < SSM_FUSED_MIN_PAIRS) return {0, false};
+    return {32, false};
 }
+int tc_gemm_scan_group(int B, int T, int H, int P) { return fused_mode(B, T, H, P).group; }
 bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) { return tc_gemm_scan_group(B, T, H, P) != 0; }
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) { return tc_gemm_scan_group(B, T, H, P) != 0; }
 
-template <int kS>
+template <int kS, bool kTPair>
 static int launch_gemm_scan_fwd_s(const GemmScanFwd& g, cudaStream_t st) {
     using namespace tc;
     using Cfg = FsCfg<kS>;
@@ -2094,8 +2277,12 @@ static int launch_gemm_scan_fwd_s(const GemmScanFwd& g, cudaStream_t st) {
     FsParams p{g.B, g.T, g.P, n_tiles, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
                g.T >= BM ? BM / kFsRows : g.T / kFsRows, n_tiles * ((units + 1) / 2),
                g.Abar, g.done, g.x0, g.xT, (uint32_t*)g.x_planes, (size_t)M * g.P, g.hdr};
+    if (kTPair) {   // a chain is one sequence; each CTA has every other tile
+        p.tblocks = g.T / (2 * BM);
+        p.nchains = n_tiles * g.B;
+    }
     count_launch();
-    auto kern = gemm_scan_fwd_kernel<kS>;
+    auto kern = gemm_scan_fwd_kernel<kS, kTPair>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SSM_ERR_CUDA;
     const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes, Cfg::kThreads);
     if (pairs <= 0) return SSM_ERR_CUDA;
@@ -2104,17 +2291,19 @@ static int launch_gemm_scan_fwd_s(const GemmScanFwd& g, cudaStream_t st) {
 }
 
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st) {
-    switch (tc_gemm_scan_group(g.B, g.T, g.H, g.P)) {
-        case 64: return launch_gemm_scan_fwd_s<64>(g, st);
-        case 32: return launch_gemm_scan_fwd_s<32>(g, st);
-        default: return SSM_ERR_SHAPE;
-    }
+    const FusedMode m = fused_mode(g.B, g.T, g.H, g.P);
+    if (m.group == 64) return m.time_pairs ? launch_gemm_scan_fwd_s<64, true>(g, st) : launch_gemm_scan_fwd_s<64, false>(g, st);
+    if (m.group == 32) return launch_gemm_scan_fwd_s<32, false>(g, st);
+    return SSM_ERR_SHAPE;
 }
 
-// Rows of gA_part that launch_gemm_scan_bwd writes: one per chain of a state group.
-int tc_gemm_scan_bwd_part_rows(int B, int T) { return fs_units(B, T); }
+// Rows of gA_part that launch_gemm_scan_bwd writes: one per chain of a state group (two per sequence where both
+// CTAs of a pair share a sequence).
+int tc_gemm_scan_bwd_part_rows(int B, int T, int H, int P) {
+    return fused_mode(B, T, H, P).time_pairs ? 2 * B : fs_units(B, T);
+}
 
-template <int kS>
+template <int kS, bool kTPair>
 static int launch_gemm_scan_bwd_s(const GemmScanBwd& g, cudaStream_t st) {
     using namespace tc;
     using Cfg = FsCfg<kS>;
@@ -2127,8 +2316,12 @@ static int launch_gemm_scan_bwd_s(const GemmScanBwd& g, cudaStream_t st) {
     FbParams p{g.B, g.T, g.P, n_tiles, g.H / BK, g.T >= BM ? g.T / BM : 1, g.T >= BM ? g.T : BM, units,
                g.T >= BM ? BM / kFsRows : g.T / kFsRows, n_tiles * ((units + 1) / 2),
                g.Abar, g.done, g.x0, g.gxT, g.gA_part, g.gx0, g.hdr};
+    if (kTPair) {
+        p.tblocks = g.T / (2 * BM);
+        p.nchains = n_tiles * g.B;
+    }
     count_launch();
-    auto kern = gemm_scan_bwd_kernel<kS>;
+    auto kern = gemm_scan_bwd_kernel<kS, kTPair>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SSM_ERR_CUDA;
     const int pairs = resident_pairs(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes, Cfg::kThreads);
     if (pairs <= 0) return SSM_ERR_CUDA;
@@ -2137,11 +2330,10 @@ static int launch_gemm_scan_bwd_s(const GemmScanBwd& g, cudaStream_t st) {
 }
 
 int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st) {
-    switch (tc_gemm_scan_group(g.B, g.T, g.H, g.P)) {
-        case 64: return launch_gemm_scan_bwd_s<64>(g, st);
-        case 32: return launch_gemm_scan_bwd_s<32>(g, st);
-        default: return SSM_ERR_SHAPE;
-    }
+    const FusedMode m = fused_mode(g.B, g.T, g.H, g.P);
+    if (m.group == 64) return m.time_pairs ? launch_gemm_scan_bwd_s<64, true>(g, st) : launch_gemm_scan_bwd_s<64, false>(g, st);
+    if (m.group == 32) return launch_gemm_scan_bwd_s<32, false>(g, st);
+    return SSM_ERR_SHAPE;
 }
 
 bool tc_nt_supported(int I, int J) { return (I % tc::BM) == 0 && (J % (tc::BN / 2)) == 0; }

@@ -23,7 +23,7 @@ void launch_pack_operands(int H, int P, bool bf16, const float2* Bbar, const flo
 
 // scan.cu
 // Scratch the scans need for a [B,T,P] problem: a work counter and the partial sums of gAbar.
-size_t scan_scratch_bytes(int B, int T, int P);
+size_t scan_scratch_bytes(int B, int T, int P, int rows_per_seq = 1);   // rows_per_seq = 2: room for launch_gemm_scan_bwd_part
 // Alo (may be NULL): low part of Abar, so that Abar + Alo carries the multiplier to ~48 bits.
 int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu, const uint8_t* done,
                     const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr, void* scratch,
@@ -157,12 +157,12 @@ struct GemmScanBwd {
     const float2* gxT;      // [B, P] or NULL
     const void* x_planes;   // bf16 hi plane [B*T, 2P], then the lo plane
     void* s_planes;         // out: the same layout
-    float2* gA_part;        // out [tc_gemm_scan_bwd_part_rows(B, T), P]
+    float2* gA_part;        // out [tc_gemm_scan_bwd_part_rows(B, T, H, P), P]
     float2* gx0;            // out [B, P] or NULL
     WsHeader* hdr;
 };
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P);
-int tc_gemm_scan_bwd_part_rows(int B, int T);   // rows of gA_part the kernel writes (one per chain of 64 states)
+int tc_gemm_scan_bwd_part_rows(int B, int T, int H, int P);   // rows of gA_part the kernel writes (at most 2 B)
 int launch_gemm_scan_bwd(const GemmScanBwd& g, cudaStream_t st);
 // scan.cu: the same with gA_part placed in `scratch` (as for launch_scan_bwd) and brought down to
 // *gA_rows <= kMaxPartialRows rows at *gA_part_out; the caller sums those.

@@ -281,13 +281,14 @@ struct ScanPlan {
     size_t off_part, off_tmp, total;
 };
 
-ScanPlan plan_scan(int B, int P) {
+// rows_per_seq: rows of partial sums per sequence (2 for the kernel that puts both CTAs of a pair on one sequence)
+ScanPlan plan_scan(int B, int P, int rows_per_seq = 1) {
     ScanPlan s{};
     size_t off = sizeof(ScanCounters);
     s.off_part = off;
-    off += align_up((size_t)B * P * 8, 256);
+    off += align_up((size_t)rows_per_seq * B * P * 8, 256);
     s.off_tmp = off;
-    off += align_up(colsum_tmp_floats(B, 2 * P) * 4, 256);
+    off += align_up(colsum_tmp_floats(rows_per_seq * B, 2 * P) * 4, 256);
     s.total = off;
     return s;
 }
@@ -298,9 +299,9 @@ ScanPlan plan_scan(int B, int P) {
 // thread per state walks them.
 static bool use_stream(int B, int T, int P) { return T >= 8 && scan_stream_supported(B, T, P); }
 
-size_t scan_scratch_bytes(int B, int T, int P) {
+size_t scan_scratch_bytes(int B, int T, int P, int rows_per_seq) {
     (void)T;
-    return align_up(plan_scan(B, P).total, 256);
+    return align_up(plan_scan(B, P, rows_per_seq).total, 256);
 }
 
 int launch_scan_fwd(int B, int T, int P, const float2* Abar, const float2* Alo, const float2* Bu, const uint8_t* done,
@@ -365,14 +366,14 @@ int launch_scan_bwd(int B, int T, int P, const float2* Abar, const float2* Alo, 
 }
 
 int launch_gemm_scan_bwd_part(GemmScanBwd g, void* scratch, const float2** gA_part_out, int* gA_rows, cudaStream_t st) {
-    const ScanPlan s = plan_scan(g.B, g.P);
+    const ScanPlan s = plan_scan(g.B, g.P, 2);
     char* base = (char*)scratch;
     float* part = reinterpret_cast<float*>(base + s.off_part);
     float* tmp = reinterpret_cast<float*>(base + s.off_tmp);
     g.gA_part = reinterpret_cast<float2*>(part);
     if (int rc = launch_gemm_scan_bwd(g, st)) return rc;
     *gA_part_out = reinterpret_cast<const float2*>(
-        launch_reduce_rows(part, tc_gemm_scan_bwd_part_rows(g.B, g.T), 2 * g.P, tmp, kMaxPartialRows, gA_rows, st));
+        launch_reduce_rows(part, tc_gemm_scan_bwd_part_rows(g.B, g.T, g.H, g.P), 2 * g.P, tmp, kMaxPartialRows, gA_rows, st));
     return SSM_OK;
 }
 

@@ -73,7 +73,9 @@ def test_plane_path_shapes_fp32(B, T, H, P):
 @pytest.mark.parametrize("B,T,H,P", [(81, 128, 256, 128), (150, 256, 256, 64), (76, 384, 512, 128),
                                      (301, 64, 256, 128), (601, 32, 256, 128), (2403, 16, 256, 64),
                                      # chains of 64 states would occupy at most half of the CTA pairs: chains of 32 states
-                                     (17, 256, 256, 256), (33, 64, 256, 256), (130, 16, 256, 256), (33, 128, 512, 128)])
+                                     (33, 64, 256, 256), (130, 16, 256, 256), (33, 128, 512, 128),
+                                     # few long sequences: both CTAs of a pair on one sequence, tile by tile in turn
+                                     (17, 256, 256, 256), (8, 768, 256, 512), (15, 512, 512, 256), (16, 2048, 256, 256)])
 def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
     # Enough (sequence, 64 states) chains and T a multiple of 128, or T = 16, 32, 64 (a 128-row tile
     # then holds whole sequences; odd B leaves the last tile ragged): the input projection and the
@@ -85,6 +87,10 @@ def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
         d["done"][-1, -1] = 1
         d["done"][1, min(127, T - 1)] = 1   # last row of a tile
         d["done"][2, 128 % T] = 1           # first row of a tile
+        if T >= 512:
+            d["done"][3, 255] = 1           # last row of a pair of tiles
+            d["done"][4, 256] = 1           # first row of the next pair
+            d["done"][5, 300:400] = 1       # a tile and its neighbour full of flags
     run(w, with_x0=True, with_gxT=True, mutate=flags)
     run(I.small_variant(w, p_done=0.0))
 
