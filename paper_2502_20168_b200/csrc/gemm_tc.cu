@@ -11,7 +11,8 @@
 //    planes of both operands (fp32-accurate results, see planes.cu).  Epilogues: fp32 store; bf16
 //    acc + diag * skip; the same with column sums of skip * dot; fp32 store with a gated bf16 result.
 //  * gemm_scan_fwd_kernel / gemm_scan_bwd_kernel: the pair kernel with the scan of Sec. III-B (and its
-//    adjoint) in the epilogue, so that Bu and g_x never reach memory.
+//    adjoint) in the epilogue, so that Bu and g_x never reach memory.  The CTAs of a pair take two
+//    sequences, or (kTPair) alternate tiles of one.
 //  * gemm_tc_nt_kernel / gemm_tc_nt_pair_kernel: part[s, i, j] = sum_{m in slice s} A[m, i] * Bm[m, j]
 //    (both operands contiguous in the output index, i.e. MN-major), split over the B*T rows: the weight
 //    gradients.
@@ -797,19 +798,27 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // eighth of the rows) reads its 16 rows into registers and folds them with packed fp32x2
 // multiply-adds - the first group from the carried state, the others from zero - and the groups
 // are joined as in the streaming scan kernels; (3) it folds again and writes the hi and lo bf16
-// halves of its results straight to global memory (a warp writes 256 contiguous bytes per row and
-// plane), so the shared-memory tile is free for the next drain as soon as everybody has read it.
+// halves of its results into its row group's part of the tile (everybody has read the tile by
+// then), which one lane per row group hands to the TMA unit (8-byte global stores from the
+// threads themselves measured 5 % slower).
 // T is a multiple of 128, or 16, 32 or 64: then a tile holds 128 / T whole sequences, a chain is one
 // tile, and every row group that begins a sequence starts from that sequence's initial state.
+// kTPair (few long sequences, T a multiple of 256): both CTAs of a pair walk ONE sequence, CTA 0 its
+// even tiles and CTA 1 its odd ones, which gives twice the chains at the full tile size.  Every row
+// group then folds from zero; the last row group joins the groups' results into the tile's own
+// contribution, waits for the state that enters the tile (written into this CTA's shared memory by
+// the peer, two slots and two barriers in turn), adds Abar^128 times that state unless a flag cuts
+// it off, and stores the result into the peer's shared memory: one multiply-add per tile and CTA
+// lies between receiving a state and passing it on.
 struct FsParams {
     int B, T, P;
     int n_tiles;      // state groups: P / kS
     int k_blocks;     // H / 64
-    int tblocks;      // tiles per chain: T / 128, or 1
+    int tblocks;      // tiles a CTA walks per chain: T / 128, or 1; kTPair: T / 256
     int unit_rows;    // rows of a chain: T, or 128 when T < 128
     int n_units;      // chains per state group: B, or ceil(B * T / 128)
     int gps;          // row groups per sequence inside a tile: 8, or T / 16
-    int nchains;      // n_tiles * ceil(n_units / 2)
+    int nchains;      // n_tiles * ceil(n_units / 2); kTPair: n_tiles * B
     const float2* Abar;
     const uint8_t* done;
     const float2* x0;
@@ -1289,21 +1298,23 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 // s_t conj(x_{t-1}) to its sums and writes the hi / lo halves of s_t to the same place, which
 // then leaves through the TMA unit as in the forward kernel.  The sums stay in registers for the
 // whole chain and are added over the row groups at its end: one entry of gA_part per (sequence,
-// state), each written once.  T must be a multiple of 128.
+// state), each written once.  T as for the forward kernel.  kTPair as there, run backwards: CTA 1
+// holds the later tile of a pair of tiles, the first row group passes s of the tile's first row
+// on, and each CTA writes its own row of gA_part (two per sequence).
 struct FbParams {
     int B, T, P;
     int n_tiles;      // state groups: P / kS
     int k_blocks;     // H / 64
-    int tblocks;      // tiles per chain: T / 128, or 1
+    int tblocks;      // tiles a CTA walks per chain: T / 128, or 1; kTPair: T / 256
     int unit_rows;    // rows of a chain: T, or 128 when T < 128 (a tile then holds 128 / T whole sequences)
     int n_units;      // chains per state group: B, or ceil(B * T / 128)
     int gps;          // row groups per sequence inside a tile: 8, or T / 16
-    int nchains;      // n_tiles * ceil(n_units / 2)
+    int nchains;      // n_tiles * ceil(n_units / 2); kTPair: n_tiles * B
     const float2* Abar;
     const uint8_t* done;
     const float2* x0;     // [B, P] or NULL
     const float2* gxT;    // [B, P] or NULL
-    float2* gA_part;      // [n_units, P]: one row of sums per chain
+    float2* gA_part;      // [n_units, P]: one row of sums per chain; kTPair: [2 B, P], row 2 b + CTA rank
     float2* gx0;          // [B, P] or NULL
     WsHeader* hdr;
 };
