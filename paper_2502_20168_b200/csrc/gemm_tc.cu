@@ -1016,6 +1016,14 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t peer_ring = map_to_cta(smem_u32(&carry_ring[0][0]), rank ^ 1u);
         const uint32_t peer_bar = map_to_cta(smem_u32(&carry_bar[0]), rank ^ 1u);
         bool ok = true;
+        // The flag of this thread's row, loaded one tile ahead (the load's latency would otherwise stand at the
+        // head of every tile).
+        auto flag_of = [&](int chain, int tb) {
+            if (!p.done || te >= BM || chain >= p.nchains) return false;
+            const int m = row_of(chain, tb) + te;
+            return seq_of(chain) < p.n_units && m < M && p.done[(size_t)m] != 0;
+        };
+        bool flag_next = flag_of(pair, 0);
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
             const bool has_seq = b < p.n_units;
@@ -1067,10 +1075,10 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             for (int tb = 0; tb < p.tblocks; ++tb) {
                 const int m0 = row_of(chain, tb);
                 if (p.done && te < BM) {
-                    const bool f = has_seq && m0 + te < M && p.done[(size_t)m0 + te] != 0;
-                    const uint32_t mk = __ballot_sync(0xffffffffu, f);
+                    const uint32_t mk = __ballot_sync(0xffffffffu, flag_next);
                     if (lane == 0) masks[te >> 5] = mk;
                 }
+                flag_next = tb + 1 < p.tblocks ? flag_of(chain, tb + 1) : flag_of(chain + npairs, 0);
                 (void)mbar_wait(s.tmem_full(acc), acc_phase, s.abort_flag);
                 if (group_leader) tma_store_wait_read();   // this row group's results of the previous tile have left shared memory
                 epi_sync();   // flags visible, tile free (nobody reads the previous one any more); also:
