@@ -177,6 +177,19 @@ def test_forward_backward_twice_is_bitwise_repeatable_and_workspace_reusable():
     second = buf.results()
     for k in ("y", "du", "dB", "dC", "dLambda", "dDelta", "dD"):
         assert np.array_equal(first[k], second[k]), k
+    # Few long sequences, bf16: the two CTAs of a pair hand the state to each other tile by tile; the values
+    # handed over do not depend on which of them runs ahead.  Five runs, all equal to the first.
+    d = I.draw_layer(I.Workload("rep_pairs", B=16, T=1024, H=256, P=256, io_dtype="bf16", p_done=0.003, seed=11),
+                     with_x0=True, with_gxT=True)
+    buf = harness.LayerBuffers(d, "bf16", with_x0=True, with_gxT=True)
+    buf.forward(); buf.backward()
+    first = buf.results()
+    for _ in range(4):
+        buf.forward(); buf.backward()
+        torch.cuda.synchronize()
+        again = buf.results()
+        for k in ("y", "xT", "du", "dx0", "dB", "dC", "dLambda", "dDelta", "dD"):
+            assert np.array_equal(first[k], again[k]), k
 
 
 def test_layer_step_replays_from_a_cuda_graph():
