@@ -2274,8 +2274,16 @@ static FusedMode fused_mode(int B, int T, int H, int P) {
     // 16 x 1024 0.242 -> 0.229; with 64 of 74 pairs busy (32 sequences) it costs 30 - 50 % in these kernels.
     // Time pairs double the chains at the full tile: 16 x 16384 1.76 -> 1.48 ms, 16 x 1024 0.228 -> 0.212.
     const int narrow_below = SSM_FUSED_NARROW_BELOW > 0 ? SSM_FUSED_NARROW_BELOW : tc::sm_count() / 4 + 1;
-    if (pairs64 >= narrow_below) return {64, false};
-    if (SSM_FUSED_TIME_PAIRS && T % (2 * tc::BM) == 0 && (P / 64) * B >= SSM_FUSED_MIN_PAIRS) return {64, true};
+    const bool tp_ok = SSM_FUSED_TIME_PAIRS && T % (2 * tc::BM) == 0;
+    if (pairs64 >= narrow_below) {
+        // Enough chains either way.  Time pairs give twice the chains at half the length, which fills the last
+        // round of chains better when there are only a few rounds (48 sequences at P = 256: 96 chains take two
+        // rounds on 74 CTA pairs, 192 half-length chains three half-rounds).
+        const int np = tc::sm_count() / 2;
+        const int rounds = (pairs64 + np - 1) / np, half_rounds = (2 * pairs64 + np - 1) / np;
+        return {64, tp_ok && half_rounds < 2 * rounds};
+    }
+    if (tp_ok && (P / 64) * B >= SSM_FUSED_MIN_PAIRS) return {64, true};
     if (pairs64 < SSM_FUSED_MIN_PAIRS) return {0, false};
     return {32, false};
 }

@@ -75,7 +75,9 @@ def test_plane_path_shapes_fp32(B, T, H, P):
                                      # chains of 64 states would occupy at most half of the CTA pairs: chains of 32 states
                                      (33, 64, 256, 256), (130, 16, 256, 256), (33, 128, 512, 128),
                                      # few long sequences: both CTAs of a pair on one sequence, tile by tile in turn
-                                     (17, 256, 256, 256), (8, 768, 256, 512), (15, 512, 512, 256), (16, 2048, 256, 256)])
+                                     (17, 256, 256, 256), (8, 768, 256, 512), (15, 512, 512, 256), (16, 2048, 256, 256),
+                                     # the same with several chains per CTA pair (taken where it fills the last round better)
+                                     (48, 256, 256, 256), (41, 512, 256, 256)])
 def test_fused_projection_and_scan_shapes_bf16(B, T, H, P):
     # Enough (sequence, 64 states) chains and T a multiple of 128, or T = 16, 32, 64 (a 128-row tile
     # then holds whole sequences; odd B leaves the last tile ragged): the input projection and the
