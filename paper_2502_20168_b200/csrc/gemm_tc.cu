@@ -1024,6 +1024,11 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             return seq_of(chain) < p.n_units && m < M && p.done[(size_t)m] != 0;
         };
         bool flag_next = flag_of(pair, 0);
+        // The chain's multipliers are loaded one chain ahead as well (a chain is a single tile when the sequences are short).
+        auto abar_of = [&](int chain, int k) {
+            return chain < p.nchains ? p.Abar[(chain % p.n_tiles) * kS + 2 * sp + k] : make_float2(0.f, 0.f);
+        };
+        float2 a0_next = abar_of(pair, 0), a1_next = abar_of(pair, 1);
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
             const bool has_seq = b < p.n_units;
@@ -1031,7 +1036,9 @@ gemm_scan_fwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const int g0 = sl - sl % p.gps;         // the first row group of this group's sequence in the tile
             const bool from_carry = !kTPair && sl == g0;   // (kTPair: the carried state arrives late; every group joins)
             const int pg = n_tile * kS + 2 * sp;    // the first of this thread's two states
-            const float2 a0 = p.Abar[pg], a1 = p.Abar[pg + 1];
+            const float2 a0 = a0_next, a1 = a1_next;
+            a0_next = abar_of(chain + npairs, 0);
+            a1_next = abar_of(chain + npairs, 1);
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
             f32x2 pr, pi, npi;   // Abar^R by squaring in fp32 (a few 1e-7 relative: the results leave as bf16 pairs)
             f32x2 tr = 0ull, ti = 0ull, nti = 0ull;
@@ -1461,11 +1468,18 @@ gemm_scan_bwd_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
+        // The chain's multipliers are loaded one chain ahead (a chain is a single tile when the sequences are short).
+        auto abar_of = [&](int chain, int k) {
+            return chain < p.nchains ? p.Abar[(chain % p.n_tiles) * kS + 2 * sp + k] : make_float2(0.f, 0.f);
+        };
+        float2 a0_next = abar_of(pair, 0), a1_next = abar_of(pair, 1);
         for (int chain = pair; chain < p.nchains && ok; chain += npairs) {
             const int n_tile = chain % p.n_tiles, b = seq_of(chain);
             const bool has_seq = b < p.n_units;
             const int pg = n_tile * kS + 2 * sp;    // the first of this thread's two states
-            const float2 a0 = cconj(p.Abar[pg]), a1 = cconj(p.Abar[pg + 1]);
+            const float2 a0 = cconj(a0_next), a1 = cconj(a1_next);
+            a0_next = abar_of(chain + npairs, 0);
+            a1_next = abar_of(chain + npairs, 1);
             const f32x2 ar = pack2(a0.x, a1.x), ai = pack2(a0.y, a1.y), nai = pack2(-a0.y, -a1.y);
             f32x2 pr, pi, npi;   // conj(Abar)^R by squaring in fp32
             f32x2 tr = 0ull, ti = 0ull, nti = 0ull;
