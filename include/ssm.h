@@ -149,6 +149,13 @@ int ssm_check_static(void* stream);
  * Forward: discretise, Bu = Bbar u, scan, y = Re(C x) + D u.  u, y are [B,T,H] in
  * io_dtype.  ws keeps the residuals (discretised parameters, states) for the backward. */
 size_t ssm_layer_workspace_bytes(const ssm_shape* shape);
+/* Which kernels ssm_layer_fwd / ssm_layer_bwd take for a shape on the current device, as text in buf
+ * (host only, nothing is launched; at most len - 1 characters and a terminating 0).  The text is
+ * "projections=<tensor-cores|tensor-cores-planes|cuda-cores> scans=<fused|separate>", and for fused scans
+ * " chain_states=<64|32> time_pairs=<0|1>": the states a CTA pair scans together, and whether its two CTAs
+ * share one sequence (few long sequences) or take two.  Returns SSM_OK, SSM_ERR_NULL (buf NULL or len 0)
+ * or the shape's error. */
+int ssm_layer_plan_string(const ssm_shape* shape, char* buf, size_t len);
 int ssm_layer_fwd(const ssm_shape* shape, const ssm_c64* Lambda /*[P]*/, const float* Delta /*[P]*/,
                   const ssm_c64* Bc /*[P,H]*/, const ssm_c64* Cc /*[H,P]*/, const float* D /*[H]*/,
                   const void* u /*[B,T,H] io*/, const uint8_t* done /*[B,T] or NULL*/,

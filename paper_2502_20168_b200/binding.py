@@ -24,7 +24,7 @@ SSM_ERR_WORKSPACE, SSM_ERR_CUDA, SSM_ERR_TIMEOUT = -5, -6, -7
 EXPORTS = (
     "ssm_status_string", "ssm_check", "ssm_discretize", "ssm_discretize_bwd",
     "ssm_scan_workspace_bytes", "ssm_scan_fwd", "ssm_scan_bwd",
-    "ssm_layer_workspace_bytes", "ssm_layer_fwd", "ssm_layer_bwd",
+    "ssm_layer_workspace_bytes", "ssm_layer_plan_string", "ssm_layer_fwd", "ssm_layer_bwd",
     "ssm_launch_count", "ssm_profile_begin", "ssm_profile_end", "ssm_scan_bwd_static", "ssm_check_static",
     "ssm_stack_workspace_bytes", "ssm_stack_fwd", "ssm_stack_bwd",
     "ssm_step_workspace_bytes", "ssm_step_prepare", "ssm_step",
@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.ssm_scan_bwd.argtypes = [S] + [P] * 10 + [c_size_t, P]
     lib.ssm_layer_workspace_bytes.restype = c_size_t
     lib.ssm_layer_workspace_bytes.argtypes = [S]
+    lib.ssm_layer_plan_string.restype = c_int
+    lib.ssm_layer_plan_string.argtypes = [S, ctypes.c_char_p, c_size_t]
     lib.ssm_layer_fwd.restype = c_int
     lib.ssm_layer_fwd.argtypes = [S] + [P] * 11 + [c_size_t, P]
     lib.ssm_layer_bwd.restype = c_int
@@ -202,6 +204,12 @@ def ssm_check_static(stream=None) -> None:
 
 def ssm_layer_workspace_bytes(shape) -> int:
     return int(_lib.ssm_layer_workspace_bytes(byref(shape)))
+
+
+def ssm_layer_plan_string(shape) -> str:
+    buf = ctypes.create_string_buffer(160)
+    _ok(_lib.ssm_layer_plan_string(byref(shape), buf, len(buf)), "ssm_layer_plan_string")
+    return buf.value.decode()
 
 
 def ssm_layer_fwd(shape, Lambda, Delta, Bc, Cc, D, u, done, x0, y, xT, ws, stream=None) -> None:

@@ -1,4 +1,5 @@
 // C-ABI entry points (see include/ssm.h): argument checks, workspace layout, launch order.
+#include <cstdio>
 #include <algorithm>
 
 #include "kernels.h"
@@ -201,6 +202,22 @@ SSM_API int ssm_scan_bwd(const ssm_shape* shape, const ssm_c64* Abar, const uint
 SSM_API size_t ssm_layer_workspace_bytes(const ssm_shape* shape) {
     if (check_shape(shape) != SSM_OK) return 0;
     return plan_layer(*shape).total;
+}
+
+SSM_API int ssm_layer_plan_string(const ssm_shape* shape, char* buf, size_t len) {
+    if (!buf || len == 0) return SSM_ERR_NULL;
+    buf[0] = 0;
+    if (int rc = check_shape(shape)) return rc;
+    const ssm_shape& s = *shape;
+    const LayerPlan p = plan_layer(s);
+    const int group = p.tc ? tc_gemm_scan_group(s.B, s.T, s.H, s.P) : 0;
+    const char* proj = p.tc ? "tensor-cores" : (p.planes ? "tensor-cores-planes" : "cuda-cores");
+    if (group)
+        snprintf(buf, len, "projections=%s scans=fused chain_states=%d time_pairs=%d", proj, group,
+                 tc_gemm_scan_time_pairs(s.B, s.T, s.H, s.P) ? 1 : 0);
+    else
+        snprintf(buf, len, "projections=%s scans=separate", proj);
+    return SSM_OK;
 }
 
 // Discretised parameters and packed projection operands into the workspace.

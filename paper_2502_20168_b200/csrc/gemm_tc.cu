@@ -2302,6 +2302,7 @@ static FusedMode fused_mode(int B, int T, int H, int P) {
     return {32, false};
 }
 int tc_gemm_scan_group(int B, int T, int H, int P) { return fused_mode(B, T, H, P).group; }
+bool tc_gemm_scan_time_pairs(int B, int T, int H, int P) { return fused_mode(B, T, H, P).time_pairs; }
 bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P) { return tc_gemm_scan_group(B, T, H, P) != 0; }
 bool tc_gemm_scan_bwd_supported(int B, int T, int H, int P) { return tc_gemm_scan_group(B, T, H, P) != 0; }
 

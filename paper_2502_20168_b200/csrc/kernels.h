@@ -141,6 +141,8 @@ bool tc_gemm_scan_fwd_supported(int B, int T, int H, int P);
 // States per chain these kernels (forward and backward alike) use for a problem: 64 or 32; 0: not taken.  The
 // hi/lo stacked operands they read are packed for that group size (launch_discretize_pack_tc).
 int tc_gemm_scan_group(int B, int T, int H, int P);
+// Whether these kernels put both CTAs of a pair on one sequence for a problem (few long sequences).
+bool tc_gemm_scan_time_pairs(int B, int T, int H, int P);
 int launch_gemm_scan_fwd(const GemmScanFwd& g, cudaStream_t st);
 
 // g_x projection and reverse scan fused (gemm_tc.cu): s = reverse scan(gy conj(C)) written as the two

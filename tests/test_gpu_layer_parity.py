@@ -249,3 +249,24 @@ def test_backward_results_do_not_depend_on_a_kernel_running_beside_it():
         busy = buf.results()
         for k in ("du", "dLambda", "dDelta", "dB", "dC", "dD"):
             assert np.array_equal(quiet[k], busy[k]), (rep, k)
+
+
+@pytest.mark.parametrize("B,T,H,P,io", [(16, 1024, 256, 256, "bf16"), (80, 128, 256, 128, "bf16"), (4, 256, 256, 256, "bf16"),
+                                        (16, 64, 256, 128, "f32"), (2, 40, 32, 16, "f32")])
+def test_plan_string_names_the_stages_that_run(B, T, H, P, io):
+    """ssm_layer_plan_string against the stages the library's own timers see for the same shape."""
+    import torch
+    from paper_2502_20168_b200 import binding as sb, harness
+    w = I.Workload("plan", B=B, T=T, H=H, P=P, io_dtype=io, seed=3)
+    buf = harness.LayerBuffers(harness.device_drawn(w), io)
+    buf.forward(); buf.backward()
+    torch.cuda.synchronize()
+    sb.ssm_profile_begin()
+    buf.forward(); buf.backward()
+    torch.cuda.synchronize()
+    stages = set(sb.ssm_profile_end())
+    sb.ssm_check(buf.ws)
+    plan = sb.ssm_layer_plan_string(sb.make_shape(B, T, H, P, io))
+    fused = "scans=fused" in plan
+    assert fused == ("gemm_Bu_scan_fwd" in stages) == ("gemm_gx_scan_bwd" in stages), (plan, stages)
+    assert fused != ("scan_fwd" in stages), (plan, stages)
