@@ -17,7 +17,7 @@
 //   3. it folds its rows again from that state and writes the results over the tile, in the
 //      layout of the output; one thread hands the tile to the TMA unit.
 // No CTA ever waits for another one, the result does not depend on scheduling, and a producer
-// warp keeps the next tiles in flight through a ring of kStages shared-memory stages.
+// warp keeps the next tiles in flight through a ring of three or four shared-memory stages.
 //
 // The tensor maps are three-dimensional (2P, T, B): rows past the end of a sequence read as
 // zero and are dropped on store; the adjoint's tile of x_{t-1} starts one row early, and row -1
@@ -33,10 +33,10 @@ using namespace tma;
 
 constexpr int kConsumers = 256;
 constexpr int kThreads = kConsumers + 32;
-constexpr int kStages = 3;
+constexpr int kMaxStages = 4;   // stages of the ring: Args::stages of them are used (3, or 4 for the forward scan of narrow chains)
 constexpr int kMaxRows = 256;   // rows of the tallest tile (limit of a TMA box)
 constexpr int kMaxG = 128;
-constexpr int kFwdRows = 16;    // rows per thread and tile, forward
+constexpr int kFwdRows = 8;     // rows per thread and tile, forward (16 measured 6 % slower on few long sequences, equal elsewhere)
 constexpr int kBwdRows = 8;     // backward: its stages also hold x
 
 struct Args {
@@ -44,6 +44,7 @@ struct Args {
     int G, g_shift;      // states per chain (power of two) and its log2
     int slices, R;       // groups of threads along time; rows per tile
     int ntiles, npg, nchains;
+    int stages;          // stages of the shared-memory ring in use (<= kMaxStages)
     const float2* Abar;
     const float2* Alo;   // low part of Abar as an fp32 pair, or NULL
     const uint8_t* done;
@@ -57,11 +58,11 @@ struct Meta {
 };
 
 struct Shared {
-    uint64_t full[kStages], empty[kStages];
-    Meta meta[kStages];
+    uint64_t full[kMaxStages], empty[kMaxStages];
+    Meta meta[kMaxStages];
     int abort_flag;       // raised by a scanning thread whose wait gave up; read by all after a barrier
     int producer_abort;   // the producer warp's own
-    uint8_t flags[kStages][kMaxRows];
+    uint8_t flags[kMaxStages][kMaxRows];
     float2 agg_e[kConsumers], agg_m[kConsumers], agg_ml[kConsumers];
     float2 carry[2][kMaxG];
     float2 gsum[kConsumers];
@@ -118,7 +119,7 @@ template <> struct TileIO<uint32_t> {
 
 __device__ __forceinline__ void init_shared(Shared& sm) {
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) {
+        for (int i = 0; i < kMaxStages; ++i) {
             mbar_init(smem_u32(&sm.full[i]), 1);
             mbar_init(smem_u32(&sm.empty[i]), 1);
         }
@@ -143,7 +144,7 @@ __device__ __forceinline__ void producer(const Args& k, Shared& sm, uint8_t* sta
         chain = __shfl_sync(0xffffffffu, chain, 0);
         const bool end = chain >= k.nchains;
         const int tiles = end ? 1 : k.ntiles;
-        for (int j = 0; j < tiles; ++j, s = (s + 1 == kStages) ? 0 : s + 1, round += (s == 0)) {
+        for (int j = 0; j < tiles; ++j, s = (s + 1 == k.stages) ? 0 : s + 1, round += (s == 0)) {
             if (round > 0 && !mbar_wait(smem_u32(&sm.empty[s]), (round - 1) & 1, &sm.producer_abort)) return;
             if (end) {
                 if (lane == 0) {
@@ -203,7 +204,7 @@ scan_fwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_in, const 
     const float2 zero2 = make_float2(0.f, 0.f);
     float2 a = zero2, al = zero2, aR = zero2, aRl = zero2, xin = zero2;
     int s = 0, round = 0, s_prev = 0;
-    for (int n = 0;; ++n, s_prev = s, s = (s + 1 == kStages) ? 0 : s + 1, round += (s == 0)) {
+    for (int n = 0;; ++n, s_prev = s, s = (s + 1 == k.stages) ? 0 : s + 1, round += (s == 0)) {
         if (!mbar_wait(smem_u32(&sm.full[s]), round & 1, &sm.abort_flag)) k.hdr->status = SSM_ERR_TIMEOUT;
         consumer_sync();   // the scanning warps leave together or not at all
         if (sm.abort_flag) break;
@@ -354,7 +355,7 @@ scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const _
     const float2 zero2 = make_float2(0.f, 0.f);
     float2 ac = zero2, acl = zero2, aR = zero2, aRl = zero2, cin = zero2, xinit = zero2, g = zero2;
     int s = 0, round = 0, s_prev = 0;
-    for (int n = 0;; ++n, s_prev = s, s = (s + 1 == kStages) ? 0 : s + 1, round += (s == 0)) {
+    for (int n = 0;; ++n, s_prev = s, s = (s + 1 == k.stages) ? 0 : s + 1, round += (s == 0)) {
         if (!mbar_wait(smem_u32(&sm.full[s]), round & 1, &sm.abort_flag)) k.hdr->status = SSM_ERR_TIMEOUT;
         consumer_sync();
         if (sm.abort_flag) break;
@@ -523,7 +524,7 @@ bool make_map3(CUtensorMap* map, const void* base, bool bf16, int B, int T, int 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-Args make_args(int B, int T, int P, int rows, const float2* Abar, const float2* Alo, const uint8_t* done, int* ticket,
+Args make_args(int B, int T, int P, int rows, bool forward, const float2* Abar, const float2* Alo, const uint8_t* done, int* ticket,
                WsHeader* hdr) {
     Args k{};
     k.B = B;
@@ -559,6 +560,10 @@ Args make_args(int B, int T, int P, int rows, const float2* Abar, const float2* 
     k.ntiles = (T + k.R - 1) / k.R;
     k.npg = (P + G - 1) / G;
     k.nchains = B * k.npg;
+    // Narrow chains (128-byte rows: few long sequences) keep one more tile in flight in the forward scan:
+    // 4.8 -> 5.4 TB/s at 16 x 16384, P = 256; with wider chains a fourth stage costs 1 %, and the adjoint, whose
+    // stages also hold x, loses 8 % with four.
+    k.stages = (forward && G <= 16) ? 4 : 3;
     k.Abar = Abar;
     k.Alo = Alo;
     k.done = done;
@@ -585,8 +590,8 @@ int launch_scan_fwd_stream(int B, int T, int P, const float2* Abar, const float2
                            const uint8_t* done, const float2* x0, void* x, bool x_bf16, float2* xT, WsHeader* hdr,
                            int* ticket, cudaStream_t st) {
     using namespace stream;
-    const Args k = make_args(B, T, P, kFwdRows, Abar, Alo, done, ticket, hdr);
-    const size_t smem = (size_t)kStages * k.R * k.G * 8 + 128;
+    const Args k = make_args(B, T, P, kFwdRows, true, Abar, Alo, done, ticket, hdr);
+    const size_t smem = (size_t)k.stages * k.R * k.G * 8 + 128;
     const int grid = k.nchains < kCtasPerSm * sm_count() ? k.nchains : kCtasPerSm * sm_count();
     const size_t plane_bytes = (size_t)B * T * P * 4;
     CUtensorMap mi, o0, o1;
@@ -624,8 +629,8 @@ int launch_scan_bwd_stream(int B, int T, int P, const float2* Abar, const float2
                            const float2* x0, const void* x, bool x_bf16, const float2* gx, const float2* gxT,
                            void* gBu, float2* gx0, float2* part, WsHeader* hdr, int* ticket, cudaStream_t st) {
     using namespace stream;
-    const Args k = make_args(B, T, P, kBwdRows, Abar, Alo, done, ticket, hdr);
-    const size_t smem = (size_t)kStages * 2 * k.R * k.G * 8 + 128;
+    const Args k = make_args(B, T, P, kBwdRows, false, Abar, Alo, done, ticket, hdr);
+    const size_t smem = (size_t)k.stages * 2 * k.R * k.G * 8 + 128;
     const int grid = k.nchains < kCtasPerSm * sm_count() ? k.nchains : kCtasPerSm * sm_count();
     const size_t plane_bytes = (size_t)B * T * P * 4;
     CUtensorMap mg, x0m, x1m, o0, o1;
