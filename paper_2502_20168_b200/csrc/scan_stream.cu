@@ -38,6 +38,8 @@ constexpr int kMaxRows = 256;   // rows of the tallest tile (limit of a TMA box)
 constexpr int kMaxG = 128;
 constexpr int kFwdRows = 8;     // rows per thread and tile, forward (16 measured 6 % slower on few long sequences, equal elsewhere)
 constexpr int kBwdRows = 8;     // backward: its stages also hold x
+constexpr int kBwdRowsLong = 16;   // backward, sequences of kBwdLongT steps or more: one CTA per SM with tiles twice as tall
+constexpr int kBwdLongT = 2048;    // (16 x 16384: 5.15 -> 5.5 TB/s, 64 x 4096: 5.7 -> 6.2; T = 1024 equal; T = 64 9 % slower, T = 16 2.7 x)
 
 struct Args {
     int B, T, P;
@@ -330,13 +332,13 @@ scan_fwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_in, const 
 // gA_part: one row of P sums per sequence, each entry written once (so the sum over rows that
 // follows does not depend on which CTA ran what).
 // ---------------------------------------------------------------------------------------------
-template <int G, typename XS, bool kPair>
+template <int G, typename XS, bool kPair, int kRowsPerThread>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_bwd_stream_kernel(Args k, const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_x0,
                        const __grid_constant__ CUtensorMap tm_x1, const __grid_constant__ CUtensorMap tm_o0,
                        const __grid_constant__ CUtensorMap tm_o1, const float2* __restrict__ x0,
                        const float2* __restrict__ gxT, float2* __restrict__ gA_part, float2* __restrict__ gx0) {
-    constexpr int r = kBwdRows, slices = kConsumers / G, R = slices * r;
+    constexpr int r = kRowsPerThread, slices = kConsumers / G, R = slices * r;
     constexpr uint32_t tile_bytes = (uint32_t)R * G * 8, stage_bytes = 2 * tile_bytes;
     extern __shared__ uint8_t stream_raw[];
     __shared__ Shared sm;
@@ -629,7 +631,8 @@ int launch_scan_bwd_stream(int B, int T, int P, const float2* Abar, const float2
                            const float2* x0, const void* x, bool x_bf16, const float2* gx, const float2* gxT,
                            void* gBu, float2* gx0, float2* part, WsHeader* hdr, int* ticket, cudaStream_t st) {
     using namespace stream;
-    const Args k = make_args(B, T, P, kBwdRows, false, Abar, Alo, done, ticket, hdr);
+    const bool tall = T >= kBwdLongT;
+    const Args k = make_args(B, T, P, tall ? kBwdRowsLong : kBwdRows, false, Abar, Alo, done, ticket, hdr);
     const size_t smem = (size_t)k.stages * 2 * k.R * k.G * 8 + 128;
     const int grid = k.nchains < kCtasPerSm * sm_count() ? k.nchains : kCtasPerSm * sm_count();
     const size_t plane_bytes = (size_t)B * T * P * 4;
@@ -647,9 +650,15 @@ int launch_scan_bwd_stream(int B, int T, int P, const float2* Abar, const float2
     count_launch();
 #define SSM_LAUNCH_G(GG, XS, PAIR)                                                                 \
     do {                                                                                           \
-        auto kern = scan_bwd_stream_kernel<GG, XS, PAIR>;                                          \
-        if (!set_smem(kern, smem)) return SSM_ERR_CUDA;                                            \
-        kern<<<grid, kThreads, smem, st>>>(k, mg, x0m, x1m, o0, o1, x0, gxT, part, gx0);           \
+        if (tall) {                                                                                \
+            auto kern = scan_bwd_stream_kernel<GG, XS, PAIR, kBwdRowsLong>;                        \
+            if (!set_smem(kern, smem)) return SSM_ERR_CUDA;                                        \
+            kern<<<grid, kThreads, smem, st>>>(k, mg, x0m, x1m, o0, o1, x0, gxT, part, gx0);       \
+        } else {                                                                                   \
+            auto kern = scan_bwd_stream_kernel<GG, XS, PAIR, kBwdRows>;                            \
+            if (!set_smem(kern, smem)) return SSM_ERR_CUDA;                                        \
+            kern<<<grid, kThreads, smem, st>>>(k, mg, x0m, x1m, o0, o1, x0, gxT, part, gx0);       \
+        }                                                                                          \
     } while (0)
 #define SSM_LAUNCH(XS, PAIR)                                                                       \
     do {                                                                                           \

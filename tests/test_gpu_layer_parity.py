@@ -54,7 +54,9 @@ def test_ragged_shapes_with_resets_x0_and_gxT(io, B, T, H, P):
 @pytest.mark.parametrize("B,T,H,P", [(1, 1, 256, 128), (2, 100, 256, 128), (3, 333, 512, 128),
                                      (5, 77, 256, 384), (700, 66, 256, 128),
                                      # H a multiple of 128 only: the last 256-column tile of y and du is half empty
-                                     (3, 200, 384, 128), (90, 128, 128, 64), (400, 96, 384, 192)])
+                                     (3, 200, 384, 128), (90, 128, 128, 64), (400, 96, 384, 192),
+                                     # long sequences, too few for the fused kernels: the streaming scans' tall reverse tiles, bf16 planes
+                                     (2, 2304, 256, 128), (3, 2100, 256, 64)])
 def test_tensor_core_path_shapes_bf16(B, T, H, P):
     # tile-sized H and P take the tcgen05 projections; B*T is ragged against the 128-row tiles
     w = I.Workload("tc", B=B, T=T, H=H, P=P, io_dtype="bf16", p_done=0.02, seed=B + T)
