@@ -326,11 +326,15 @@ struct TnParams {
 //          bf16 slab leaves by TMA, both as 32 x 32 boxes with the 64-byte swizzle, so a lane reads
 //          and writes its own 64-byte row without bank conflicts and nothing passes through the
 //          load/store path to global memory.  `skip_phase`: the warp's barrier parities (bit b).
+//          With next_m0 >= 0 (the tile this warp drains next) a buffer that has been read is refilled with the next
+//          tile's first slabs, so that they have arrived when that tile starts; *skip_ahead says whether the
+//          tile now starting found its first slabs requested already.
 template <int kEpi, bool kSplitW>
 __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, const CUtensorMap* tmOut,
                                               const CUtensorMap* tmSkip, const CUtensorMap* tmGate, int warp, int lane,
                                               int m0, int n_out0, int acc, uint32_t acc_phase, uint32_t tmem_base,
-                                              uint32_t& skip_phase) {
+                                              uint32_t& skip_phase, int next_m0 = -1, int next_n_out0 = 0,
+                                              bool* skip_ahead = nullptr) {
     constexpr int kOutCols = kSplitW ? BN / 2 : BN;
     const int q = warp & 3;             // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;   // which half of the tile's columns this warp drains
@@ -379,13 +383,18 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
     uint8_t* skb = s.skipbuf + (size_t)w * (kDot ? 8192 : 4096);   // two 2 KB skip tiles (then two dot tiles)
     const uint32_t sbar[2] = {s.skip_full(2 * w), s.skip_full(2 * w + 1)};
     const int swz = (lane >> 1) & 3;               // 64-byte swizzle: chunk c of row `lane` sits at chunk c ^ swz
-    auto fetch_skip = [&](int sl) {
+    auto fetch_skip_at = [&](int sl, int n_first, int row_first) {
         const int b = sl & 1;
         mbar_expect_tx(sbar[b], kDot ? 4096 : 2048);
-        tma_load_2d(smem_u32(skb + b * 2048), tmSkip, sbar[b], n_out0 + (slab0 + sl) * 32, row0);
-        if (kDot) tma_load_2d(smem_u32(skb + 4096 + b * 2048), tmGate, sbar[b], n_out0 + (slab0 + sl) * 32, row0);
+        tma_load_2d(smem_u32(skb + b * 2048), tmSkip, sbar[b], n_first + (slab0 + sl) * 32, row_first);
+        if (kDot) tma_load_2d(smem_u32(skb + 4096 + b * 2048), tmGate, sbar[b], n_first + (slab0 + sl) * 32, row_first);
     };
-    if (lane == 0) {
+    auto fetch_skip = [&](int sl) { fetch_skip_at(sl, n_out0, row0); };
+    static_assert(kSlabs % 2 == 0, "slab s of the next tile takes the buffer of slab s of this one");
+    const bool ahead = skip_ahead && *skip_ahead;   // this tile's first two slabs were requested while the last one was drained
+    const bool prefetch_next = kEpi != 2 && skip_ahead && next_m0 >= 0;
+    if (skip_ahead) *skip_ahead = prefetch_next;
+    if (lane == 0 && !ahead) {
         fence_async_smem();   // (the lanes' reads of the previous tile's last slabs: fenced and joined there)
         fetch_skip(0);
         if (kSlabs > 1) fetch_skip(1);
@@ -476,9 +485,14 @@ __device__ __forceinline__ bool tn_drain_tile(const Smem& s, const TnParams& p, 
         // kernel shared the SMs and the skip rows came from L2).
         fence_async_smem();
         __syncwarp();
-        if (lane == 0 && sl + 2 < kSlabs) {
-            fence_async_smem();
-            fetch_skip(sl + 2);
+        if (lane == 0) {
+            if (sl + 2 < kSlabs) {
+                fence_async_smem();
+                fetch_skip(sl + 2);
+            } else if (prefetch_next) {   // the next tile's slab sl + 2 - kSlabs (0 or 1) into the buffer just read
+                fence_async_smem();
+                fetch_skip_at(sl + 2 - kSlabs, next_n_out0, next_m0 + q * 32);
+            }
         }
         uint4 o[4];
 #pragma unroll
@@ -751,10 +765,13 @@ gemm_tc_tn_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         int acc = 0;
         uint32_t acc_phase = 0, skip_phase = 0;
         bool ok = true;
+        bool skip_ahead = false;
         for (int tile = pair; tile < total && ok; tile += npairs) {
             const int m0 = (tile / p.n_tiles) * (2 * BM) + (int)rank * BM, n_out0 = (tile % p.n_tiles) * kOutCols;
+            const int nxt = tile + npairs;
+            const int next_m0 = nxt < total ? (nxt / p.n_tiles) * (2 * BM) + (int)rank * BM : -1;
             if (!(ok = tn_drain_tile<kEpi, kSplitW>(s, p, &tmOut, &tmSkip, &tmGate, warp, lane, m0, n_out0, acc, acc_phase, tmem_base,
-                                                    skip_phase)))
+                                                    skip_phase, next_m0, nxt < total ? (nxt % p.n_tiles) * kOutCols : 0, &skip_ahead)))
                 break;
             tc_fence_before();
             mbar_arrive_cluster(leader_empty0 + 8u * acc);
