@@ -56,12 +56,12 @@ STAGE_MODEL = {
 # moves this figure times its timesteps.  They hold for H = 512, P = 256, bf16 I/O, T = 1024; an entry is None where
 # no capture of the kernel as it stands exists.
 NCU_TRAFFIC_PER_TIMESTEP = {
-    "gemm_Bu_scan_fwd": 351.6e6 / 131072,
-    "gemm_gx_scan_bwd": 645.8e6 / 131072,
-    "gemm_y": 377.4e6 / 131072,
-    "gemm_du": 534.7e6 / 131072,
-    "gemm_gBbar": 406.7e6 / 131072,
-    "gemm_gC": 408.2e6 / 131072,
+    "gemm_Bu_scan_fwd": 349.9e6 / 131072,
+    "gemm_gx_scan_bwd": 644.7e6 / 131072,
+    "gemm_y": 379.7e6 / 131072,
+    "gemm_du": 546.9e6 / 131072,
+    "gemm_gBbar": 406.5e6 / 131072,
+    "gemm_gC": 406.6e6 / 131072,
     "scan_fwd": None,
     "scan_bwd": None,
     "gemm_Bu": None,
